@@ -1,0 +1,303 @@
+"""Pins for the oracle's attention, score update, routing and ledger.
+
+Each check is against something other than the oracle itself: a textbook softmax written with a library
+routine, closed forms, a brute-force sort, and the invariants the paper states."""
+
+import hashlib
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import softmax
+
+from oracle import (
+    LEDGER_ACTIVE,
+    LEDGER_DORMANT,
+    LEDGER_NONE,
+    TIER_AGED,
+    TIER_EVICTED,
+    TIER_FULL,
+    TIER_OPEN,
+    TIER_QUANT,
+    OracleConfig,
+    UnitOracle,
+    accessible_attention,
+    round_to_dtype,
+    tier_capacities,
+    window_bytes,
+)
+from paper_2608_05326_b200 import workloads as wlmod
+
+
+def _full_attention_reference(q, k, v, scale):
+    """Textbook GQA softmax attention with library routines (scipy softmax, einsum)."""
+    hq, d = q.shape
+    hkv = k.shape[0]
+    kk = np.repeat(k, hq // hkv, axis=0)
+    vv = np.repeat(v, hq // hkv, axis=0)
+    p = softmax(np.einsum("hd,hnd->hn", q, kk) * scale, axis=-1)
+    return np.einsum("hn,hnd->hd", p, vv), p
+
+
+def _rand_T(rng, shape, dtype, scale=1.0):
+    return round_to_dtype(rng.standard_normal(shape) * scale, dtype)
+
+
+# ------------------------------------------------------------------------------ attention
+def test_attention_matches_textbook_softmax():
+    rng = np.random.default_rng(10)
+    q = rng.standard_normal((8, 64))
+    k = rng.standard_normal((2, 300, 64))
+    v = rng.standard_normal((2, 300, 64))
+    out, p = accessible_attention(q, k, v, 0.125)
+    ref_out, ref_p = _full_attention_reference(q, k, v, 0.125)
+    assert np.allclose(out, ref_out, rtol=1e-12, atol=1e-13)
+    assert np.allclose(p, ref_p, rtol=1e-12, atol=1e-15)
+
+
+def test_attention_closed_forms():
+    rng = np.random.default_rng(11)
+    q = rng.standard_normal((4, 32))
+    key = rng.standard_normal((1, 1, 32))
+    k = np.repeat(key, 50, axis=1)  # all keys equal -> uniform probabilities
+    v = rng.standard_normal((1, 50, 32))
+    out, p = accessible_attention(q, k, v, 0.3)
+    assert np.allclose(p, 1.0 / 50)
+    assert np.allclose(out, np.broadcast_to(v.mean(axis=1), (4, 32)))
+    # one key aligned with the query and huge: the output is that token's value
+    k2 = rng.standard_normal((1, 50, 32)) * 0.01
+    k2[0, 17] = q[0] * 1000
+    out2, p2 = accessible_attention(q[:1], k2, v, 1.0)
+    assert p2[0, 17] > 1 - 1e-12 and np.allclose(out2[0], v[0, 17])
+    # GQA: head h reads KV head h // (H_q / H_kv)
+    k3 = rng.standard_normal((2, 20, 32))
+    v3 = rng.standard_normal((2, 20, 32))
+    out3, _ = accessible_attention(q, k3, v3, 0.2)
+    for h in range(4):
+        o1, _ = accessible_attention(q[h:h + 1], k3[h // 2:h // 2 + 1], v3[h // 2:h // 2 + 1], 0.2)
+        assert np.allclose(out3[h], o1[0])
+
+
+# -------------------------------------------------------------------------------- helpers
+def _small_cfg(dtype="fp16", k_f=4, k_q=6, bits=4, hq=4, hkv=2, d=64, w=32, ctx_windows=16, extra=8):
+    return OracleConfig(hq, hkv, d, dtype, w, bits, 32, k_f, k_q, (ctx_windows + extra) * w, aged_windows=2)
+
+
+def _prefilled(cfg, rng, ctx_windows=16, scores=None):
+    ctx = ctx_windows * cfg.window
+    k = _rand_T(rng, (cfg.n_kv_heads, ctx, cfg.head_dim), cfg.dtype)
+    v = _rand_T(rng, (cfg.n_kv_heads, ctx, cfg.head_dim), cfg.dtype)
+    if scores is None:
+        scores = rng.random(ctx_windows).astype(np.float32)
+    u = UnitOracle(cfg)
+    u.prefill_assign(k, v, scores)
+    return u, k, v, scores
+
+
+# ------------------------------------------------- (a) everything in full precision = full attention
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_full_budget_equals_brute_force_attention(dtype):
+    rng = np.random.default_rng(12)
+    cfg = _small_cfg(dtype, k_f=64, k_q=4)
+    u, k, v, _ = _prefilled(cfg, rng)
+    assert u.tier_counts()["full"] == 16 and u.tier_counts()["quant"] == 0
+    ks, vs = [k], [v]
+    for t in range(40):
+        q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), dtype)
+        kn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), dtype)
+        vn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), dtype)
+        ks.append(kn[:, None]); vs.append(vn[:, None])
+        out, mass = u.decode_attn(q, kn, vn)
+        ref, p = _full_attention_reference(q, np.concatenate(ks, 1), np.concatenate(vs, 1), cfg.scale)
+        assert np.array_equal(out, round_to_dtype(ref, dtype))
+        n_tok = p.shape[1]
+        ref_mass = np.add.reduceat(p.sum(0), np.arange(0, n_tok, cfg.window))
+        assert np.allclose(mass[: len(ref_mass)], ref_mass, rtol=1e-12, atol=1e-15)
+        if t % 8 == 7:
+            u.rebalance()
+            assert u.tier_counts()["evicted"] == 0 and u.tier_counts()["quant"] == 0
+
+
+# --------------------------------------------------------- (c) mass conservation, (d) budgets
+def test_mass_sums_to_heads_times_steps_and_budgets_hold():
+    wl = wlmod.config(0)
+    k, v = wlmod.gen_prompt_kv(wl, 0)
+    k = k.double().numpy(); v = v.double().numpy()
+    cfg = OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits,
+                       wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context)
+    scores = wlmod.place_planted(wlmod.synthetic_window_scores(wl, 0), wlmod.planted_windows(wl, 0),
+                                 wl.fp_budget_windows, wl.q_budget_windows)
+    u = UnitOracle(cfg)
+    u.prefill_assign(k, v, scores.numpy())
+    base = u.importance.sum()
+    assert u.tier_counts() == {"open": 0, "aged": 0, "full": 8, "quant": 16, "evicted": 40}
+    q_all = wlmod.gen_queries(wl, 0, torch.from_numpy(k), scores).double().numpy()
+    kn, vn = wlmod.gen_new_kv(wl, 0)
+    evicted_before = set()
+    for t in range(wl.steps):
+        out, mass = u.decode_attn(q_all[t], kn[t].double().numpy(), vn[t].double().numpy())
+        assert abs(mass.sum() - cfg.n_q_heads) < 1e-9
+        assert abs(u.importance.sum() - base - cfg.n_q_heads * (t + 1)) < 1e-7
+        u.rebalance()
+        c = u.tier_counts()
+        assert c["full"] <= cfg.fp_budget_windows and c["quant"] <= cfg.q_budget_windows
+        assert c["aged"] == 0
+        ev = set(np.flatnonzero(u.tier == TIER_EVICTED).tolist())
+        assert evicted_before <= ev  # evicted windows never return
+        evicted_before = ev
+        # physical pools: no page held twice, occupancy within the pool
+        fp_held = u.fp_page[u.fp_page >= 0]
+        q_held = u.q_page[u.q_page >= 0]
+        assert len(set(fp_held.tolist())) == len(fp_held) <= cfg.fp_pool_pages
+        assert len(set(q_held.tolist())) == len(q_held) <= cfg.q_pool_pages
+        for w in range(u.n_windows):
+            assert (u.fp_page[w] >= 0) == (u.tier[w] in (TIER_FULL, TIER_AGED, TIER_OPEN))
+            assert (u.q_page[w] >= 0) == (u.ledger_flag[w] != LEDGER_NONE)
+            assert (u.tier[w] == TIER_QUANT) == (u.ledger_flag[w] == LEDGER_ACTIVE)
+    # the drifting queries force recoveries from the quantized tier
+    assert u.stats["promotions"] > 0 and u.stats["deletions"] > 40
+
+
+# --------------------------------------------------------------------------------- routing
+def test_routing_matches_brute_force_sort():
+    rng = np.random.default_rng(13)
+    for trial in range(20):
+        cfg = _small_cfg(k_f=int(rng.integers(1, 6)), k_q=int(rng.integers(1, 8)))
+        scores = rng.integers(0, 6, 16).astype(np.float32)  # many ties
+        u, *_ = _prefilled(cfg, rng, scores=scores)
+        ranked = sorted(range(16), key=lambda w: (-float(scores[w]), w))
+        exp_f = set(ranked[: cfg.fp_budget_windows])
+        exp_q = set(ranked[cfg.fp_budget_windows: cfg.fp_budget_windows + cfg.q_budget_windows])
+        assert set(np.flatnonzero(u.tier == TIER_FULL).tolist()) == exp_f
+        assert set(np.flatnonzero(u.tier == TIER_QUANT).tolist()) == exp_q
+        assert set(np.flatnonzero(u.tier == TIER_EVICTED).tolist()) == set(range(16)) - exp_f - exp_q
+        # prefill page order: ascending window index takes ascending page ids
+        assert [int(u.fp_page[w]) for w in sorted(exp_f)] == list(range(len(exp_f)))
+        assert [int(u.q_page[w]) for w in sorted(exp_q)] == list(range(len(exp_q)))
+
+
+def test_rebalance_is_idempotent_and_small_pools_keep_everything_full():
+    rng = np.random.default_rng(14)
+    cfg = _small_cfg(k_f=3, k_q=5)
+    u, *_ = _prefilled(cfg, rng)
+    snap = (u.tier.copy(), u.fp_page.copy(), u.q_page.copy(), u.ledger_flag.copy(), dict(u.stats))
+    u.rebalance()
+    assert np.array_equal(snap[0], u.tier) and np.array_equal(snap[1], u.fp_page)
+    assert np.array_equal(snap[2], u.q_page) and np.array_equal(snap[3], u.ledger_flag)
+    assert snap[4] == u.stats
+    cfg2 = _small_cfg(k_f=20, k_q=5)
+    u2, *_ = _prefilled(cfg2, rng)
+    assert u2.tier_counts()["full"] == 16
+
+
+def test_scores_are_ranked_in_float32():
+    """Two float64 scores that collapse to the same float32 are a tie: the lower index wins."""
+    rng = np.random.default_rng(15)
+    cfg = _small_cfg(k_f=1, k_q=1)
+    u, *_ = _prefilled(cfg, rng, scores=np.zeros(16, np.float32))
+    u.importance[:] = 0.0
+    u.importance[5] = 1.0
+    u.importance[9] = 1.0 + 1e-12
+    # only windows 0 (F) and 1 (Q) are still candidates; give them the colliding scores instead
+    u.importance[0] = 1.0
+    u.importance[1] = 1.0 + 1e-12
+    u.rebalance()
+    assert u.tier[0] == TIER_FULL and u.tier[1] == TIER_QUANT
+
+
+# ---------------------------------------------------------------------------------- ledger
+def _ledger_hash(e):
+    m = hashlib.sha256()
+    for key in ("k_codes", "k_s", "k_z", "v_codes", "v_s", "v_z"):
+        m.update(np.ascontiguousarray(e[key]).tobytes())
+    return m.hexdigest()
+
+
+def test_write_once_ledger_and_promotion_invariance():
+    rng = np.random.default_rng(16)
+    cfg = _small_cfg("bf16", k_f=2, k_q=3, bits=2)
+    scores = np.arange(16, 0, -1).astype(np.float32)  # window 0 highest
+    u, k, v, _ = _prefilled(cfg, rng, scores=scores)
+    assert list(np.flatnonzero(u.tier == TIER_FULL)) == [0, 1]
+    assert list(np.flatnonzero(u.tier == TIER_QUANT)) == [2, 3, 4]
+    h2 = _ledger_hash(u.ledger[2])
+    q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), "bf16")
+    u.decode_attn(q)  # fixed-context step, window 2 read from its codes
+    u.importance[:16] = scores  # undo the score change, then lift window 2 to the top
+    u.importance[2] = 100.0
+    u.rebalance()
+    assert u.tier[2] == TIER_FULL and u.ledger_flag[2] == LEDGER_DORMANT and u.q_page[2] >= 0
+    assert u.tier[1] == TIER_QUANT and u.ledger_flag[1] == LEDGER_ACTIVE  # window 1 demoted, quantized now
+    assert u.stats["promotions"] == 1 and u.stats["quantizations"] == 4
+    # the promoted copy is the dequantized approximation, not the original values
+    assert not np.array_equal(u.fp[2][0], k[:, 64:96])
+    assert _ledger_hash(u.ledger[2]) == h2
+    # demote window 2 again: reactivation, codes untouched, no new quantization
+    u.importance[2] = 13.5  # between windows 1 and 3: back into the quantized tier
+    u.importance[1] = 100.0
+    u.rebalance()
+    assert u.tier[2] == TIER_QUANT and u.ledger_flag[2] == LEDGER_ACTIVE
+    assert u.stats["reactivations"] == 1 and u.stats["quantizations"] == 4
+    assert _ledger_hash(u.ledger[2]) == h2
+    assert u.tier[1] == TIER_FULL and u.ledger_flag[1] == LEDGER_DORMANT  # back as its own approximation
+    # promotion invariance: swap windows 1 and 2 between the tiers once more.  Both already are
+    # approximations, so no value changes and attention must be bit-identical.
+    out_a, mass_a = u.decode_attn(q)
+    u.importance -= mass_a
+    u.importance[2] = 200.0
+    u.importance[1] = 13.5
+    u.rebalance()
+    assert u.tier[2] == TIER_FULL and u.tier[1] == TIER_QUANT and u.tier[0] == TIER_FULL
+    assert u.stats["quantizations"] == 4 and u.stats["reactivations"] == 2 and u.stats["promotions"] == 3
+    out_b, mass_b = u.decode_attn(q)
+    assert np.array_equal(out_a, out_b) and np.array_equal(mass_a, mass_b)
+
+
+def test_eviction_deletes_ledger_and_is_permanent():
+    rng = np.random.default_rng(17)
+    cfg = _small_cfg(k_f=2, k_q=2)
+    scores = np.arange(16, 0, -1).astype(np.float32)
+    u, *_ = _prefilled(cfg, rng, scores=scores)
+    assert u.tier_counts()["evicted"] == 12
+    # fill one window by appending: it ages and must displace the weakest quantized window
+    for t in range(cfg.window):
+        u.decode_attn(_rand_T(rng, (cfg.n_q_heads, cfg.head_dim), cfg.dtype),
+                      _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype),
+                      _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype))
+    assert u.tier[16] == TIER_AGED
+    u.importance[16] = 1e6
+    victim = 3  # lowest-ranked retained window
+    page = u.q_page[victim]
+    u.rebalance()
+    assert u.tier[16] == TIER_FULL
+    assert u.tier[victim] == TIER_EVICTED and u.ledger_flag[victim] == LEDGER_NONE
+    assert victim not in u.ledger and u.q_owner[page] != victim
+    u.importance[victim] = 1e9  # an evicted window is not a candidate any more, whatever its score
+    u.rebalance()
+    assert u.tier[victim] == TIER_EVICTED
+
+
+def test_open_window_is_attended_and_ages():
+    rng = np.random.default_rng(18)
+    cfg = _small_cfg(k_f=2, k_q=2)
+    u, *_ = _prefilled(cfg, rng)
+    q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), cfg.dtype)
+    kn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+    vn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+    out, mass = u.decode_attn(q, kn, vn)
+    assert u.tier[16] == TIER_OPEN and u.open_fill == 1 and mass[16] > 0
+    assert u.fp_page[16] == 2  # lowest free full-precision page after pages 0 and 1
+    assert sum(a[3] for a in u.accessible()) == 4 * cfg.window + 1
+
+
+# ------------------------------------------------------------------------------ capacities
+def test_tier_capacities_closed_form():
+    cfg = OracleConfig(32, 8, 128, "bf16", 32, 4, 32, 1, 1, 4096)
+    m_f, m_q = window_bytes(cfg)
+    assert (m_f, m_q) == (131072, 40960)
+    assert tier_capacities(100 * m_f, 0.0, m_f, m_q) == (100, 0)
+    assert tier_capacities(100 * m_f, 1.0, m_f, m_q) == (0, 320)
+    k_f, k_q = tier_capacities(10_000_000, 0.7, m_f, m_q)
+    assert (k_f, k_q) == (22, 170)
+    assert k_f * m_f <= 0.3 * 10_000_000 < (k_f + 1) * m_f
+    assert k_q * m_q <= 0.7 * 10_000_000 < (k_q + 1) * m_q
