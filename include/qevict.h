@@ -1,0 +1,204 @@
+/*
+ * qevict.h -- C ABI of the B200 decode hot path of a three-tier, window-granular KV cache.
+ *
+ * What the library computes (paper sections in brackets):
+ *   - per (sequence, layer) the historical KV cache is cut into windows of W tokens; every window is
+ *     Full (stored in the execution datatype), Quantized (stored as low-bit codes, still attended
+ *     to) or Evicted (gone for good)                         [Methodology: Preliminaries, Recoverable
+ *                                                             Cache Hierarchy]
+ *   - a decode step is softmax attention of one query per head over the accessible tokens only,
+ *     grouped-query heads sharing a KV head                  [Preliminaries, attention equation]
+ *   - each step adds to every window the attention probability mass its tokens received, summed
+ *     over the query heads (the cumulative window score)      [Eq. 1]
+ *   - a routing event ranks the candidate windows by score and keeps the best K_f Full, the next
+ *     K_q Quantized and deletes the rest; a window is quantized only on its first demotion, a
+ *     promotion rebuilds it from its codes, a later demotion reuses the codes  [Dynamic Routing and
+ *                                                             Recovery; Migration-Stable
+ *                                                             Quantization; Algorithm 1]
+ *   - K_f and K_q follow from a byte budget                   [tier-capacity equation; memory
+ *                                                             accounting appendix]
+ *
+ * Conventions
+ *   - Every pointer argument says "device" or "host".  Device pointers must be valid on the device
+ *     named in the configuration, 16-byte aligned and contiguous; the caller owns them, the library
+ *     neither frees nor keeps them after the enqueued work has run.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *     enqueue work unless the comment says "synchronises".
+ *   - A "unit" is one (layer, sequence) pair; unit = layer * batch + sequence.  `layer == -1` means
+ *     every layer in one launch; tensors then carry a leading [n_layers] dimension.
+ *   - Errors are returned as qevict_status; a failed call enqueues nothing.  Kernels never trap:
+ *     device-side checks record a code that the synchronising getters report as
+ *     QEVICT_ERR_DEVICE_CHECK.
+ *   - The library holds no global state; one handle must not be used from two threads at once.
+ *   - There is no CPU fallback: without a CUDA device every compute call returns QEVICT_ERR_CUDA.
+ */
+#ifndef QEVICT_H_
+#define QEVICT_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define QEVICT_API __attribute__((visibility("default")))
+#else
+#define QEVICT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qevict_ctx* qevict_handle;
+
+typedef enum {
+  QEVICT_OK = 0,
+  QEVICT_ERR_INVALID_ARG = 1,  /* null pointer, out-of-range value, inconsistent configuration */
+  QEVICT_ERR_BAD_STATE = 2,    /* call order: decode before prefill, prefill twice, rebalance overdue */
+  QEVICT_ERR_NO_MEMORY = 3,    /* caller's device buffer too small, or host allocation failed */
+  QEVICT_ERR_UNSUPPORTED = 4,  /* a shape the kernels are not built for */
+  QEVICT_ERR_CUDA = 5,         /* a CUDA runtime call failed (qevict_last_error has the text) */
+  QEVICT_ERR_DEVICE_CHECK = 6  /* a kernel recorded an internal check failure */
+} qevict_status;
+
+enum { QEVICT_DTYPE_FP16 = 0, QEVICT_DTYPE_BF16 = 1 };
+
+/* window states, as exported by qevict_export_tables */
+enum {
+  QEVICT_TIER_NONE = 0,    /* window index not created yet */
+  QEVICT_TIER_OPEN = 1,    /* recent region: the window being filled by appended tokens */
+  QEVICT_TIER_AGED = 2,    /* recent region: filled, waiting for the next routing event */
+  QEVICT_TIER_FULL = 3,
+  QEVICT_TIER_QUANT = 4,
+  QEVICT_TIER_EVICTED = 5
+};
+/* ledger states */
+enum { QEVICT_LEDGER_NONE = 0, QEVICT_LEDGER_ACTIVE = 1, QEVICT_LEDGER_DORMANT = 2 };
+
+typedef struct {
+  uint32_t struct_size;      /* sizeof(qevict_config) of the caller, for ABI growth */
+  int32_t batch;             /* sequences per layer */
+  int32_t n_layers;
+  int32_t n_q_heads;         /* H_q */
+  int32_t n_kv_heads;        /* H_kv; H_q % H_kv == 0 and H_q / H_kv <= 8 */
+  int32_t head_dim;          /* d: 64 or 128 */
+  int32_t dtype;             /* QEVICT_DTYPE_* : execution datatype of q, k, v, out */
+  int32_t window;            /* W tokens: 32 or 64 */
+  int32_t quant_bits;        /* b: 2 or 4 */
+  int32_t group_size;        /* g: 32 or 64; W % g == 0 and d % g == 0 */
+  int32_t fp_budget_windows; /* K_f per unit */
+  int32_t q_budget_windows;  /* K_q per unit */
+  int32_t max_context;       /* upper bound on prompt + generated tokens; multiple of W */
+  int32_t rebalance_interval_hint; /* decode steps the caller lets pass between routing events; sizes
+                                      the full-precision pages that hold aged windows; 0 => W */
+  float softmax_scale;       /* 0 => 1/sqrt(d) */
+  int32_t device;            /* CUDA device ordinal */
+} qevict_config;
+
+typedef struct {
+  uint64_t promotions;     /* Quantized -> Full (dequantize into a full-precision page) */
+  uint64_t quantizations;  /* first demotions: the only time a window's codes are produced */
+  uint64_t reactivations;  /* Full -> Quantized with a dormant ledger entry: no data moved */
+  uint64_t deletions;      /* windows evicted */
+  uint64_t n_full, n_quant, n_aged, n_open, n_evicted; /* current window counts */
+  uint64_t decode_steps;
+} qevict_stats;
+
+/* Bytes of one Full window and one Quantized window (all KV heads, keys and values), and the tier
+ * capacities K_f = floor((1-q_frac) * hist_bytes / M_f), K_q = floor(q_frac * hist_bytes / M_q)
+ * [tier-capacity equation].  M_q counts packed codes plus one (scale, zero) pair of the execution
+ * datatype per group [memory accounting appendix].  Host arithmetic only; any output pointer may be
+ * NULL.  Only the shape fields of `cfg` are read. */
+QEVICT_API qevict_status qevict_budget_from_bytes(const qevict_config* cfg, uint64_t hist_bytes, double q_frac,
+                                       int32_t* k_f, int32_t* k_q, uint64_t* m_f, uint64_t* m_q);
+
+/* Size of the device buffer qevict_create needs for this configuration (pools, tables, scratch). */
+QEVICT_API qevict_status qevict_workspace_bytes(const qevict_config* cfg, uint64_t* bytes);
+
+/* Build a cache inside `device_mem` (device pointer, 256-byte aligned, `bytes` long, owned by the
+ * caller and kept alive until qevict_destroy).  Clears the tables; synchronises the device once.
+ * The memory is fixed from here on: the pools hold K_f + aged + 1 full-precision pages and
+ * K_q + K_f quantized pages per unit (the extra K_f keep the codes of promoted windows). */
+QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_mem, uint64_t bytes, qevict_handle* out);
+QEVICT_API qevict_status qevict_destroy(qevict_handle h);
+
+/* Prefill initialisation [Methodology: prompt attention initialises the window scores and the first
+ * tier assignment].  For every sequence of `layer`: the prompt is cut into ctx_tokens / W windows,
+ * window w starts with score window_scores[seq][w], one routing event runs, Full windows are copied
+ * and Quantized windows are quantized straight from the prompt, the rest is never stored.
+ *   k, v          device, [batch][H_kv][ctx_tokens][d] in the execution datatype ([n_layers][...] first
+ *                 when layer == -1)
+ *   window_scores device, float32 [batch][ctx_tokens / W]: raw attention mass summed over heads
+ *   ctx_tokens    multiple of W, at most max_context
+ * Once per layer. */
+QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, const void* k, const void* v,
+                                    int32_t ctx_tokens, const float* window_scores, void* stream);
+
+/* One decode step [attention equation; Eq. 1].  If k_new != NULL the new token's key and value
+ * first enter the recent region (the open window); then every query head attends over all accessible
+ * tokens (open, aged, Full and Quantized windows, the latter dequantized in registers) and each
+ * window's score grows by the probability mass it received, summed over the query heads.
+ *   q            device, [batch][H_q][d]
+ *   k_new, v_new device, [batch][H_kv][d], or both NULL (fixed context)
+ *   out          device, [batch][H_q][d]
+ * Returns QEVICT_ERR_BAD_STATE if more filled windows are waiting than the pages sized by
+ * rebalance_interval_hint can hold (call qevict_rebalance first). */
+QEVICT_API qevict_status qevict_decode_attn(qevict_handle h, int32_t layer, const void* q, const void* k_new,
+                                 const void* v_new, void* out, void* stream);
+
+/* The same step with HOST buffers (pageable or pinned): copies q, k_new, v_new to the device, runs the
+ * step, copies `out` back and synchronises the stream. */
+QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer, const void* q_host,
+                                      const void* k_new_host, const void* v_new_host, void* out_host,
+                                      void* stream);
+
+/* One routing event [Algorithm 1].  Candidates = Full, Quantized and aged windows, ranked by score
+ * (float32, higher first, lower window index first among equals); the first K_f become Full, the next
+ * K_q Quantized, the rest Evicted.  Pages are released, then handed out in ascending page id to the
+ * windows that need one in ascending window index; first demotions are quantized, promotions are
+ * dequantized (after the quantizations, because a promotion may receive a page a demotion released);
+ * a demotion with a dormant ledger entry only flips its flag. */
+QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* stream);
+
+/* Counters of one layer (layer == -1: all layers), summed over its sequences.  Synchronises. */
+QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict_stats* out);
+
+/* Tables of one unit, written to DEVICE buffers sized for max_context / W windows (any may be NULL):
+ * n_windows int32[1], tier uint8[], ledger uint8[], fp_page int32[], q_page int32[] (-1 = none),
+ * importance float32[].  Enqueues only. */
+QEVICT_API qevict_status qevict_export_tables(qevict_handle h, int32_t layer, int32_t seq, int32_t* n_windows,
+                                   uint8_t* tier, uint8_t* ledger, int32_t* fp_page, int32_t* q_page,
+                                   float* importance, void* stream);
+
+/* Attention mass of the last decode step per window, DEVICE float32[max_context / W] (0 where the
+ * window was not attended). */
+QEVICT_API qevict_status qevict_export_last_mass(qevict_handle h, int32_t layer, int32_t seq, float* mass, void* stream);
+
+/* Contents of the full-precision page `fp_page` of a unit in plain layout: DEVICE k_out, v_out
+ * [H_kv][W][d] in the execution datatype. */
+QEVICT_API qevict_status qevict_export_fp_page(qevict_handle h, int32_t layer, int32_t seq, int32_t fp_page,
+                                    void* k_out, void* v_out, void* stream);
+
+/* Contents of the quantized page `q_page` of a unit in plain layout, DEVICE buffers:
+ * k_codes, v_codes uint8 [H_kv][W][d] (one code per byte);
+ * k_params [H_kv][W/g][d][2], v_params [H_kv][W][d/g][2] in the execution datatype, (scale, zero). */
+QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, int32_t seq, int32_t q_page,
+                                   uint8_t* k_codes, void* k_params, uint8_t* v_codes, void* v_params,
+                                   void* stream);
+
+/* Tuning: force the number of KV splits per (unit, KV head) of the decode kernel (1..64); 0 restores
+ * the built-in choice, which fills the GPU in whole waves.  Results do not depend on it beyond
+ * floating-point summation order. */
+QEVICT_API qevict_status qevict_set_splits(qevict_handle h, int32_t splits);
+
+/* Number of kernels this handle has launched since creation (host counter). */
+QEVICT_API uint64_t qevict_launch_count(qevict_handle h);
+
+/* Text of the last error on this handle (never NULL). */
+QEVICT_API const char* qevict_last_error(qevict_handle h);
+QEVICT_API const char* qevict_status_string(qevict_status s);
+/* Library version, "major.minor". */
+QEVICT_API const char* qevict_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QEVICT_H_ */

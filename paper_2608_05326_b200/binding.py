@@ -1,0 +1,260 @@
+"""ctypes binding of libqevict.so: the same entry points as include/qevict.h, plus a small convenience
+class that owns the device workspace.  Argument marshalling only -- every step of the path runs in the
+CUDA kernels of the library; there is no fallback of any kind."""
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqevict.so")
+
+QEVICT_OK = 0
+DTYPE_FP16, DTYPE_BF16 = 0, 1
+TIER_NONE, TIER_OPEN, TIER_AGED, TIER_FULL, TIER_QUANT, TIER_EVICTED = range(6)
+LEDGER_NONE, LEDGER_ACTIVE, LEDGER_DORMANT = range(3)
+STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "NO_MEMORY", "UNSUPPORTED", "CUDA", "DEVICE_CHECK"]
+
+
+class QEvictError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("qevict: %s (%s)" % (message, STATUS_NAMES[status] if 0 <= status < 7 else status))
+        self.status = status
+
+
+class qevict_config(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("batch", C.c_int32), ("n_layers", C.c_int32), ("n_q_heads", C.c_int32),
+        ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32), ("window", C.c_int32),
+        ("quant_bits", C.c_int32), ("group_size", C.c_int32), ("fp_budget_windows", C.c_int32),
+        ("q_budget_windows", C.c_int32), ("max_context", C.c_int32), ("rebalance_interval_hint", C.c_int32),
+        ("softmax_scale", C.c_float), ("device", C.c_int32),
+    ]
+
+
+class qevict_stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "promotions", "quantizations", "reactivations", "deletions", "n_full", "n_quant", "n_aged", "n_open",
+        "n_evicted", "decode_steps")]
+
+
+_lib = None
+
+_SIGNATURES = {
+    "qevict_version": (C.c_char_p, []),
+    "qevict_status_string": (C.c_char_p, [C.c_int]),
+    "qevict_last_error": (C.c_char_p, [C.c_void_p]),
+    "qevict_launch_count": (C.c_uint64, [C.c_void_p]),
+    "qevict_budget_from_bytes": (C.c_int, [C.POINTER(qevict_config), C.c_uint64, C.c_double, C.POINTER(C.c_int32),
+                                           C.POINTER(C.c_int32), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]),
+    "qevict_workspace_bytes": (C.c_int, [C.POINTER(qevict_config), C.POINTER(C.c_uint64)]),
+    "qevict_create": (C.c_int, [C.POINTER(qevict_config), C.c_void_p, C.c_uint64, C.POINTER(C.c_void_p)]),
+    "qevict_destroy": (C.c_int, [C.c_void_p]),
+    "qevict_set_splits": (C.c_int, [C.c_void_p, C.c_int32]),
+    "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_rebalance": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
+    "qevict_get_stats": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(qevict_stats)]),
+    "qevict_export_tables": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 7),
+    "qevict_export_last_mass": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "qevict_export_fp_page": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_export_q_page": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 5),
+}
+
+
+def lib():
+    """The loaded shared library.  Raises if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libqevict.so is missing: run `python -m paper_2608_05326_b200.build` "
+                               "(or __graft_entry__.build()) first; there is no fallback path")
+        handle = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def _check(status, handle=None):
+    if status != QEVICT_OK:
+        msg = lib().qevict_last_error(handle).decode() if handle else lib().qevict_status_string(status).decode()
+        raise QEvictError(status, msg or lib().qevict_status_string(status).decode())
+
+
+def make_config(batch, n_layers, n_q_heads, n_kv_heads, head_dim, dtype, window, quant_bits, group_size,
+                fp_budget_windows, q_budget_windows, max_context, rebalance_interval_hint=0, softmax_scale=0.0,
+                device=0):
+    dt = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, torch.float16: DTYPE_FP16, torch.bfloat16: DTYPE_BF16}[dtype]
+    return qevict_config(C.sizeof(qevict_config), batch, n_layers, n_q_heads, n_kv_heads, head_dim, dt, window,
+                         quant_bits, group_size, fp_budget_windows, q_budget_windows, max_context,
+                         rebalance_interval_hint, softmax_scale, device)
+
+
+# --- plain function wrappers, same names as the C entry points -----------------------------------------
+def qevict_version():
+    return lib().qevict_version().decode()
+
+
+def qevict_budget_from_bytes(cfg, hist_bytes, q_frac):
+    kf, kq, mf, mq = C.c_int32(), C.c_int32(), C.c_uint64(), C.c_uint64()
+    _check(lib().qevict_budget_from_bytes(C.byref(cfg), int(hist_bytes), float(q_frac), C.byref(kf), C.byref(kq),
+                                          C.byref(mf), C.byref(mq)))
+    return kf.value, kq.value, mf.value, mq.value
+
+
+def qevict_workspace_bytes(cfg):
+    n = C.c_uint64()
+    _check(lib().qevict_workspace_bytes(C.byref(cfg), C.byref(n)))
+    return n.value
+
+
+def qevict_create(cfg, device_mem_ptr, n_bytes):
+    h = C.c_void_p()
+    _check(lib().qevict_create(C.byref(cfg), device_mem_ptr, n_bytes, C.byref(h)))
+    return h
+
+
+def qevict_destroy(h):
+    _check(lib().qevict_destroy(h))
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def qevict_prefill_assign(h, layer, k, v, ctx_tokens, window_scores, stream=None):
+    _check(lib().qevict_prefill_assign(h, layer, _ptr(k), _ptr(v), ctx_tokens, _ptr(window_scores), _stream(stream)), h)
+
+
+def qevict_decode_attn(h, layer, q, k_new, v_new, out, stream=None):
+    _check(lib().qevict_decode_attn(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
+
+
+def qevict_decode_attn_host(h, layer, q, k_new, v_new, out, stream=None):
+    """q, k_new, v_new, out: HOST tensors (pinned or pageable)."""
+    _check(lib().qevict_decode_attn_host(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
+
+
+def qevict_rebalance(h, layer, stream=None):
+    _check(lib().qevict_rebalance(h, layer, _stream(stream)), h)
+
+
+def qevict_set_splits(h, splits):
+    _check(lib().qevict_set_splits(h, splits), h)
+
+
+def qevict_get_stats(h, layer=-1):
+    st = qevict_stats()
+    _check(lib().qevict_get_stats(h, layer, C.byref(st)), h)
+    return {n: getattr(st, n) for n, _ in qevict_stats._fields_}
+
+
+def qevict_launch_count(h):
+    return lib().qevict_launch_count(h)
+
+
+class QEvictCache:
+    """A cache handle together with the torch-allocated device workspace it lives in."""
+
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.device = torch.device("cuda", cfg.device)
+        self.torch_dtype = torch.float16 if cfg.dtype == DTYPE_FP16 else torch.bfloat16
+        self.n_bytes = qevict_workspace_bytes(cfg)
+        self.workspace = torch.empty(self.n_bytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.handle = qevict_create(cfg, C.c_void_p(base), self.n_bytes)
+        self.max_windows = cfg.max_context // cfg.window
+
+    def close(self):
+        if self.handle is not None:
+            torch.cuda.synchronize(self.device)
+            qevict_destroy(self.handle)
+            self.handle = None
+            self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the hot path -----------------------------------------------------------------------------
+    def prefill_assign(self, layer, k, v, window_scores, stream=None):
+        assert k.is_cuda and k.is_contiguous() and v.is_contiguous() and k.dtype == self.torch_dtype
+        assert window_scores.dtype == torch.float32 and window_scores.is_contiguous()
+        qevict_prefill_assign(self.handle, layer, k, v, k.shape[-2], window_scores, stream)
+
+    def decode_attn(self, layer, q, k_new=None, v_new=None, out=None, stream=None):
+        assert q.is_cuda and q.is_contiguous() and q.dtype == self.torch_dtype
+        if out is None:
+            out = torch.empty_like(q)
+        qevict_decode_attn(self.handle, layer, q, k_new, v_new, out, stream)
+        return out
+
+    def decode_attn_host(self, layer, q, k_new, v_new, out, stream=None):
+        qevict_decode_attn_host(self.handle, layer, q, k_new, v_new, out, stream)
+        return out
+
+    def rebalance(self, layer, stream=None):
+        qevict_rebalance(self.handle, layer, stream)
+
+    def set_splits(self, splits):
+        qevict_set_splits(self.handle, splits)
+
+    def stats(self, layer=-1):
+        return qevict_get_stats(self.handle, layer)
+
+    def launch_count(self):
+        return qevict_launch_count(self.handle)
+
+    # -- exports (parity checks, snapshots) -------------------------------------------------------
+    def export_tables(self, layer, seq):
+        n = self.max_windows
+        dev = self.device
+        out = {
+            "n_windows": torch.zeros(1, dtype=torch.int32, device=dev),
+            "tier": torch.zeros(n, dtype=torch.uint8, device=dev),
+            "ledger": torch.zeros(n, dtype=torch.uint8, device=dev),
+            "fp_page": torch.zeros(n, dtype=torch.int32, device=dev),
+            "q_page": torch.zeros(n, dtype=torch.int32, device=dev),
+            "importance": torch.zeros(n, dtype=torch.float32, device=dev),
+        }
+        _check(lib().qevict_export_tables(self.handle, layer, seq, _ptr(out["n_windows"]), _ptr(out["tier"]),
+                                          _ptr(out["ledger"]), _ptr(out["fp_page"]), _ptr(out["q_page"]),
+                                          _ptr(out["importance"]), _stream(None)), self.handle)
+        return {k: v.cpu() for k, v in out.items()}
+
+    def export_last_mass(self, layer, seq):
+        m = torch.zeros(self.max_windows, dtype=torch.float32, device=self.device)
+        _check(lib().qevict_export_last_mass(self.handle, layer, seq, _ptr(m), _stream(None)), self.handle)
+        return m.cpu()
+
+    def export_fp_page(self, layer, seq, page):
+        c = self.cfg
+        k = torch.empty((c.n_kv_heads, c.window, c.head_dim), dtype=self.torch_dtype, device=self.device)
+        v = torch.empty_like(k)
+        _check(lib().qevict_export_fp_page(self.handle, layer, seq, page, _ptr(k), _ptr(v), _stream(None)), self.handle)
+        return k.cpu(), v.cpu()
+
+    def export_q_page(self, layer, seq, page):
+        c = self.cfg
+        g = c.group_size
+        kc = torch.empty((c.n_kv_heads, c.window, c.head_dim), dtype=torch.uint8, device=self.device)
+        vc = torch.empty_like(kc)
+        kp = torch.empty((c.n_kv_heads, c.window // g, c.head_dim, 2), dtype=self.torch_dtype, device=self.device)
+        vp = torch.empty((c.n_kv_heads, c.window, c.head_dim // g, 2), dtype=self.torch_dtype, device=self.device)
+        _check(lib().qevict_export_q_page(self.handle, layer, seq, page, _ptr(kc), _ptr(kp), _ptr(vc), _ptr(vp),
+                                          _stream(None)), self.handle)
+        return kc.cpu(), kp.cpu(), vc.cpu(), vp.cpu()

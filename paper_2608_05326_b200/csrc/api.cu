@@ -1,0 +1,534 @@
+// Host side of the C ABI: validation, workspace carving, call-order bookkeeping, kernel launches.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <string>
+#include <vector>
+
+#include "decode_attn.cuh"
+#include "kernels.cuh"
+
+using namespace qevict;
+
+namespace {
+
+struct LayerMirror {  // what the host must know without reading device memory (same for every sequence)
+  bool prefilled = false;
+  bool has_open = false;
+  int open_fill = 0;
+  int n_windows = 0;
+  int aged = 0;  // filled windows waiting for a routing event
+};
+
+constexpr int SM_COUNT_FALLBACK = 148;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int next_pow2(int x) {
+  int p = 2;
+  while (p < x) p <<= 1;
+  return p;
+}
+
+}  // namespace
+
+struct qevict_ctx {
+  qevict_config cfg;
+  Geometry geo;
+  State st;
+  std::vector<LayerMirror> layers;
+  std::string last_error;
+  uint64_t launches = 0;
+  uint64_t decode_steps = 0;
+  decode_launch_fn decode_fn = nullptr;
+  int forced_splits = 0;
+  int sm_count = SM_COUNT_FALLBACK;
+  char* stage_q = nullptr;    // device staging for the host-buffer entry point
+  char* stage_k = nullptr;
+  char* stage_v = nullptr;
+  char* stage_out = nullptr;
+};
+
+namespace {
+
+qevict_status fail(qevict_handle h, qevict_status s, const std::string& msg) {
+  if (h) h->last_error = msg;
+  return s;
+}
+
+const char* validate(const qevict_config* c) {
+  if (!c) return "config is NULL";
+  if (c->struct_size != sizeof(qevict_config)) return "struct_size does not match this library's qevict_config";
+  if (c->batch < 1 || c->n_layers < 1) return "batch and n_layers must be >= 1";
+  if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c->n_q_heads > 128) return "n_q_heads > 128";
+  if (c->dtype != QEVICT_DTYPE_FP16 && c->dtype != QEVICT_DTYPE_BF16) return "dtype must be fp16 or bf16";
+  if (c->fp_budget_windows < 0 || c->q_budget_windows < 0 || c->fp_budget_windows + c->q_budget_windows < 1)
+    return "tier budgets must be >= 0 and not both zero";
+  if (c->window < 1 || c->max_context < c->window || c->max_context % c->window) return "max_context must be a positive multiple of window";
+  if (c->group_size < 1 || c->window % c->group_size || c->head_dim % c->group_size) return "group_size must divide window and head_dim";
+  if (c->rebalance_interval_hint < 0) return "rebalance_interval_hint < 0";
+  if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return "softmax_scale must be finite and >= 0";
+  return nullptr;
+}
+
+const char* unsupported(const qevict_config* c) {
+  if (c->n_q_heads / c->n_kv_heads > 8) return "more than 8 query heads per KV head";
+  if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
+  if (c->window != 32 && c->window != 64) return "window must be 32 or 64";
+  if (c->quant_bits != 2 && c->quant_bits != 4) return "quant_bits must be 2 or 4";
+  if (c->group_size != 32 && c->group_size != 64) return "group_size must be 32 or 64";
+  if (c->max_context / c->window > 8192) return "more than 8192 windows per sequence";
+  return nullptr;
+}
+
+void make_geometry(const qevict_config& c, Geometry& g) {
+  memset(&g, 0, sizeof(g));
+  g.batch = c.batch; g.n_layers = c.n_layers; g.n_units = c.batch * c.n_layers;
+  g.Hq = c.n_q_heads; g.Hkv = c.n_kv_heads; g.G = g.Hq / g.Hkv; g.D = c.head_dim; g.dtype = c.dtype;
+  g.W = c.window; g.bits = c.quant_bits; g.group = c.group_size; g.Kf = c.fp_budget_windows; g.Kq = c.q_budget_windows;
+  g.NW = c.max_context / c.window;
+  const int r = c.rebalance_interval_hint > 0 ? c.rebalance_interval_hint : c.window;
+  g.aged_cap = (r + g.W - 1) / g.W + 1;
+  g.PF = g.Kf + g.aged_cap + 1;
+  g.PQ = g.Kq + g.Kf;
+  g.EMAX = g.Kf + g.Kq + g.aged_cap + 1;
+  g.tiles = g.W / 32;
+  g.fp_tile_bytes = 32u * g.D * 2u;
+  g.fp_head_bytes = g.tiles * 2u * g.fp_tile_bytes;
+  g.fp_page_bytes = g.Hkv * g.fp_head_bytes;
+  g.q_kc_bytes = 32u * g.D * g.bits / 8u;
+  g.q_vc_bytes = g.q_kc_bytes;
+  g.q_vp_bytes = 32u * (g.D / g.group) * 4u;
+  g.q_tile_stride = g.q_kc_bytes + g.q_vc_bytes + g.q_vp_bytes;
+  g.q_kp_bytes = g.D * 4u;
+  g.q_kp_off = g.tiles * g.q_tile_stride;
+  g.q_head_bytes = g.q_kp_off + (g.W / g.group) * g.q_kp_bytes;
+  g.q_page_bytes = g.Hkv * g.q_head_bytes;
+  const double scale = c.softmax_scale > 0.f ? (double)c.softmax_scale : 1.0 / sqrt((double)c.head_dim);
+  g.scale_log2 = (float)(scale * 1.4426950408889634074);
+}
+
+// Lays the cache out inside one buffer; with base == nullptr only the size is computed.
+size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char* p = base ? base + off : nullptr;
+    off = align_up(off + bytes, 256);
+    return p;
+  };
+  const size_t U = g.n_units;
+  State s;
+  s.fp_pool = take(U * g.PF * (size_t)g.fp_page_bytes);
+  s.q_pool = take(U * g.PQ * (size_t)g.q_page_bytes);
+  s.tier = (uint8_t*)take(U * g.NW);
+  s.ledger = (uint8_t*)take(U * g.NW);
+  s.fp_page = (int32_t*)take(U * g.NW * 4);
+  s.q_page = (int32_t*)take(U * g.NW * 4);
+  s.importance = (float*)take(U * g.NW * 4);
+  s.fp_owner = (int32_t*)take(U * g.PF * 4);
+  s.q_owner = (int32_t*)take(U * g.PQ * 4);
+  s.n_windows = (int32_t*)take(U * 4);
+  s.open_window = (int32_t*)take(U * 4);
+  s.open_fill = (int32_t*)take(U * 4);
+  s.n_live = (int32_t*)take(U * 4);
+  s.entries = (uint2*)take(U * g.EMAX * 8);
+  s.quant_list = (int4*)take(U * (size_t)(g.PF + g.Kq) * 16);
+  s.promote_list = (int4*)take(U * (size_t)(g.Kf > 0 ? g.Kf : 1) * 16);
+  s.copy_list = (int4*)take(U * (size_t)(g.Kf > 0 ? g.Kf : 1) * 16);
+  s.n_quant = (int32_t*)take(U * 4);
+  s.n_promote = (int32_t*)take(U * 4);
+  s.n_copy = (int32_t*)take(U * 4);
+  s.counters = (unsigned long long*)take(U * 4 * 8);
+  s.o_part = (float*)take(U * g.Hq * (size_t)MAX_SPLITS * g.D * 4);
+  s.ml = (float*)take(U * g.Hq * (size_t)MAX_SPLITS * 2 * 4);
+  s.wrec = (float2*)take(U * g.Hq * (size_t)g.EMAX * 8);
+  s.mass_e = (float*)take(U * (size_t)g.EMAX * 4);
+  s.status = (int32_t*)take(256);
+  char* sq = take(U * g.Hq * (size_t)g.D * 2);
+  char* sk = take(U * g.Hkv * (size_t)g.D * 2);
+  char* sv = take(U * g.Hkv * (size_t)g.D * 2);
+  char* so = take(U * g.Hq * (size_t)g.D * 2);
+  if (st) *st = s;
+  if (ctx) { ctx->stage_q = sq; ctx->stage_k = sk; ctx->stage_v = sv; ctx->stage_out = so; }
+  return off;
+}
+
+bool layer_range(qevict_handle h, int layer, int* l0, int* l1) {
+  if (layer == -1) { *l0 = 0; *l1 = h->geo.n_layers; return true; }
+  if (layer < 0 || layer >= h->geo.n_layers) return false;
+  *l0 = layer; *l1 = layer + 1;
+  return true;
+}
+
+KernelArgs make_args(qevict_handle h, int l0, int l1) {
+  KernelArgs a;
+  a.geo = h->geo;
+  a.st = h->st;
+  a.unit0 = l0 * h->geo.batch;
+  a.n_units = (l1 - l0) * h->geo.batch;
+  return a;
+}
+
+// Splits per (unit, KV head): enough CTAs to fill the GPU in whole waves while every warp still walks
+// several windows.
+int choose_splits(const qevict_ctx* h, int n_units) {
+  if (h->forced_splits > 0) return h->forced_splits < MAX_SPLITS ? h->forced_splits : MAX_SPLITS;
+  const Geometry& g = h->geo;
+  const int entries = g.Kf + g.Kq + 1;
+  const long pairs = (long)n_units * g.Hkv;
+  const long slots = (long)h->sm_count * 3;  // resident CTAs
+  int best = 1;
+  double best_cost = 1e30;
+  const int smax = entries / DECODE_WARPS < 1 ? 1 : (entries / DECODE_WARPS > MAX_SPLITS ? MAX_SPLITS : entries / DECODE_WARPS);
+  for (int s = 1; s <= smax; ++s) {
+    const long ctas = pairs * s;
+    const long waves = (ctas + slots - 1) / slots;
+    const double per_warp = ceil((double)entries / (s * DECODE_WARPS)) * g.tiles;
+    const double cost = (double)waves * (per_warp + 2.0);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+#define QE_CUDA(h, expr)                                                                  \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess) return fail(h, QEVICT_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+
+qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                          cudaStream_t stream) {
+  int l0, l1;
+  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  if (!q || !out) return fail(h, QEVICT_ERR_INVALID_ARG, "q and out must not be NULL");
+  if ((k_new == nullptr) != (v_new == nullptr)) return fail(h, QEVICT_ERR_INVALID_ARG, "k_new and v_new must both be given or both be NULL");
+  const Geometry& g = h->geo;
+  for (int l = l0; l < l1; ++l) {
+    const LayerMirror& m = h->layers[l];
+    if (!m.prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "decode before prefill_assign");
+    if (k_new && !m.has_open) {
+      if (m.aged > g.aged_cap) return fail(h, QEVICT_ERR_BAD_STATE, "too many filled windows are waiting: call qevict_rebalance");
+      if (m.n_windows + 1 > g.NW) return fail(h, QEVICT_ERR_BAD_STATE, "context would exceed max_context");
+    }
+  }
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  const KernelArgs a = make_args(h, l0, l1);
+  if (k_new) {
+    QE_CUDA(h, launch_append(a, k_new, v_new, stream));
+    h->launches++;
+    for (int l = l0; l < l1; ++l) {
+      LayerMirror& m = h->layers[l];
+      if (!m.has_open) { m.has_open = true; m.open_fill = 0; m.n_windows++; }
+      if (++m.open_fill == g.W) { m.has_open = false; m.open_fill = 0; m.aged++; }
+    }
+  }
+  DecodeParams p;
+  p.q = q; p.entries = h->st.entries; p.n_live = h->st.n_live; p.open_fill = h->st.open_fill;
+  p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
+  p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
+  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
+  QE_CUDA(h, h->decode_fn(p, a.n_units, stream));
+  h->launches++;
+  QE_CUDA(h, launch_combine(a, p.S, out, stream));
+  h->launches++;
+  h->decode_steps++;
+  return QEVICT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+QEVICT_API const char* qevict_version(void) { return "0.1"; }
+
+QEVICT_API const char* qevict_status_string(qevict_status s) {
+  switch (s) {
+    case QEVICT_OK: return "ok";
+    case QEVICT_ERR_INVALID_ARG: return "invalid argument";
+    case QEVICT_ERR_BAD_STATE: return "bad state";
+    case QEVICT_ERR_NO_MEMORY: return "not enough memory";
+    case QEVICT_ERR_UNSUPPORTED: return "unsupported configuration";
+    case QEVICT_ERR_CUDA: return "CUDA error";
+    case QEVICT_ERR_DEVICE_CHECK: return "device-side check failed";
+  }
+  return "unknown status";
+}
+
+QEVICT_API const char* qevict_last_error(qevict_handle h) { return h ? h->last_error.c_str() : "handle is NULL"; }
+
+QEVICT_API uint64_t qevict_launch_count(qevict_handle h) { return h ? h->launches : 0; }
+
+QEVICT_API qevict_status qevict_budget_from_bytes(const qevict_config* cfg, uint64_t hist_bytes, double q_frac, int32_t* k_f,
+                                       int32_t* k_q, uint64_t* m_f, uint64_t* m_q) {
+  if (!cfg || !(q_frac >= 0.0 && q_frac <= 1.0)) return QEVICT_ERR_INVALID_ARG;
+  if (cfg->n_kv_heads < 1 || cfg->head_dim < 1 || cfg->window < 1 || cfg->group_size < 1 || cfg->quant_bits < 1 ||
+      cfg->window % cfg->group_size || cfg->head_dim % cfg->group_size)
+    return QEVICT_ERR_INVALID_ARG;
+  const uint64_t h = cfg->n_kv_heads, w = cfg->window, d = cfg->head_dim, g = cfg->group_size, b = cfg->quant_bits;
+  const uint64_t mf = 2 * h * w * d * 2;
+  const uint64_t mq = h * (2 * w * d * b / 8 + (w / g) * d * 4 + w * (d / g) * 4);
+  if (m_f) *m_f = mf;
+  if (m_q) *m_q = mq;
+  if (k_f) *k_f = (int32_t)floor((1.0 - q_frac) * (double)hist_bytes / (double)mf);
+  if (k_q) *k_q = (int32_t)floor(q_frac * (double)hist_bytes / (double)mq);
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_workspace_bytes(const qevict_config* cfg, uint64_t* bytes) {
+  if (!bytes) return QEVICT_ERR_INVALID_ARG;
+  if (validate(cfg)) return QEVICT_ERR_INVALID_ARG;
+  if (unsupported(cfg)) return QEVICT_ERR_UNSUPPORTED;
+  Geometry g;
+  make_geometry(*cfg, g);
+  *bytes = carve(g, nullptr, nullptr, nullptr);
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_mem, uint64_t bytes, qevict_handle* out) {
+  if (!out) return QEVICT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (validate(cfg)) return QEVICT_ERR_INVALID_ARG;
+  if (unsupported(cfg)) return QEVICT_ERR_UNSUPPORTED;
+  if (!device_mem || ((uintptr_t)device_mem & 255)) return QEVICT_ERR_INVALID_ARG;
+  qevict_ctx* h = new (std::nothrow) qevict_ctx();
+  if (!h) return QEVICT_ERR_NO_MEMORY;
+  h->cfg = *cfg;
+  make_geometry(*cfg, h->geo);
+  const Geometry& g = h->geo;
+  const size_t need = carve(g, (char*)device_mem, &h->st, h);
+  if (need > bytes) { delete h; return QEVICT_ERR_NO_MEMORY; }
+  switch ((g.dtype == QEVICT_DTYPE_BF16 ? 2 : 0) + (g.D == 128 ? 1 : 0)) {
+    case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles); break;
+    case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles); break;
+    case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles); break;
+    default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles); break;
+  }
+  if (!h->decode_fn) { delete h; return QEVICT_ERR_UNSUPPORTED; }
+  h->layers.resize(g.n_layers);
+  cudaError_t e = cudaSetDevice(cfg->device);
+  if (e == cudaSuccess) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) h->sm_count = sms;
+    const size_t U = g.n_units;
+    // tables: everything between the pools and the scratch starts cleared
+    e = cudaMemset(h->st.tier, 0, U * g.NW);
+    if (e == cudaSuccess) e = cudaMemset(h->st.ledger, 0, U * g.NW);
+    if (e == cudaSuccess) e = cudaMemset(h->st.fp_page, 0xFF, U * g.NW * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.q_page, 0xFF, U * g.NW * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.importance, 0, U * g.NW * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.fp_owner, 0xFF, U * g.PF * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.q_owner, 0xFF, U * g.PQ * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.n_windows, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.open_window, 0xFF, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.open_fill, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.n_live, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.n_quant, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.n_promote, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.n_copy, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.counters, 0, U * 32);
+    if (e == cudaSuccess) e = cudaMemset(h->st.mass_e, 0, U * (size_t)g.EMAX * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.status, 0, 256);
+    if (e == cudaSuccess) e = route_prepare(route_smem_bytes(g, next_pow2(g.NW)));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  }
+  if (e != cudaSuccess) {
+    delete h;
+    return QEVICT_ERR_CUDA;
+  }
+  *out = h;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_destroy(qevict_handle h) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  delete h;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_set_splits(qevict_handle h, int32_t splits) {
+  if (!h || splits < 0 || splits > MAX_SPLITS) return QEVICT_ERR_INVALID_ARG;
+  h->forced_splits = splits;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, const void* k, const void* v, int32_t ctx_tokens,
+                                    const float* window_scores, void* stream) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  int l0, l1;
+  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  if (!k || !v || !window_scores) return fail(h, QEVICT_ERR_INVALID_ARG, "k, v and window_scores must not be NULL");
+  const Geometry& g = h->geo;
+  if (ctx_tokens < g.W || ctx_tokens % g.W) return fail(h, QEVICT_ERR_UNSUPPORTED, "ctx_tokens must be a positive multiple of window");
+  if (ctx_tokens > h->cfg.max_context) return fail(h, QEVICT_ERR_INVALID_ARG, "ctx_tokens exceeds max_context");
+  for (int l = l0; l < l1; ++l)
+    if (h->layers[l].prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "prefill_assign called twice for a layer");
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  cudaStream_t s = (cudaStream_t)stream;
+  const KernelArgs a = make_args(h, l0, l1);
+  const int n_prompt = ctx_tokens / g.W;
+  QE_CUDA(h, launch_prefill_init(a, n_prompt, window_scores, s));
+  QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
+  QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kf, s));
+  QE_CUDA(h, launch_quantize(a, k, v, ctx_tokens, g.Kq, s));
+  h->launches += 2 + (g.Kf > 0) + (g.Kq > 0);
+  for (int l = l0; l < l1; ++l) {
+    h->layers[l].prefilled = true;
+    h->layers[l].n_windows = n_prompt;
+  }
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_decode_attn(qevict_handle h, int32_t layer, const void* q, const void* k_new, const void* v_new,
+                                 void* out, void* stream) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  return decode_impl(h, layer, q, k_new, v_new, out, (cudaStream_t)stream);
+}
+
+QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer, const void* q_host, const void* k_new_host,
+                                      const void* v_new_host, void* out_host, void* stream) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  int l0, l1;
+  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  if (!q_host || !out_host) return fail(h, QEVICT_ERR_INVALID_ARG, "q_host and out_host must not be NULL");
+  if ((k_new_host == nullptr) != (v_new_host == nullptr)) return fail(h, QEVICT_ERR_INVALID_ARG, "k_new and v_new must both be given or both be NULL");
+  const Geometry& g = h->geo;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t nu = (size_t)(l1 - l0) * g.batch;
+  const size_t qb = nu * g.Hq * g.D * 2, kb = nu * g.Hkv * g.D * 2;
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_CUDA(h, cudaMemcpyAsync(h->stage_q, q_host, qb, cudaMemcpyHostToDevice, s));
+  if (k_new_host) {
+    QE_CUDA(h, cudaMemcpyAsync(h->stage_k, k_new_host, kb, cudaMemcpyHostToDevice, s));
+    QE_CUDA(h, cudaMemcpyAsync(h->stage_v, v_new_host, kb, cudaMemcpyHostToDevice, s));
+  }
+  const qevict_status st = decode_impl(h, layer, h->stage_q, k_new_host ? h->stage_k : nullptr,
+                                       k_new_host ? h->stage_v : nullptr, h->stage_out, s);
+  if (st != QEVICT_OK) return st;
+  QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
+  QE_CUDA(h, cudaStreamSynchronize(s));
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* stream) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  int l0, l1;
+  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  for (int l = l0; l < l1; ++l)
+    if (!h->layers[l].prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "rebalance before prefill_assign");
+  const Geometry& g = h->geo;
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  cudaStream_t s = (cudaStream_t)stream;
+  const KernelArgs a = make_args(h, l0, l1);
+  QE_CUDA(h, launch_route(a, 0, next_pow2(g.Kf + g.Kq + g.aged_cap + 1), s));
+  // quantizations read full-precision pages that promotions may overwrite: quantize first
+  QE_CUDA(h, launch_quantize(a, nullptr, nullptr, 0, g.Kq > 0 ? g.PF : 0, s));
+  const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
+  QE_CUDA(h, launch_promote(a, max_promote, s));
+  h->launches += 1 + (g.Kq > 0) + (max_promote > 0);
+  for (int l = l0; l < l1; ++l) h->layers[l].aged = 0;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict_stats* out) {
+  if (!h || !out) return QEVICT_ERR_INVALID_ARG;
+  int l0, l1;
+  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  const Geometry& g = h->geo;
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_CUDA(h, cudaDeviceSynchronize());
+  memset(out, 0, sizeof(*out));
+  const size_t u0 = (size_t)l0 * g.batch, nu = (size_t)(l1 - l0) * g.batch;
+  std::vector<unsigned long long> c(nu * 4);
+  std::vector<uint8_t> tiers(nu * g.NW);
+  int32_t status = 0;
+  QE_CUDA(h, cudaMemcpy(c.data(), h->st.counters + u0 * 4, nu * 32, cudaMemcpyDeviceToHost));
+  QE_CUDA(h, cudaMemcpy(tiers.data(), h->st.tier + u0 * g.NW, nu * g.NW, cudaMemcpyDeviceToHost));
+  QE_CUDA(h, cudaMemcpy(&status, h->st.status, 4, cudaMemcpyDeviceToHost));
+  for (size_t u = 0; u < nu; ++u) {
+    out->promotions += c[u * 4]; out->quantizations += c[u * 4 + 1];
+    out->reactivations += c[u * 4 + 2]; out->deletions += c[u * 4 + 3];
+  }
+  for (uint8_t t : tiers) {
+    switch (t) {
+      case QEVICT_TIER_FULL: out->n_full++; break;
+      case QEVICT_TIER_QUANT: out->n_quant++; break;
+      case QEVICT_TIER_AGED: out->n_aged++; break;
+      case QEVICT_TIER_OPEN: out->n_open++; break;
+      case QEVICT_TIER_EVICTED: out->n_evicted++; break;
+      default: break;
+    }
+  }
+  out->decode_steps = h->decode_steps;
+  if (status != 0) {
+    char buf[96];
+    snprintf(buf, sizeof(buf), "device check %d failed", status);
+    return fail(h, QEVICT_ERR_DEVICE_CHECK, buf);
+  }
+  return QEVICT_OK;
+}
+
+static bool unit_of(qevict_handle h, int layer, int seq, int* u) {
+  if (layer < 0 || layer >= h->geo.n_layers || seq < 0 || seq >= h->geo.batch) return false;
+  *u = layer * h->geo.batch + seq;
+  return true;
+}
+
+QEVICT_API qevict_status qevict_export_tables(qevict_handle h, int32_t layer, int32_t seq, int32_t* n_windows, uint8_t* tier,
+                                   uint8_t* ledger, int32_t* fp_page, int32_t* q_page, float* importance, void* stream) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  int u;
+  if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
+  const Geometry& g = h->geo;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t o = (size_t)u * g.NW;
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  if (n_windows) QE_CUDA(h, cudaMemcpyAsync(n_windows, h->st.n_windows + u, 4, cudaMemcpyDeviceToDevice, s));
+  if (tier) QE_CUDA(h, cudaMemcpyAsync(tier, h->st.tier + o, g.NW, cudaMemcpyDeviceToDevice, s));
+  if (ledger) QE_CUDA(h, cudaMemcpyAsync(ledger, h->st.ledger + o, g.NW, cudaMemcpyDeviceToDevice, s));
+  if (fp_page) QE_CUDA(h, cudaMemcpyAsync(fp_page, h->st.fp_page + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
+  if (q_page) QE_CUDA(h, cudaMemcpyAsync(q_page, h->st.q_page + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
+  if (importance) QE_CUDA(h, cudaMemcpyAsync(importance, h->st.importance + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_export_last_mass(qevict_handle h, int32_t layer, int32_t seq, float* mass, void* stream) {
+  if (!h || !mass) return QEVICT_ERR_INVALID_ARG;
+  int u;
+  if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  const KernelArgs a = make_args(h, 0, h->geo.n_layers);
+  QE_CUDA(h, launch_export_mass(a, u, mass, (cudaStream_t)stream));
+  h->launches++;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_export_fp_page(qevict_handle h, int32_t layer, int32_t seq, int32_t fp_page, void* k_out,
+                                    void* v_out, void* stream) {
+  if (!h || !k_out || !v_out) return QEVICT_ERR_INVALID_ARG;
+  int u;
+  if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
+  if (fp_page < 0 || fp_page >= h->geo.PF) return fail(h, QEVICT_ERR_INVALID_ARG, "fp_page out of range");
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  const KernelArgs a = make_args(h, 0, h->geo.n_layers);
+  QE_CUDA(h, launch_export_fp_page(a, u, fp_page, k_out, v_out, (cudaStream_t)stream));
+  h->launches++;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, int32_t seq, int32_t q_page, uint8_t* k_codes,
+                                   void* k_params, uint8_t* v_codes, void* v_params, void* stream) {
+  if (!h || !k_codes || !k_params || !v_codes || !v_params) return QEVICT_ERR_INVALID_ARG;
+  int u;
+  if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
+  if (q_page < 0 || q_page >= h->geo.PQ) return fail(h, QEVICT_ERR_INVALID_ARG, "q_page out of range");
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  const KernelArgs a = make_args(h, 0, h->geo.n_layers);
+  QE_CUDA(h, launch_export_q_page(a, u, q_page, k_codes, k_params, v_codes, v_params, (cudaStream_t)stream));
+  h->launches++;
+  return QEVICT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,145 @@
+// Shared declarations of the qevict CUDA library: geometry, device state, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/qevict.h"
+
+namespace qevict {
+
+// entry kinds of the decode work list
+enum : uint32_t { KIND_FP = 0u, KIND_Q = 1u, KIND_OPEN = 2u };
+static constexpr int ENTRY_KIND_SHIFT = 28;
+static constexpr uint32_t ENTRY_WINDOW_MASK = (1u << ENTRY_KIND_SHIFT) - 1u;
+
+// device status word values (first failure wins)
+enum : int {
+  CHECK_OK = 0,
+  CHECK_FP_POOL_EXHAUSTED = 1,
+  CHECK_Q_POOL_EXHAUSTED = 2,
+  CHECK_ENTRY_OVERFLOW = 3,
+  CHECK_WINDOW_OVERFLOW = 4,
+  CHECK_COPY_TIMEOUT = 5,
+};
+
+static constexpr int TILE_TOKENS = 32;    // tokens per attention tile
+static constexpr int DECODE_WARPS = 4;    // warps per decode CTA
+static constexpr int MAX_SPLITS = 64;
+
+// Geometry derived from the configuration (host and device).
+struct Geometry {
+  int batch, n_layers, n_units;
+  int Hq, Hkv, G, D, dtype, W, bits, group, Kf, Kq;
+  int NW;        // max windows per unit
+  int PF, PQ;    // pages per unit in the full-precision / quantized pool
+  int EMAX;      // max entries of a unit's work list
+  int aged_cap;  // filled windows that may wait for a routing event
+  int tiles;     // W / 32
+  // full-precision page: [H_kv][tile]{K tile, V tile}, each tile 32 x D elements, fragment-major
+  uint32_t fp_tile_bytes, fp_head_bytes, fp_page_bytes;
+  // quantized page: [H_kv]{ [tile]{K codes, V codes, V params}, K params x (W/group) }
+  uint32_t q_kc_bytes, q_vc_bytes, q_vp_bytes, q_tile_stride, q_kp_bytes, q_kp_off, q_head_bytes, q_page_bytes;
+  float scale_log2;  // softmax scale * log2(e)
+};
+
+// Device pointers of one cache (all arrays are [n_units][...]).
+struct State {
+  uint8_t* tier;        // [NW]
+  uint8_t* ledger;      // [NW]
+  int32_t* fp_page;     // [NW]
+  int32_t* q_page;      // [NW]
+  float* importance;    // [NW]
+  int32_t* fp_owner;    // [PF] window holding the page, -1 free
+  int32_t* q_owner;     // [PQ]
+  int32_t* n_windows;   // [1]
+  int32_t* open_window; // [1] -1 if none
+  int32_t* open_fill;   // [1]
+  int32_t* n_live;      // [1] entries in the work list
+  uint2* entries;       // [EMAX] {window | kind << 28, page}
+  int4* quant_list;     // [PF + Kq] {window, src fp page (-1: prompt), dst q page, 0}
+  int4* promote_list;   // [Kf] {window, src q page, dst fp page, 0}
+  int4* copy_list;      // [Kf] {window, dst fp page, 0, 0} (prefill only)
+  int32_t* n_quant;
+  int32_t* n_promote;
+  int32_t* n_copy;
+  unsigned long long* counters;  // [4] promotions, quantizations, reactivations, deletions
+  char* fp_pool;        // [PF] pages
+  char* q_pool;         // [PQ] pages
+  float* o_part;        // [Hq][MAX_SPLITS][D]
+  float* ml;            // [Hq][MAX_SPLITS][2]
+  float2* wrec;         // [Hq][EMAX] {window exp-sum, reference max (log2 domain)}
+  float* mass_e;        // [EMAX] last step's mass per entry
+  int32_t* status;      // [1] (shared by all units)
+};
+
+template <class T> struct Tr;
+template <> struct Tr<__half> {
+  using T2 = __half2;
+  static constexpr uint32_t MAGIC = 0x64006400u;  // 1024.0 in both halves: 1024 + code is exact
+  static __device__ __forceinline__ __half from_float(float x) { return __float2half_rn(x); }
+  static __device__ __forceinline__ float to_float(__half x) { return __half2float(x); }
+};
+template <> struct Tr<__nv_bfloat16> {
+  using T2 = __nv_bfloat162;
+  static constexpr uint32_t MAGIC = 0x43004300u;  // 128.0 in both halves: 128 + code is exact
+  static __device__ __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+  static __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+};
+
+template <class T2> __device__ __forceinline__ T2 as_t2(uint32_t x) {
+  T2 r;
+  *reinterpret_cast<uint32_t*>(&r) = x;
+  return r;
+}
+template <class T2> __device__ __forceinline__ uint32_t as_u32(T2 x) { return *reinterpret_cast<uint32_t*>(&x); }
+
+// Dequantize two codes held in the low bits of each 16-bit half of `x` (already OR-ed with MAGIC):
+// value = RNE_T(code * s + z), one correctly rounded fused multiply-add in the execution datatype.
+template <class T> __device__ __forceinline__ uint32_t dequant2(uint32_t x, uint32_t s2, uint32_t z2) {
+  using T2 = typename Tr<T>::T2;
+  T2 c = __hsub2(as_t2<T2>(x), as_t2<T2>(Tr<T>::MAGIC));  // exact
+  return as_u32(__hfma2(c, as_t2<T2>(s2), as_t2<T2>(z2)));
+}
+
+// D = A(16x16, row) * B(16x8, col) + D, fp32 accumulate.
+template <class T>
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1);
+template <>
+__device__ __forceinline__ void mma16816<__half>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                 uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+template <>
+__device__ __forceinline__ void mma16816<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                        uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ void record_check(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// ---- kernels launched by the host API (defined in the .cu files) -------------------------------
+struct LaunchCtx {
+  Geometry geo;
+  State st;        // pointers of unit 0; per-unit strides are implied by the geometry
+  cudaStream_t stream;
+};
+
+}  // namespace qevict

@@ -1,0 +1,6 @@
+// Instantiations of the tiered flash-decode kernel for one (datatype, head dimension) pair.
+#include "decode_attn.cuh"
+
+namespace qevict {
+QEVICT_DECODE_DISPATCH(decode_dispatch_b128, __nv_bfloat16, 128)
+}  // namespace qevict

@@ -1,0 +1,6 @@
+// Instantiations of the tiered flash-decode kernel for one (datatype, head dimension) pair.
+#include "decode_attn.cuh"
+
+namespace qevict {
+QEVICT_DECODE_DISPATCH(decode_dispatch_h64, __half, 64)
+}  // namespace qevict

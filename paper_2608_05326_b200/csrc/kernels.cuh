@@ -1,0 +1,45 @@
+// Host-callable launchers of the table, page and combine kernels (definitions in the .cu files).
+#pragma once
+
+#include "common.cuh"
+
+namespace qevict {
+
+struct KernelArgs {
+  Geometry geo;
+  State st;
+  int unit0;    // first unit of this call
+  int n_units;  // units of this call
+};
+
+// decode step ---------------------------------------------------------------------------------------
+// A0: append one token per unit to its open window (opens one first if needed, zeroing the page).
+cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s);
+// A2: merge the split partials into `out`, add each window's mass to its score in fixed head order.
+cudaError_t launch_combine(const KernelArgs& a, int n_splits, void* out, cudaStream_t s);
+
+// routing event ---------------------------------------------------------------------------------------
+// P0 (first half): every prompt window becomes an aged candidate with the given score.
+cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt_windows, const float* scores, cudaStream_t s);
+// A3 + A4 + A7: rank, assign tiers, release / allocate pages, build migration lists and the work list.
+cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_capacity, cudaStream_t s);
+// A5: quantize the windows of the quantization list (source: their full-precision page, or the prompt).
+cudaError_t launch_quantize(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx,
+                            int max_items, cudaStream_t s);
+// A6: dequantize the windows of the promotion list into their new full-precision page.
+cudaError_t launch_promote(const KernelArgs& a, int max_items, cudaStream_t s);
+// P0 (second half): copy the prompt windows of the copy list into their full-precision page.
+cudaError_t launch_copy_prompt(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx,
+                               int max_items, cudaStream_t s);
+
+// export ------------------------------------------------------------------------------------------------
+cudaError_t launch_export_fp_page(const KernelArgs& a, int unit, int page, void* k_out, void* v_out, cudaStream_t s);
+cudaError_t launch_export_q_page(const KernelArgs& a, int unit, int page, uint8_t* k_codes, void* k_params,
+                                 uint8_t* v_codes, void* v_params, cudaStream_t s);
+cudaError_t launch_export_mass(const KernelArgs& a, int unit, float* mass, cudaStream_t s);
+
+// dynamic shared memory the route kernel needs for a given sort capacity (power of two)
+size_t route_smem_bytes(const Geometry& g, int sort_capacity);
+cudaError_t route_prepare(size_t max_smem);
+
+}  // namespace qevict

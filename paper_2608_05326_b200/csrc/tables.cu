@@ -1,0 +1,363 @@
+// Window tables: append to the recent region, prefill initialisation, and the routing event
+// (rank -> tiers -> page release / allocation -> migration lists -> decode work list).
+#include "kernels.cuh"
+#include "layout.cuh"
+
+namespace qevict {
+
+namespace {
+
+constexpr int ROUTE_THREADS = 256;
+constexpr unsigned long long KEY_SENTINEL = ~0ull;
+
+// order-preserving map float -> uint32 (ascending); -0 and +0 collapse
+__device__ __forceinline__ uint32_t mono_bits(float f) {
+  if (f == 0.f) f = 0.f;
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Stable, deterministic block-wide stream compaction: calls emit(i, rank) for every i in [0, n)
+// with pred(i), rank = number of smaller i with pred.  Returns the total.  pred must be pure until
+// emit(i) has run.  scratch: 33 ints of shared memory.
+template <class Pred, class Emit>
+__device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int chunk = (n + nt - 1) / nt;
+  const int b = min(n, tid * chunk), e = min(n, b + chunk);
+  int cnt = 0;
+  for (int i = b; i < e; ++i) cnt += pred(i) ? 1 : 0;
+  const int lane = tid & 31, wid = tid >> 5;
+  int inc = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) scratch[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    const int v = (lane < (nt >> 5)) ? scratch[lane] : 0;
+    int iv = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, iv, o);
+      if (lane >= o) iv += x;
+    }
+    scratch[lane] = iv - v;
+    if (lane == 31) scratch[32] = iv;
+  }
+  __syncthreads();
+  int rank = scratch[wid] + inc - cnt;
+  const int total = scratch[32];
+  for (int i = b; i < e; ++i) {
+    if (pred(i)) emit(i, rank++);
+  }
+  __syncthreads();
+  return total;
+}
+
+// ------------------------------------------------------------------------------------------ append
+template <class T>
+__global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T* __restrict__ k_new,
+                                                     const T* __restrict__ v_new) {
+  const Geometry& g = a.geo;
+  const int ul = blockIdx.x, u = a.unit0 + ul, tid = threadIdx.x;
+  __shared__ int s_page, s_slot, s_new, s_window;
+  if (tid == 0) {
+    int ow = a.st.open_window[u];
+    int page = -1, is_new = 0, slot = 0;
+    if (ow < 0) {
+      const int w = a.st.n_windows[u];
+      if (w >= g.NW) {
+        record_check(a.st.status, CHECK_WINDOW_OVERFLOW);
+      } else {
+        int32_t* owner = a.st.fp_owner + (size_t)u * g.PF;
+        for (int pg = 0; pg < g.PF; ++pg) {
+          if (owner[pg] < 0) { page = pg; break; }
+        }
+        const int e = a.st.n_live[u];
+        if (page < 0) {
+          record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED);
+        } else if (e >= g.EMAX) {
+          record_check(a.st.status, CHECK_ENTRY_OVERFLOW);
+          page = -1;
+        } else {
+          owner[page] = w;
+          const size_t wi = (size_t)u * g.NW + w;
+          a.st.fp_page[wi] = page;
+          a.st.q_page[wi] = -1;
+          a.st.tier[wi] = QEVICT_TIER_OPEN;
+          a.st.ledger[wi] = QEVICT_LEDGER_NONE;
+          a.st.importance[wi] = 0.f;
+          a.st.n_windows[u] = w + 1;
+          a.st.open_window[u] = w;
+          a.st.entries[(size_t)u * g.EMAX + e] = make_uint2((uint32_t)w | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)page);
+          a.st.n_live[u] = e + 1;
+          ow = w;
+          is_new = 1;
+        }
+      }
+    } else {
+      page = a.st.fp_page[(size_t)u * g.NW + ow];
+      slot = a.st.open_fill[u];
+    }
+    s_page = page; s_slot = slot; s_new = is_new; s_window = ow;
+  }
+  __syncthreads();
+  const int page = s_page, slot = s_slot;
+  if (page < 0) return;
+  char* pbase = a.st.fp_pool + ((size_t)u * g.PF + page) * g.fp_page_bytes;
+  if (s_new) {
+    // unfilled token slots of the open window must hold finite values (they are multiplied by a zero
+    // probability in the PV product)
+    uint4* z = reinterpret_cast<uint4*>(pbase);
+    for (uint32_t i = tid; i < g.fp_page_bytes / 16; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+  }
+  const int tile = slot >> 5, tk = slot & 31;
+  for (int idx = tid; idx < g.Hkv * g.D; idx += blockDim.x) {
+    const int h = idx / g.D, ch = idx - h * g.D;
+    T* kt = reinterpret_cast<T*>(pbase + (size_t)h * g.fp_head_bytes + (size_t)tile * 2 * g.fp_tile_bytes);
+    T* vt = reinterpret_cast<T*>(reinterpret_cast<char*>(kt) + g.fp_tile_bytes);
+    kt[fpk_off(tk, ch, g.D)] = k_new[((size_t)ul * g.Hkv + h) * g.D + ch];
+    vt[fpv_off(tk, ch)] = v_new[((size_t)ul * g.Hkv + h) * g.D + ch];
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const int fill = slot + 1;
+    if (fill == g.W) {
+      const int w = s_window;
+      a.st.tier[(size_t)u * g.NW + w] = QEVICT_TIER_AGED;
+      const int e = a.st.n_live[u] - 1;  // the open window is always the last entry
+      a.st.entries[(size_t)u * g.EMAX + e] = make_uint2((uint32_t)w | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)page);
+      a.st.open_window[u] = -1;
+      a.st.open_fill[u] = 0;
+    } else {
+      a.st.open_fill[u] = fill;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ prefill init
+__global__ void prefill_init_kernel(const KernelArgs a, int n_prompt, const float* __restrict__ scores) {
+  const Geometry& g = a.geo;
+  const int ul = blockIdx.y, u = a.unit0 + ul;
+  const int w = blockIdx.x * blockDim.x + threadIdx.x;
+  if (w < n_prompt) {
+    const size_t wi = (size_t)u * g.NW + w;
+    a.st.tier[wi] = QEVICT_TIER_AGED;
+    a.st.importance[wi] = scores[(size_t)ul * n_prompt + w];
+  }
+  if (w == 0) a.st.n_windows[u] = n_prompt;
+}
+
+// ------------------------------------------------------------------------------------------- route
+__global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a, int prefill, int sort_cap) {
+  const Geometry& g = a.geo;
+  const int u = a.unit0 + blockIdx.x, tid = threadIdx.x;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
+  int32_t* free_fp = reinterpret_cast<int32_t*>(keys + sort_cap);            // [PF]
+  int32_t* free_q = free_fp + g.PF;                                          // [PQ]
+  int32_t* scratch = free_q + g.PQ;                                          // [40]
+  uint8_t* newt = reinterpret_cast<uint8_t*>(scratch + 40);                  // [NW]
+
+  uint8_t* tier = a.st.tier + (size_t)u * g.NW;
+  uint8_t* ledger = a.st.ledger + (size_t)u * g.NW;
+  int32_t* fp_page = a.st.fp_page + (size_t)u * g.NW;
+  int32_t* q_page = a.st.q_page + (size_t)u * g.NW;
+  const float* imp = a.st.importance + (size_t)u * g.NW;
+  int32_t* fp_owner = a.st.fp_owner + (size_t)u * g.PF;
+  int32_t* q_owner = a.st.q_owner + (size_t)u * g.PQ;
+  const int nw = a.st.n_windows[u];
+
+  int* s_ncand = scratch + 33;
+  int* s_react = scratch + 34;
+  int* s_del = scratch + 35;
+  if (tid == 0) { *s_ncand = 0; *s_react = 0; *s_del = 0; }
+  for (int i = tid; i < sort_cap; i += ROUTE_THREADS) keys[i] = KEY_SENTINEL;
+  __syncthreads();
+
+  // candidates = Full, Quantized and aged windows; key orders by score (higher first), then index
+  for (int w = tid; w < nw; w += ROUTE_THREADS) {
+    const uint8_t t = tier[w];
+    newt[w] = t;
+    if (t == QEVICT_TIER_FULL || t == QEVICT_TIER_QUANT || t == QEVICT_TIER_AGED) {
+      const int pos = atomicAdd(s_ncand, 1);
+      if (pos < sort_cap) keys[pos] = ((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)w;
+    }
+  }
+  __syncthreads();
+  const int n_cand = min(*s_ncand, sort_cap);
+  int n_sort = 2;
+  while (n_sort < n_cand) n_sort <<= 1;
+  for (int k = 2; k <= n_sort; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < n_sort; i += ROUTE_THREADS) {
+        const int ixj = i ^ j;
+        if (ixj > i) {
+          const unsigned long long x = keys[i], y = keys[ixj];
+          const bool asc = (i & k) == 0;
+          if ((x > y) == asc) { keys[i] = y; keys[ixj] = x; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // TopK_{K_f} -> Full, next TopK_{K_q} -> Quantized, remainder -> Evicted
+  for (int pos = tid; pos < n_cand; pos += ROUTE_THREADS) {
+    const uint32_t w = (uint32_t)keys[pos];
+    newt[w] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+  }
+  __syncthreads();
+
+  // releases (page owner tables only; the per-window page ids stay readable until the lists are built)
+  for (int w = tid; w < nw; w += ROUTE_THREADS) {
+    const uint8_t old = tier[w], nt = newt[w];
+    if (old != QEVICT_TIER_FULL && old != QEVICT_TIER_QUANT && old != QEVICT_TIER_AGED) continue;
+    if ((nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT) || nt == QEVICT_TIER_EVICTED) {
+      if (fp_page[w] >= 0) fp_owner[fp_page[w]] = -1;
+    }
+    if (nt == QEVICT_TIER_EVICTED && q_page[w] >= 0) q_owner[q_page[w]] = -1;
+    if (nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT && ledger[w] == QEVICT_LEDGER_DORMANT) {
+      ledger[w] = QEVICT_LEDGER_ACTIVE;  // reactivation: the retained codes are reused, no data moves
+      atomicAdd(s_react, 1);
+    }
+  }
+  __syncthreads();
+
+  // free pages in ascending id
+  const int n_free_fp = block_compact(g.PF, scratch, [&](int pg) { return fp_owner[pg] < 0; },
+                                      [&](int pg, int k) { free_fp[k] = pg; });
+  const int n_free_q = block_compact(g.PQ, scratch, [&](int pg) { return q_owner[pg] < 0; },
+                                     [&](int pg, int k) { free_q[k] = pg; });
+
+  // windows entering the Full tier without a full-precision page (promotions; prompt windows at
+  // prefill), ascending window index
+  int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
+  int4* copy_list = a.st.copy_list + (size_t)u * g.Kf;
+  const int n_fp_need = block_compact(
+      nw, scratch, [&](int w) { return newt[w] == QEVICT_TIER_FULL && tier[w] != QEVICT_TIER_FULL && fp_page[w] < 0; },
+      [&](int w, int k) {
+        if (k >= n_free_fp || k >= g.Kf) { record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED); return; }
+        const int pg = free_fp[k];
+        fp_owner[pg] = w;
+        fp_page[w] = pg;
+        if (prefill) copy_list[k] = make_int4(w, pg, 0, 0);
+        else promote_list[k] = make_int4(w, q_page[w], pg, 0);
+      });
+  // first demotions need a quantized page, ascending window index
+  const int qcap = g.PF + g.Kq;
+  int4* quant_list = a.st.quant_list + (size_t)u * qcap;
+  const int n_q_need = block_compact(
+      nw, scratch,
+      [&](int w) {
+        return newt[w] == QEVICT_TIER_QUANT && tier[w] != QEVICT_TIER_QUANT && tier[w] != QEVICT_TIER_EVICTED &&
+               tier[w] != QEVICT_TIER_OPEN && tier[w] != QEVICT_TIER_NONE && ledger[w] == QEVICT_LEDGER_NONE;
+      },
+      [&](int w, int k) {
+        if (k >= n_free_q || k >= qcap) { record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED); return; }
+        const int pg = free_q[k];
+        q_owner[pg] = w;
+        quant_list[k] = make_int4(w, prefill ? -1 : fp_page[w], pg, 0);
+        q_page[w] = pg;
+        ledger[w] = QEVICT_LEDGER_ACTIVE;
+      });
+
+  // commit the new states
+  for (int w = tid; w < nw; w += ROUTE_THREADS) {
+    const uint8_t old = tier[w], nt = newt[w];
+    if (old != QEVICT_TIER_FULL && old != QEVICT_TIER_QUANT && old != QEVICT_TIER_AGED) continue;
+    if (nt == QEVICT_TIER_FULL) {
+      if (old == QEVICT_TIER_QUANT) ledger[w] = QEVICT_LEDGER_DORMANT;  // codes retained for a later demotion
+    } else if (nt == QEVICT_TIER_QUANT) {
+      if (old != QEVICT_TIER_QUANT) fp_page[w] = -1;
+    } else {  // evicted: everything released, ledger deleted
+      fp_page[w] = -1;
+      q_page[w] = -1;
+      ledger[w] = QEVICT_LEDGER_NONE;
+      atomicAdd(s_del, 1);
+    }
+    tier[w] = nt;
+  }
+  __syncthreads();
+
+  // decode work list: Full.., Quantized.., open window last
+  uint2* entries = a.st.entries + (size_t)u * g.EMAX;
+  const int n_f = block_compact(nw, scratch, [&](int w) { return tier[w] == QEVICT_TIER_FULL; },
+                                [&](int w, int k) {
+                                  if (k < g.EMAX) entries[k] = make_uint2((uint32_t)w | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)fp_page[w]);
+                                });
+  const int n_q = block_compact(nw, scratch, [&](int w) { return tier[w] == QEVICT_TIER_QUANT; },
+                                [&](int w, int k) {
+                                  if (n_f + k < g.EMAX) entries[n_f + k] = make_uint2((uint32_t)w | (KIND_Q << ENTRY_KIND_SHIFT), (uint32_t)q_page[w]);
+                                });
+  if (tid == 0) {
+    int n = n_f + n_q;
+    const int ow = a.st.open_window[u];
+    if (ow >= 0) {
+      if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)fp_page[ow]);
+      n += 1;
+    }
+    if (n > g.EMAX) { record_check(a.st.status, CHECK_ENTRY_OVERFLOW); n = g.EMAX; }
+    a.st.n_live[u] = n;
+    a.st.n_quant[u] = min(n_q_need, min(n_free_q, qcap));
+    a.st.n_promote[u] = prefill ? 0 : min(n_fp_need, min(n_free_fp, g.Kf));
+    a.st.n_copy[u] = prefill ? min(n_fp_need, min(n_free_fp, g.Kf)) : 0;
+    unsigned long long* c = a.st.counters + (size_t)u * 4;
+    c[0] += prefill ? 0 : (unsigned long long)min(n_fp_need, min(n_free_fp, g.Kf));
+    c[1] += (unsigned long long)min(n_q_need, min(n_free_q, qcap));
+    c[2] += (unsigned long long)*s_react;
+    c[3] += (unsigned long long)*s_del;
+  }
+}
+
+__global__ void export_mass_kernel(const KernelArgs a, int u, float* __restrict__ mass) {
+  const Geometry& g = a.geo;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  // caller zeroed `mass`; scatter the per-entry masses of the last step
+  if (i < a.st.n_live[u]) {
+    const uint32_t w = a.st.entries[(size_t)u * g.EMAX + i].x & ENTRY_WINDOW_MASK;
+    mass[w] = a.st.mass_e[(size_t)u * g.EMAX + i];
+  }
+}
+
+}  // namespace
+
+size_t route_smem_bytes(const Geometry& g, int sort_cap) {
+  return (size_t)sort_cap * 8 + (size_t)(g.PF + g.PQ + 40) * 4 + (size_t)((g.NW + 15) / 16) * 16;
+}
+
+cudaError_t route_prepare(size_t max_smem) {
+  if (max_smem <= 48 * 1024) return cudaSuccess;
+  return cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+}
+
+cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s) {
+  if (a.geo.dtype == QEVICT_DTYPE_FP16)
+    append_kernel<__half><<<a.n_units, 128, 0, s>>>(a, (const __half*)k_new, (const __half*)v_new);
+  else
+    append_kernel<__nv_bfloat16><<<a.n_units, 128, 0, s>>>(a, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt, const float* scores, cudaStream_t s) {
+  dim3 grid((n_prompt + 255) / 256, a.n_units);
+  prefill_init_kernel<<<grid, 256, 0, s>>>(a, n_prompt, scores);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_cap, cudaStream_t s) {
+  route_kernel<<<a.n_units, ROUTE_THREADS, route_smem_bytes(a.geo, sort_cap), s>>>(a, prefill, sort_cap);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_export_mass(const KernelArgs& a, int unit, float* mass, cudaStream_t s) {
+  cudaError_t e = cudaMemsetAsync(mass, 0, sizeof(float) * a.geo.NW, s);
+  if (e != cudaSuccess) return e;
+  export_mass_kernel<<<(a.geo.EMAX + 255) / 256, 256, 0, s>>>(a, unit, mass);
+  return cudaGetLastError();
+}
+
+}  // namespace qevict

@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer results (codes, tiers, page tables, ledger flags) and everything derived exactly
+from them (parameters, promoted page contents) are compared bit for bit; attention outputs within
+max-abs 2e-3 + 1e-2 relative; window mass and scores within 1e-4 relative."""
+
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_05326_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _lockstep():
+    import lockstep  # tests/ is on sys.path (conftest)
+    return lockstep
+
+
+def _small(name, **kw):
+    base = dict(name=name, batch=1, n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64, dtype="fp16", context=1024,
+                window=32, quant_bits=4, group_size=32, fp_budget_windows=4, q_budget_windows=8, steps=40,
+                rebalance_interval=1)
+    base.update(kw)
+    return workloads.Workload(**base)
+
+
+def test_config0_append_rebalance_every_step():
+    ls = _lockstep()
+    run = ls.LockstepRun(workloads.config(0))
+    run.check_state("all", "after prefill")
+    st = run.cache.stats()
+    assert (st["n_full"], st["n_quant"], st["n_evicted"]) == (8, 16, 40)
+    for _ in range(run.wl.steps):
+        run.step(append=True)
+    run.check_state("all", "end")
+    st = run.cache.stats()
+    o = run.oracles[0].stats
+    assert st["promotions"] == o["promotions"] > 0
+    assert st["quantizations"] == o["quantizations"] and st["reactivations"] == o["reactivations"]
+    assert st["deletions"] == o["deletions"]
+    run.close()
+
+
+def test_config0_fixed_context_rebalance_every_window():
+    ls = _lockstep()
+    run = ls.LockstepRun(workloads.config(0), rebalance_interval=32)
+    for _ in range(run.wl.steps):
+        run.step(append=False)
+    run.check_state("all", "end")
+    assert run.cache.stats()["n_evicted"] == 40  # with a fixed context nothing is deleted after prefill
+    run.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, quant_bits=2),
+    dict(dtype="fp16", head_dim=64, quant_bits=2),
+    dict(dtype="bf16", head_dim=64, n_q_heads=7, n_kv_heads=1),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1, window=64, group_size=64, context=2048),
+    dict(dtype="bf16", head_dim=128, n_q_heads=4, n_kv_heads=2, window=64, group_size=32, context=2048, quant_bits=2),
+    dict(dtype="fp16", head_dim=128, n_q_heads=2, n_kv_heads=2, window=64, group_size=64, context=2048, quant_bits=2),
+    dict(dtype="fp16", head_dim=64, n_q_heads=3, n_kv_heads=1, window=64, group_size=32, context=2048),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, outlier_channels=4, outlier_scale=8.0),
+], ids=lambda kw: "-".join("%s%s" % (k[0], v) for k, v in kw.items()))
+def test_shapes_lockstep(kw):
+    ls = _lockstep()
+    wl = _small("small", steps=2 * kw.get("window", 32) + 6, **kw)
+    run = ls.LockstepRun(wl, rebalance_interval=3)
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    run.close()
+
+
+def test_multiple_units_and_layers():
+    ls = _lockstep()
+    wl = _small("multi", batch=3, n_layers=2, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, steps=40)
+    run = ls.LockstepRun(wl, rebalance_interval=2)
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    run.close()
+
+
+def test_per_layer_calls_match_all_layer_call():
+    """layer >= 0 calls on one layer give the same bits as the layer == -1 launch."""
+    ls = _lockstep()
+    wl = _small("perlayer", batch=2, n_layers=2, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, steps=8)
+    run = ls.LockstepRun(wl, oracle_units=[])
+    cache2 = binding.QEvictCache(ls.gpu_config(wl))
+    dev = run.dev
+    for layer in range(2):
+        units = [layer * 2, layer * 2 + 1]
+        k = torch.stack([workloads.gen_prompt_kv(wl, u)[0] for u in units]).to(dev)
+        v = torch.stack([workloads.gen_prompt_kv(wl, u)[1] for u in units]).to(dev)
+        s = torch.stack([run.scores[u] for u in units]).to(dev)
+        cache2.prefill_assign(layer, k, v, s)
+    for t in range(wl.steps):
+        out_all = run.step(append=True, check_mass=False)
+        for layer in range(2):
+            units = [layer * 2, layer * 2 + 1]
+            q = torch.stack([run.queries[u][t] for u in units]).to(dev)
+            kn = torch.stack([run.new_kv[u][0][t] for u in units]).to(dev)
+            vn = torch.stack([run.new_kv[u][1][t] for u in units]).to(dev)
+            o = cache2.decode_attn(layer, q, kn, vn).cpu()
+            assert torch.equal(o, out_all[units[0]:units[1] + 1])
+            cache2.rebalance(layer)
+    for u in range(4):
+        a = run.cache.export_tables(u // 2, u % 2)
+        b = cache2.export_tables(u // 2, u % 2)
+        for key in a:
+            assert torch.equal(a[key], b[key]), key
+    cache2.close()
+    run.close()
+
+
+def test_split_count_changes_only_rounding_order():
+    ls = _lockstep()
+    wl = replace(workloads.config(0), steps=6)
+    outs = []
+    for splits in (1, 3, 16):
+        run = ls.LockstepRun(wl, oracle_units=[])
+        run.cache.set_splits(splits)
+        o = [run.step(append=True, check_mass=False).double() for _ in range(wl.steps)]
+        imp = run.cache.export_tables(0, 0)["importance"].double()
+        outs.append((torch.stack(o), imp))
+        run.close()
+    for o, imp in outs[1:]:
+        assert torch.allclose(o, outs[0][0], atol=2e-3, rtol=1e-2)
+        assert torch.allclose(imp, outs[0][1], rtol=1e-5, atol=1e-7)
+
+
+def test_runs_are_bit_reproducible():
+    ls = _lockstep()
+    wl = _small("repro", dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, steps=20)
+    res = []
+    for _ in range(2):
+        run = ls.LockstepRun(wl, oracle_units=[])
+        o = torch.stack([run.step(append=True, check_mass=False) for _ in range(wl.steps)])
+        tab = run.cache.export_tables(0, 0)
+        res.append((o, tab))
+        run.close()
+    assert torch.equal(res[0][0], res[1][0])
+    for key in res[0][1]:
+        assert torch.equal(res[0][1][key], res[1][1][key]), key
+
+
+def test_everything_full_precision_equals_plain_attention():
+    """With the full-precision budget covering the whole context the output is ordinary attention."""
+    wl = _small("allfp", dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, context=512, fp_budget_windows=24,
+                q_budget_windows=2, steps=10)
+    ls = _lockstep()
+    run = ls.LockstepRun(wl)
+    k, v = workloads.gen_prompt_kv(wl, 0)
+    ks, vs = [k.double()], [v.double()]
+    for t in range(wl.steps):
+        out = run.step(append=True)[0].double()
+        ks.append(run.new_kv[0][0][t].double()[:, None]); vs.append(run.new_kv[0][1][t].double()[:, None])
+        kk = torch.cat(ks, 1).repeat_interleave(4, 0); vv = torch.cat(vs, 1).repeat_interleave(4, 0)
+        q = run.queries[0][t].double()
+        p = torch.softmax(torch.einsum("hd,hnd->hn", q, kk) / np.sqrt(wl.head_dim), -1)
+        ref = torch.einsum("hn,hnd->hd", p, vv)
+        assert torch.all((out - ref).abs() <= 2e-3 + 1e-2 * ref.abs())
+    assert run.cache.stats()["n_evicted"] == 0
+    run.close()
+
+
+def test_host_buffer_entry_point_matches_device_call():
+    ls = _lockstep()
+    wl = _small("host", dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, steps=5, batch=2)
+    a = ls.LockstepRun(wl, oracle_units=[])
+    b = ls.LockstepRun(wl, oracle_units=[])
+    for t in range(wl.steps):
+        oa = a.step(append=True, check_mass=False)
+        q = torch.stack([b.queries[u][t] for u in range(2)]).contiguous().pin_memory()
+        kn = torch.stack([b.new_kv[u][0][t] for u in range(2)]).contiguous().pin_memory()
+        vn = torch.stack([b.new_kv[u][1][t] for u in range(2)]).contiguous().pin_memory()
+        out = torch.empty_like(q).pin_memory()
+        b.cache.decode_attn_host(-1, q, kn, vn, out)
+        b.cache.rebalance(-1)
+        assert torch.equal(out, oa)
+    a.close(); b.close()
+
+
+def test_call_order_errors():
+    wl = _small("errors", rebalance_interval=32, steps=200)
+    ls = _lockstep()
+    cache = binding.QEvictCache(ls.gpu_config(wl))
+    q = torch.zeros((1, 1, wl.n_q_heads, wl.head_dim), dtype=torch.float16, device="cuda")
+    with pytest.raises(binding.QEvictError) as e:
+        cache.decode_attn(-1, q)
+    assert e.value.status == 2
+    with pytest.raises(binding.QEvictError) as e:
+        cache.rebalance(0)
+    assert e.value.status == 2
+    k, v = workloads.gen_prompt_kv(wl, 0)
+    s = workloads.synthetic_window_scores(wl, 0)
+    cache.prefill_assign(0, k[None].cuda(), v[None].cuda(), s[None].cuda())
+    with pytest.raises(binding.QEvictError) as e:
+        cache.prefill_assign(0, k[None].cuda(), v[None].cuda(), s[None].cuda())
+    assert e.value.status == 2
+    # appending without ever rebalancing runs out of pages for aged windows: refused on the host
+    kn = torch.zeros((1, 1, wl.n_kv_heads, wl.head_dim), dtype=torch.float16, device="cuda")
+    with pytest.raises(binding.QEvictError) as e:
+        for _ in range(10 * wl.window):
+            cache.decode_attn(-1, q, kn, kn)
+    assert e.value.status == 2
+    cache.rebalance(-1)
+    cache.decode_attn(-1, q, kn, kn)
+    assert cache.stats()["n_aged"] == 0
+    cache.close()
+
+
+def test_config1_llama_shape_lockstep():
+    ls = _lockstep()
+    wl = replace(workloads.config(1), steps=40)
+    run = ls.LockstepRun(wl)
+    run.check_state("all", "after prefill")
+    st = run.cache.stats()
+    assert (st["n_full"], st["n_quant"], st["n_evicted"]) == (64, 128, 832)
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    assert run.cache.stats()["promotions"] == run.oracles[0].stats["promotions"]
+    run.close()
