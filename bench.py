@@ -1,0 +1,381 @@
+"""Benchmark of the decode hot path: one step = append + tiered attention + mass update (decode_attn)
+followed by one routing event (rebalance) over every (layer, sequence) unit of a synthetic workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--layers L] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is whole-workload decode steps per second with all inputs resident in
+HBM; `e2e` is the same loop through the host-buffer entry point (H2D of q/k_new/v_new and D2H of the
+output inside the timed region); `roofline` is the attention kernel's algorithmic bytes per launch
+over its CUDA-event duration, against the measured HBM copy bandwidth; `cpu_baseline` is the CPU
+oracle timed on a bounded sample of the same workload on this host.
+"""
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_05326_b200 import workloads  # noqa: E402
+
+METRIC = "decode_steps_per_sec"
+UNIT = "steps/s"
+HBM_FALLBACK_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures
+# summarised under profiles/ (bytes per launch, keyed by workload name); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=None, help="stacked layers (config 1 defaults to 32)")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--bits", type=int, default=None, help="config 4 sweep point")
+    ap.add_argument("--fp-frac", type=float, default=None, help="config 4 sweep point")
+    ap.add_argument("--rebalance-interval", type=int, default=1)
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    return ap.parse_args()
+
+
+def make_workload(args, total_steps):
+    kw = {}
+    if args.config == 4:
+        if args.bits is not None:
+            kw["bits"] = args.bits
+        if args.fp_frac is not None:
+            kw["fp_frac"] = args.fp_frac
+    wl = workloads.config(args.config, **kw)
+    layers = args.layers if args.layers is not None else (32 if args.config == 1 else (8 if args.config == 3 else wl.n_layers))
+    batch = args.batch if args.batch is not None else wl.batch
+    return replace(wl, n_layers=layers, batch=batch, steps=total_steps, rebalance_interval=args.rebalance_interval)
+
+
+def peak_hbm_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) >= 7:
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------ ours
+def build_inputs(wl, device):
+    """All inputs of the run, resident on `device`: prompts are consumed by prefill layer by layer."""
+    scores, queries, knew, vnew = [], [], [], []
+    prompts = {}
+    for u in range(wl.n_units):
+        k, v = workloads.gen_prompt_kv(wl, u, device=device)
+        s = workloads.place_planted(workloads.synthetic_window_scores(wl, u), workloads.planted_windows(wl, u),
+                                    wl.fp_budget_windows, wl.q_budget_windows)
+        scores.append(s)
+        queries.append(workloads.gen_queries(wl, u, k, s, device=device))
+        kn, vn = workloads.gen_new_kv(wl, u, device=device)
+        knew.append(kn); vnew.append(vn)
+        prompts[u] = (k, v)
+        yield_layer = (u + 1) % wl.batch == 0
+        if yield_layer:
+            layer = u // wl.batch
+            units = range(layer * wl.batch, (layer + 1) * wl.batch)
+            yield ("layer", layer, torch.stack([prompts[x][0] for x in units]), torch.stack([prompts[x][1] for x in units]),
+                   torch.stack([scores[x] for x in units]).to(device))
+            for x in units:
+                del prompts[x]
+    shape_q = (wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim)
+    shape_kv = (wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim)
+    q = torch.stack(queries, 1).reshape((wl.steps,) + shape_q).contiguous()
+    kn = torch.stack(knew, 1).reshape((wl.steps,) + shape_kv).contiguous()
+    vn = torch.stack(vnew, 1).reshape((wl.steps,) + shape_kv).contiguous()
+    yield ("steps", q, kn, vn)
+
+
+def attention_kernel_bytes(wl, stats, n_splits_hint=None):
+    """Algorithmic bytes one attention-kernel launch must move: every live window once (Full and recent
+    windows at 16 bit, Quantized windows as codes + parameters), the queries, the work list, and the
+    partial results it writes."""
+    m_f, m_q = wl.fp_window_bytes(), wl.q_window_bytes()
+    kv = (stats["n_full"] + stats["n_aged"]) * m_f + stats["n_quant"] * m_q + stats["n_open"] * m_f // 2
+    live = stats["n_full"] + stats["n_aged"] + stats["n_quant"] + stats["n_open"]
+    q_bytes = wl.n_units * wl.n_q_heads * wl.head_dim * 2
+    lists = live * 8 + live * wl.n_q_heads * 8  # work list read, per-(head, window) records written
+    return kv + q_bytes + lists
+
+
+def run_ours(args, rank, world):
+    from paper_2608_05326_b200 import binding, build
+    if rank == 0:
+        build.build()  # no-op when the in-tree library is newer than its sources
+    if world > 1:
+        torch.distributed.barrier()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    K, W = args.steps, args.warmup
+    phases = 2 + (0 if args.no_e2e else 1)
+    total_steps = W + phases * K
+    wl = make_workload(args, total_steps)
+    wl = replace(wl, seed=wl.seed + rank)  # every rank owns its own sequences (weak scaling, no exchange)
+    cfg = binding.make_config(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window,
+                              wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
+                              rebalance_interval_hint=args.rebalance_interval, device=dev.index)
+    cache = binding.QEvictCache(cfg)
+    if args.splits:
+        cache.set_splits(args.splits)
+    q = kn = vn = None
+    for item in build_inputs(wl, dev):
+        if item[0] == "layer":
+            _, layer, k, v, s = item
+            cache.prefill_assign(layer, k, v, s)
+            torch.cuda.synchronize()
+            del k, v
+        else:
+            _, q, kn, vn = item
+    out = torch.empty_like(q[0])
+    R = args.rebalance_interval
+    append = not args.fixed_context
+
+    def step(t):
+        cache.decode_attn(-1, q[t], kn[t] if append else None, vn[t] if append else None, out)
+        if (t + 1) % R == 0:
+            cache.rebalance(-1)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(W):
+        step(t); t += 1
+    # ---- timed region: device-resident inputs ----
+    launches0 = cache.launch_count()
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        step(t); t += 1
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = cache.launch_count() - launches0
+    # ---- same loop with the attention kernel bracketed by events ----
+    cache.set_kernel_timing(True)
+    for _ in range(K):
+        step(t); t += 1
+    torch.cuda.synchronize()
+    kernel_ms, kernel_n = cache.kernel_time()
+    cache.set_kernel_timing(False)
+    stats = cache.stats()
+    # ---- end to end: host buffers through the host entry point ----
+    e2e = None
+    if not args.no_e2e:
+        qh = q[t:t + K].cpu().pin_memory(); knh = kn[t:t + K].cpu().pin_memory(); vnh = vn[t:t + K].cpu().pin_memory()
+        outh = torch.empty_like(qh[0]).pin_memory()
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(K):
+            cache.decode_attn_host(-1, qh[i], knh[i] if append else None, vnh[i] if append else None, outh)
+            if (t + i + 1) % R == 0:
+                cache.rebalance(-1)
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        h2d = qh[0].numel() * 2 + (2 * knh[0].numel() * 2 if append else 0)
+        e2e = {"seconds": e2e_s, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": outh.numel() * 2}
+
+    if world > 1:
+        tm = torch.tensor([ms, e2e["seconds"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(tm, op=torch.distributed.ReduceOp.MAX)
+        ms = float(tm[0]);
+        if e2e:
+            e2e["seconds"] = float(tm[1])
+    if rank != 0:
+        cache.close()
+        return None
+    peak, peak_kind = peak_hbm_gbs()
+    kbytes = attention_kernel_bytes(wl, stats)
+    k_avg_ms = kernel_ms / max(kernel_n, 1)
+    achieved = kbytes / (k_avg_ms * 1e-3) / 1e9 if k_avg_ms > 0 else 0.0
+    line = {
+        "metric": METRIC, "value": world * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+        "data": "synthetic",
+        "config": {
+            "workload": "%s x %d layers x batch %d (layer-batched launches)" % (wl.name, wl.n_layers, wl.batch),
+            "units_per_step": wl.n_units, "context": wl.context, "window": wl.window, "quant_bits": wl.quant_bits,
+            "group_size": wl.group_size, "fp_budget_windows": wl.fp_budget_windows,
+            "q_budget_windows": wl.q_budget_windows, "rebalance_interval": R, "append": append,
+            "l2": "inputs larger than L2 (KV working set %.0f MB per step)" % (kbytes / 1e6),
+        },
+        "layer_steps_per_sec": world * K * wl.n_units / (ms * 1e-3),
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "roofline": {
+            "bound": "hbm", "kernel": "decode_attn_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth", "frac_of_8TBs": achieved / 8000.0,
+            "bytes_per_launch": kbytes, "kernel_ms": k_avg_ms, "kernel_launches_timed": int(kernel_n),
+            "kernel_share_of_step": k_avg_ms / (ms / K),
+            "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+        },
+        "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_open", "n_evicted", "promotions",
+                                             "quantizations", "reactivations", "deletions")},
+    }
+    if e2e:
+        line["e2e"] = {"value": world * K / e2e["seconds"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d_bytes_per_step"],
+                       "d2h_bytes_per_step": e2e["d2h_bytes_per_step"]}
+    cache.close()
+    return line, wl
+
+
+# ------------------------------------------------------------------------------------- CPU oracle
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def time_oracle(wl, n_steps, warmup, budget_s):
+    """Times the CPU oracle, as it stands, on unit 0 of the workload: `n_steps` decode + rebalance steps
+    (at most `budget_s` seconds).  Returns (whole-workload steps/s, description)."""
+    import numpy as np
+
+    from oracle import OracleConfig, UnitOracle
+    aged = (wl.rebalance_interval + wl.window - 1) // wl.window + 1
+    ocfg = OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
+                        wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged)
+    k, v = workloads.gen_prompt_kv(wl, 0)
+    s = workloads.place_planted(workloads.synthetic_window_scores(wl, 0), workloads.planted_windows(wl, 0),
+                                wl.fp_budget_windows, wl.q_budget_windows)
+    q = workloads.gen_queries(wl, 0, k, s).double().numpy()
+    kn, vn = workloads.gen_new_kv(wl, 0)
+    kn, vn = kn.double().numpy(), vn.double().numpy()
+    orc = UnitOracle(ocfg)
+    orc.prefill_assign(k.double().numpy(), v.double().numpy(), s.numpy())
+    del k, v
+    t = 0
+    for _ in range(warmup):
+        orc.decode_attn(q[t], kn[t], vn[t]); orc.rebalance(); t += 1
+    done = 0
+    t0 = time.perf_counter()
+    while done < n_steps and t < q.shape[0] and time.perf_counter() - t0 < budget_s:
+        orc.decode_attn(q[t], kn[t], vn[t])
+        if (t + 1) % wl.rebalance_interval == 0:
+            orc.rebalance()
+        t += 1; done += 1
+    dt = time.perf_counter() - t0
+    unit_steps_per_s = done / dt
+    value = unit_steps_per_s / wl.n_units
+    sample = "unit 0 of %d, %d decode+rebalance steps in %.1f s" % (wl.n_units, done, dt)
+    return value, sample, done, dt
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return None
+    K, W = args.steps, args.warmup
+    wl = make_workload(args, max(W + K, 8))
+    value, sample, done, dt = time_oracle(wl, K, W, budget_s=180.0)
+    cores = oracle_threads()
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": done,
+        "warmup": W, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s x %d layers x batch %d" % (wl.name, wl.n_layers, wl.batch), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        line = run_reference(args, rank)
+        if line is not None:
+            print(json.dumps(line))
+        return
+    if world > 1:
+        torch.distributed.init_process_group("nccl")
+    res = run_ours(args, rank, world)
+    if rank == 0:
+        line, wl = res
+        if not args.no_cpu_baseline and world >= 1:
+            small = replace(wl, steps=256, seed=wl.seed)
+            value, sample, _, _ = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds)
+            line["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample}
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -189,6 +189,12 @@ QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, in
  * floating-point summation order. */
 QEVICT_API qevict_status qevict_set_splits(qevict_handle h, int32_t splits);
 
+/* Instrumentation: while enabled, every decode call brackets its attention kernel (the dominant
+ * kernel of the path) with CUDA events on the call's stream.  qevict_kernel_time synchronises on the
+ * recorded events, returns their summed duration in milliseconds and their count, and forgets them. */
+QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enable);
+QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches);
+
 /* Number of kernels this handle has launched since creation (host counter). */
 QEVICT_API uint64_t qevict_launch_count(qevict_handle h);
 

@@ -52,6 +52,8 @@ _SIGNATURES = {
     "qevict_create": (C.c_int, [C.POINTER(qevict_config), C.c_void_p, C.c_uint64, C.POINTER(C.c_void_p)]),
     "qevict_destroy": (C.c_int, [C.c_void_p]),
     "qevict_set_splits": (C.c_int, [C.c_void_p, C.c_int32]),
+    "qevict_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32]),
+    "qevict_kernel_time": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
     "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -154,6 +156,16 @@ def qevict_set_splits(h, splits):
     _check(lib().qevict_set_splits(h, splits), h)
 
 
+def qevict_set_kernel_timing(h, enable):
+    _check(lib().qevict_set_kernel_timing(h, int(enable)), h)
+
+
+def qevict_kernel_time(h):
+    ms, n = C.c_double(), C.c_uint64()
+    _check(lib().qevict_kernel_time(h, C.byref(ms), C.byref(n)), h)
+    return ms.value, n.value
+
+
 def qevict_get_stats(h, layer=-1):
     st = qevict_stats()
     _check(lib().qevict_get_stats(h, layer, C.byref(st)), h)
@@ -212,6 +224,13 @@ class QEvictCache:
 
     def set_splits(self, splits):
         qevict_set_splits(self.handle, splits)
+
+    def set_kernel_timing(self, enable):
+        qevict_set_kernel_timing(self.handle, enable)
+
+    def kernel_time(self):
+        """(summed milliseconds, launches) of the attention kernel since the last call."""
+        return qevict_kernel_time(self.handle)
 
     def stats(self, layer=-1):
         return qevict_get_stats(self.handle, layer)

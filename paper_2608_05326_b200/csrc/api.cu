@@ -45,6 +45,9 @@ struct qevict_ctx {
   decode_launch_fn decode_fn = nullptr;
   int forced_splits = 0;
   int sm_count = SM_COUNT_FALLBACK;
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
+  size_t ev_used = 0;
   char* stage_q = nullptr;    // device staging for the host-buffer entry point
   char* stage_k = nullptr;
   char* stage_v = nullptr;
@@ -230,7 +233,21 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (h->timing) {
+    if (h->ev_used + 2 > h->ev_pool.size()) {
+      cudaEvent_t e0, e1;
+      QE_CUDA(h, cudaEventCreate(&e0));
+      QE_CUDA(h, cudaEventCreate(&e1));
+      h->ev_pool.push_back(e0);
+      h->ev_pool.push_back(e1);
+    }
+    ev0 = h->ev_pool[h->ev_used]; ev1 = h->ev_pool[h->ev_used + 1];
+    h->ev_used += 2;
+    QE_CUDA(h, cudaEventRecord(ev0, stream));
+  }
   QE_CUDA(h, h->decode_fn(p, a.n_units, stream));
+  if (ev1) QE_CUDA(h, cudaEventRecord(ev1, stream));
   h->launches++;
   QE_CUDA(h, launch_combine(a, p.S, out, stream));
   h->launches++;
@@ -344,7 +361,29 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
 
 QEVICT_API qevict_status qevict_destroy(qevict_handle h) {
   if (!h) return QEVICT_ERR_INVALID_ARG;
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   delete h;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enable) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  h->timing = enable != 0;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches) {
+  if (!h || !total_ms || !n_launches) return QEVICT_ERR_INVALID_ARG;
+  double sum = 0.0;
+  for (size_t i = 0; i + 1 < h->ev_used; i += 2) {
+    QE_CUDA(h, cudaEventSynchronize(h->ev_pool[i + 1]));
+    float ms = 0.f;
+    QE_CUDA(h, cudaEventElapsedTime(&ms, h->ev_pool[i], h->ev_pool[i + 1]));
+    sum += ms;
+  }
+  *total_ms = sum;
+  *n_launches = h->ev_used / 2;
+  h->ev_used = 0;
   return QEVICT_OK;
 }
 

@@ -12,7 +12,8 @@
 //
 // Per 32-token tile:  S = Q K^T with the (<= 8) grouped heads on the M side of mma.m16n8k16 and
 // tokens on N, softmax in fp32 in the log2 domain, O^T += V^T P^T with channels on M, tokens on K and
-// heads on N, so the probability fragments feed the second product without any shuffle.  Pages are
+// heads on N, so the probability fragments feed the second product without any shuffle; the
+// probabilities enter it as a 16-bit value plus its rounding residual (two products per fragment).  Pages are
 // stored fragment-major (layout.cuh): a full-precision tile is read with 16-byte loads that are
 // already operands; a quantized tile is read as packed words, and codes become operands in
 // registers with one exact subtract and one fused multiply-add per pair.
@@ -108,21 +109,23 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)
 
 // ---- O^T += V^T P^T for one tile --------------------------------------------------------------------
 template <class T, int D, class LD>
-__device__ __forceinline__ void pv_fp_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2], const uint4* vt,
-                                           int lane, LD ld) {
+__device__ __forceinline__ void pv_fp_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2],
+                                           const uint32_t (&pb)[2][2], const uint4* vt, int lane, LD ld) {
 #pragma unroll
   for (int i = 0; i < D / 16; ++i) {
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks) {
       const uint4 vv = ld(vt + (i * 2 + ks) * 32 + lane);
       mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pa[ks][0], pa[ks][1]);
+      mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pb[ks][0], pb[ks][1]);
     }
   }
 }
 
 template <class T, int D, int BITS, int GROUP, class LD>
-__device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2], const uint4* vc,
-                                          const uint4* vp, int lane, LD ld) {
+__device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2],
+                                          const uint32_t (&pb)[2][2], const uint4* vc, const uint4* vp, int lane,
+                                          LD ld) {
   constexpr int MT = D / 16;
   constexpr int WPL = 32 * D * BITS / 8 / 128;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
@@ -152,24 +155,32 @@ __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t 
         const uint32_t a2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, pr.z, pr.w);
         const uint32_t a3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, pr.z, pr.w);
         mma16816<T>(o[i], a0, a1, a2, a3, pa[ks][0], pa[ks][1]);
+        mma16816<T>(o[i], a0, a1, a2, a3, pb[ks][0], pb[ks][1]);
       }
     }
   }
   (void)MT;
 }
 
-template <class T> __device__ __forceinline__ uint32_t pack_pair(float lo, float hi);
-template <> __device__ __forceinline__ uint32_t pack_pair<__half>(float lo, float hi) {
-  return as_u32(__floats2half2_rn(lo, hi));
+// Two probabilities -> a 16-bit pair plus the pair of rounding residuals.  The PV product is taken with
+// both (P = P_main + P_res), so the 8 (11) significand bits of the operand type do not limit the output.
+template <class T> __device__ __forceinline__ void split_pair(float lo, float hi, uint32_t& main, uint32_t& res);
+template <> __device__ __forceinline__ void split_pair<__half>(float lo, float hi, uint32_t& main, uint32_t& res) {
+  const __half2 m = __floats2half2_rn(lo, hi);
+  main = as_u32(m);
+  res = as_u32(__floats2half2_rn(lo - __low2float(m), hi - __high2float(m)));
 }
-template <> __device__ __forceinline__ uint32_t pack_pair<__nv_bfloat16>(float lo, float hi) {
-  return as_u32(__floats2bfloat162_rn(lo, hi));
+template <> __device__ __forceinline__ void split_pair<__nv_bfloat16>(float lo, float hi, uint32_t& main, uint32_t& res) {
+  const __nv_bfloat162 m = __floats2bfloat162_rn(lo, hi);
+  main = as_u32(m);
+  res = as_u32(__floats2bfloat162_rn(lo - __low2float(m), hi - __high2float(m)));
 }
 
 // Online softmax update for one tile; returns the probability fragments for the PV product.
 template <class T, int MT>
 __device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float scale_log2, int lane, float& m_run,
-                                             float& l_run, float& wsum, float (&o)[MT][4], uint32_t (&pa)[2][2]) {
+                                             float& l_run, float& wsum, float (&o)[MT][4], uint32_t (&pa)[2][2],
+                                             uint32_t (&pb)[2][2]) {
   const int t = lane & 3;
   float x[4][2];
   float tmax = -INFINITY;
@@ -209,10 +220,10 @@ __device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float s
   for (int i = 0; i < MT; ++i) {
     o[i][0] *= a_lo; o[i][1] *= a_hi; o[i][2] *= a_lo; o[i][3] *= a_hi;
   }
-  pa[0][0] = pack_pair<T>(p[0][0], p[0][1]);
-  pa[0][1] = pack_pair<T>(p[1][0], p[1][1]);
-  pa[1][0] = pack_pair<T>(p[2][0], p[2][1]);
-  pa[1][1] = pack_pair<T>(p[3][0], p[3][1]);
+  split_pair<T>(p[0][0], p[0][1], pa[0][0], pb[0][0]);
+  split_pair<T>(p[1][0], p[1][1], pa[0][1], pb[0][1]);
+  split_pair<T>(p[2][0], p[2][1], pa[1][0], pb[1][0]);
+  split_pair<T>(p[3][0], p[3][1], pa[1][1], pb[1][1]);
 }
 
 template <class T, int D, int BITS, int GROUP, int TILES>
@@ -265,9 +276,9 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32) decode_attn_kernel(const De
 #pragma unroll
         for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
         qk_fp_tile<T, D>(sacc, qa, kt, lane, ld);
-        uint32_t pa[2][2];
-        softmax_tile<T, MT>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa);
-        pv_fp_tile<T, D>(o, pa, vt, lane, ld);
+        uint32_t pa[2][2], pb[2][2];
+        softmax_tile<T, MT>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+        pv_fp_tile<T, D>(o, pa, pb, vt, lane, ld);
       }
     } else {
       const char* base = p.q_pool + ((size_t)u * p.PQ + page) * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
@@ -282,9 +293,9 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32) decode_attn_kernel(const De
 #pragma unroll
         for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
         qk_q_tile<T, D, BITS>(sacc, qa, kc, kp, lane, ld);
-        uint32_t pa[2][2];
-        softmax_tile<T, MT>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa);
-        pv_q_tile<T, D, BITS, GROUP>(o, pa, vc, vp, lane, ld);
+        uint32_t pa[2][2], pb[2][2];
+        softmax_tile<T, MT>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+        pv_q_tile<T, D, BITS, GROUP>(o, pa, pb, vc, vp, lane, ld);
       }
     }
     if (t == 0 && g < p.G) {

@@ -189,14 +189,15 @@ def gen_queries(wl, unit, k_prompt, scores=None, n_steps=None, device="cpu"):
     focus_on = torch.rand(n, generator=gq) < 0.5
     steer = torch.rand(n, generator=gq) < 0.10
     walk = torch.randn(n, generator=gq) * 4.0
-    kp = k_prompt.to(device="cpu", dtype=torch.float32) if k_prompt.device.type != "cpu" or \
-        k_prompt.dtype != torch.float32 else k_prompt
+    cache = {}
 
     def anchor_keys(win):  # [H_q, d] key of the centre token of window `win`, expanded over the GQA group
-        a = win * w + w // 2
-        ka = kp[:, a, :]  # [H_kv, d]
-        beta = 0.75 * d / (ka * ka).sum(-1, keepdim=True).clamp_min(1e-6)
-        return (beta * ka).repeat_interleave(group, dim=0)
+        if win not in cache:
+            a = win * w + w // 2
+            ka = k_prompt[:, a, :].to(device="cpu", dtype=torch.float32)  # [H_kv, d]
+            beta = 0.75 * d / (ka * ka).sum(-1, keepdim=True).clamp_min(1e-6)
+            cache[win] = (beta * ka).repeat_interleave(group, dim=0)
+        return cache[win]
 
     q = eps.clone()
     planted = planted_windows(wl, unit)
