@@ -1,6 +1,7 @@
 // Host side of the C ABI: validation, workspace carving, call-order bookkeeping, kernel launches.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -178,15 +179,20 @@ KernelArgs make_args(qevict_handle h, int l0, int l1) {
 // Splits per (unit, KV head): enough CTAs to fill the GPU in whole waves while every warp still walks
 // several windows.
 int choose_splits(const qevict_ctx* h, int n_units) {
-  if (h->forced_splits > 0) return h->forced_splits < MAX_SPLITS ? h->forced_splits : MAX_SPLITS;
   const Geometry& g = h->geo;
+  // a warp holds its work-list entries one per lane: at most 32 entries per warp
+  const int smin = (g.EMAX + 32 * DECODE_WARPS - 1) / (32 * DECODE_WARPS);
+  if (h->forced_splits > 0) {
+    const int f = h->forced_splits < smin ? smin : h->forced_splits;
+    return f < MAX_SPLITS ? f : MAX_SPLITS;
+  }
   const int entries = g.Kf + g.Kq + 1;
   const long pairs = (long)n_units * g.Hkv;
   const long slots = (long)h->sm_count * 3;  // resident CTAs
-  int best = 1;
+  int best = smin;
   double best_cost = 1e30;
   const int smax = entries / DECODE_WARPS < 1 ? 1 : (entries / DECODE_WARPS > MAX_SPLITS ? MAX_SPLITS : entries / DECODE_WARPS);
-  for (int s = 1; s <= smax; ++s) {
+  for (int s = smin; s <= (smax < smin ? smin : smax); ++s) {
     const long ctas = pairs * s;
     const long waves = (ctas + slots - 1) / slots;
     const double per_warp = ceil((double)entries / (s * DECODE_WARPS)) * g.tiles;
@@ -232,7 +238,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.q = q; p.entries = h->st.entries; p.n_live = h->st.n_live; p.open_fill = h->st.open_fill;
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
-  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
+  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (h->timing) {
     if (h->ev_used + 2 > h->ev_pool.size()) {
@@ -318,10 +324,10 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
   const size_t need = carve(g, (char*)device_mem, &h->st, h);
   if (need > bytes) { delete h; return QEVICT_ERR_NO_MEMORY; }
   switch ((g.dtype == QEVICT_DTYPE_BF16 ? 2 : 0) + (g.D == 128 ? 1 : 0)) {
-    case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles); break;
-    case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles); break;
-    case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles); break;
-    default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles); break;
+    case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles, g.G); break;
+    case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles, g.G); break;
+    case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles, g.G); break;
+    default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles, g.G); break;
   }
   if (!h->decode_fn) { delete h; return QEVICT_ERR_UNSUPPORTED; }
   h->layers.resize(g.n_layers);

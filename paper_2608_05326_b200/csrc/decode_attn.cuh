@@ -10,12 +10,19 @@
 // warp runs an independent online softmax over its windows; the four warps are merged in shared
 // memory and the CTA writes one partial (m, l, O) per query head of its KV head.
 //
+// Data movement: every warp owns a ring of NSLOT shared-memory slots.  Lane 0 streams the warp's
+// pages into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on one
+// mbarrier per slot) NSLOT-1 pieces ahead of the math; a page is stored fragment-major (layout.cuh),
+// so a piece is one contiguous run in global memory and every lane reads its operands from shared
+// memory with conflict-free 16-byte loads.  Waits on the mbarriers are bounded: a wait that runs out
+// records CHECK_COPY_TIMEOUT, the warp stops issuing, drains what it has in flight and returns.
+//
 // Per 32-token tile:  S = Q K^T with the (<= 8) grouped heads on the M side of mma.m16n8k16 and
 // tokens on N, softmax in fp32 in the log2 domain, O^T += V^T P^T with channels on M, tokens on K and
-// heads on N, so the probability fragments feed the second product without any shuffle; the
-// probabilities enter it as a 16-bit value plus its rounding residual (two products per fragment).  Pages are
-// stored fragment-major (layout.cuh): a full-precision tile is read with 16-byte loads that are
-// already operands; a quantized tile is read as packed words, and codes become operands in
+// heads on N, so the probability fragments feed the second product without any transposition.  The
+// probabilities enter it as a 16-bit value plus its rounding residual; with at most 4 heads per KV
+// head the residuals ride in the unused N columns 4..7 of the same product (PACK), otherwise they take
+// a second product.  A quantized tile is read as packed words, and codes become operands in
 // registers with one exact subtract and one fused multiply-add per pair.
 #pragma once
 
@@ -33,10 +40,14 @@ struct DecodeParams {
   float* o_part;          // [n_units][Hq][MAX_SPLITS][D]
   float* ml;              // [n_units][Hq][MAX_SPLITS][2]
   float2* wrec;           // [n_units][Hq][EMAX]
+  int32_t* status;
   int unit0, S, Hq, Hkv, G, EMAX, PF, PQ;
   uint32_t fp_page_bytes, q_page_bytes;
   float scale_log2;
 };
+
+static constexpr int NSLOT = 4;                   // ring slots per warp
+static constexpr uint32_t WAIT_LIMIT = 1u << 20;  // mbarrier try_wait attempts before giving up
 
 template <class T, int D, int BITS, int GROUP, int TILES>
 struct DecodeTraits {
@@ -53,45 +64,94 @@ struct DecodeTraits {
   static constexpr uint32_t KP_BYTES = D * 4;
   static constexpr uint32_t KP_OFF = TILES * Q_TILE_STRIDE;
   static constexpr uint32_t Q_HEAD_BYTES = KP_OFF + (W / GROUP) * KP_BYTES;
-  static constexpr int WPL = KC_BYTES / 128;  // code words per lane per tile (keys; same for values)
-  static constexpr int STEP = BITS;           // bit distance between consecutive pair slots
-  static constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
+  // a ring slot holds half of a full-precision key or value tile, or the key part (codes + params)
+  // or the value part (codes + params) of a quantized tile
+  static constexpr uint32_t SLOT_BYTES = FP_TILE_BYTES / 2;
+  static constexpr uint32_t RING_BYTES = DECODE_WARPS * NSLOT * SLOT_BYTES;
+  static constexpr uint32_t SMEM_BYTES = RING_BYTES + DECODE_WARPS * NSLOT * 8;
+  static_assert(KC_BYTES + KP_BYTES <= SLOT_BYTES && VC_BYTES + VP_BYTES <= SLOT_BYTES, "quantized part must fit a slot");
+  static_assert(8 * (D + 4) * 4 + 64 <= NSLOT * SLOT_BYTES, "merge buffer must fit the warp's ring");
 };
 
-// ---- S = Q K^T for one tile -----------------------------------------------------------------------
-template <class T, int D, class LD>
-__device__ __forceinline__ void qk_fp_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], const uint4* kt,
-                                           int lane, LD ld) {
+// ---- shared-memory / mbarrier / bulk-copy primitives -------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 lds16(uint32_t addr) {
+  uint4 r;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  return r;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait; false if the phase did not complete within WAIT_LIMIT attempts.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- S = Q K^T -----------------------------------------------------------------------------------------
+// Half of a full-precision key tile (16 tokens: score blocks j0, j0+1) from a ring slot.
+template <class T, int D>
+__device__ __forceinline__ void qk_fp_half(float (&s)[4][4], int j0, const uint32_t (&qa)[D / 16][2], uint32_t slot,
+                                           int lane) {
   constexpr int KG = D / 32;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int jj = 0; jj < 2; ++jj) {
 #pragma unroll
     for (int c = 0; c < KG; ++c) {
-      const uint4 kv = ld(kt + (j * KG + c) * 32 + lane);
-      mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, kv.x, kv.y);
-      mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, kv.z, kv.w);
+      const uint4 kv = lds16(slot + ((jj * KG + c) * 32 + lane) * 16);
+      mma16816<T>(s[j0 + jj], qa[2 * c][0], 0u, qa[2 * c][1], 0u, kv.x, kv.y);
+      mma16816<T>(s[j0 + jj], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, kv.z, kv.w);
     }
   }
 }
 
-template <class T, int D, int BITS, class LD>
-__device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], const uint4* kc,
-                                          const uint4* kp, int lane, LD ld) {
+// Key part of a quantized tile: codes at `slot`, parameters at `slot + KC_BYTES`.
+template <class T, int D, int BITS>
+__device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
   constexpr int KG = D / 32;
   constexpr int WPL = 32 * D * BITS / 8 / 128;
+  constexpr uint32_t KC_BYTES = 32 * D * BITS / 8;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
   const int t = lane & 3;
   uint32_t cw[WPL];
 #pragma unroll
   for (int v = 0; v < WPL / 4; ++v) {
-    const uint4 x = ld(kc + v * 32 + lane);
+    const uint4 x = lds16(slot + (v * 32 + lane) * 16);
     cw[4 * v] = x.x; cw[4 * v + 1] = x.y; cw[4 * v + 2] = x.z; cw[4 * v + 3] = x.w;
   }
+  const uint32_t kp = slot + KC_BYTES;
 #pragma unroll
   for (int c = 0; c < KG; ++c) {
-    const uint4 p0 = ld(kp + (c * 2 + 0) * 4 + t);  // k-step 2c:   {s,z} for the low / high channel octet
-    const uint4 p1 = ld(kp + (c * 2 + 1) * 4 + t);  // k-step 2c+1
+    const uint4 p0 = lds16(kp + ((c * 2 + 0) * 4 + t) * 16);  // k-step 2c:   {s,z} low / high channel octet
+    const uint4 p1 = lds16(kp + ((c * 2 + 1) * 4 + t) * 16);  // k-step 2c+1
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       uint32_t w;
@@ -107,40 +167,42 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)
   }
 }
 
-// ---- O^T += V^T P^T for one tile --------------------------------------------------------------------
-template <class T, int D, class LD>
-__device__ __forceinline__ void pv_fp_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2],
-                                           const uint32_t (&pb)[2][2], const uint4* vt, int lane, LD ld) {
+// ---- O^T += V^T P^T ----------------------------------------------------------------------------------------
+// Half of a full-precision value tile (channel blocks i0 .. i0 + MT/2 - 1) from a ring slot.
+template <class T, int D, bool PACK>
+__device__ __forceinline__ void pv_fp_half(float (&o)[D / 16][4], int i0, const uint32_t (&pa)[2][2],
+                                           const uint32_t (&pb)[2][2], uint32_t slot, int lane) {
 #pragma unroll
-  for (int i = 0; i < D / 16; ++i) {
+  for (int ii = 0; ii < D / 32; ++ii) {
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks) {
-      const uint4 vv = ld(vt + (i * 2 + ks) * 32 + lane);
-      mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pa[ks][0], pa[ks][1]);
-      mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pb[ks][0], pb[ks][1]);
+      const uint4 vv = lds16(slot + ((ii * 2 + ks) * 32 + lane) * 16);
+      mma16816<T>(o[i0 + ii], vv.x, vv.y, vv.z, vv.w, pa[ks][0], pa[ks][1]);
+      if (!PACK) mma16816<T>(o[i0 + ii], vv.x, vv.y, vv.z, vv.w, pb[ks][0], pb[ks][1]);
     }
   }
 }
 
-template <class T, int D, int BITS, int GROUP, class LD>
-__device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2],
-                                          const uint32_t (&pb)[2][2], const uint4* vc, const uint4* vp, int lane,
-                                          LD ld) {
-  constexpr int MT = D / 16;
+// Value part of a quantized tile: codes at `slot`, parameters at `slot + VC_BYTES`.
+template <class T, int D, int BITS, int GROUP, bool PACK>
+__device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2], const uint32_t (&pb)[2][2],
+                                          uint32_t slot, int lane) {
   constexpr int WPL = 32 * D * BITS / 8 / 128;
+  constexpr uint32_t VC_BYTES = 32 * D * BITS / 8;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
   const int t = lane & 3;
   uint32_t vw[WPL];
 #pragma unroll
   for (int v = 0; v < WPL / 4; ++v) {
-    const uint4 x = ld(vc + v * 32 + lane);
+    const uint4 x = lds16(slot + (v * 32 + lane) * 16);
     vw[4 * v] = x.x; vw[4 * v + 1] = x.y; vw[4 * v + 2] = x.z; vw[4 * v + 3] = x.w;
   }
+  const uint32_t vp = slot + VC_BYTES;
 #pragma unroll
   for (int gc = 0; gc < D / GROUP; ++gc) {
-    const uint4 pr0 = ld(vp + (gc * 2 + 0) * 4 + t);  // tokens 0..15:  {s,z} low octet, {s,z} high octet
-    const uint4 pr1 = ld(vp + (gc * 2 + 1) * 4 + t);  // tokens 16..31
+    const uint4 pr0 = lds16(vp + ((gc * 2 + 0) * 4 + t) * 16);  // tokens 0..15:  {s,z} low octet, {s,z} high octet
+    const uint4 pr1 = lds16(vp + ((gc * 2 + 1) * 4 + t) * 16);  // tokens 16..31
 #pragma unroll
     for (int ii = 0; ii < GROUP / 16; ++ii) {
       const int i = gc * (GROUP / 16) + ii;
@@ -155,11 +217,10 @@ __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t 
         const uint32_t a2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, pr.z, pr.w);
         const uint32_t a3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, pr.z, pr.w);
         mma16816<T>(o[i], a0, a1, a2, a3, pa[ks][0], pa[ks][1]);
-        mma16816<T>(o[i], a0, a1, a2, a3, pb[ks][0], pb[ks][1]);
+        if (!PACK) mma16816<T>(o[i], a0, a1, a2, a3, pb[ks][0], pb[ks][1]);
       }
     }
   }
-  (void)MT;
 }
 
 // Two probabilities -> a 16-bit pair plus the pair of rounding residuals.  The PV product is taken with
@@ -176,8 +237,8 @@ template <> __device__ __forceinline__ void split_pair<__nv_bfloat16>(float lo, 
   res = as_u32(__floats2bfloat162_rn(lo - __low2float(m), hi - __high2float(m)));
 }
 
-// Online softmax update for one tile; returns the probability fragments for the PV product.
-template <class T, int MT>
+// Online softmax update for one tile; leaves the probability fragments for the PV product in pa / pb.
+template <class T, int MT, bool PACK>
 __device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float scale_log2, int lane, float& m_run,
                                              float& l_run, float& wsum, float (&o)[MT][4], uint32_t (&pa)[2][2],
                                              uint32_t (&pb)[2][2]) {
@@ -187,23 +248,30 @@ __device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float s
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int tok = 8 * j + 2 * t + e;
-      x[j][e] = (tok < ntok) ? s[j][e] * scale_log2 : -INFINITY;
-      tmax = fmaxf(tmax, x[j][e]);
+    for (int e = 0; e < 2; ++e) x[j][e] = s[j][e] * scale_log2;
+  }
+  if (ntok < 32) {  // only the open window has unfilled token slots
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        if (8 * j + 2 * t + e >= ntok) x[j][e] = -INFINITY;
+      }
     }
   }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) tmax = fmaxf(tmax, fmaxf(x[j][0], x[j][1]));
   tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
   tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
   const float m_new = fmaxf(m_run, tmax);  // finite: the caller guarantees ntok >= 1
-  const float alpha = exp2f(m_run - m_new);
+  const float alpha = ex2(m_run - m_new);
   float rs = 0.f;
   float p[4][2];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      p[j][e] = exp2f(x[j][e] - m_new);
+      p[j][e] = ex2(x[j][e] - m_new);
       rs += p[j][e];
     }
   }
@@ -212,28 +280,51 @@ __device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float s
   l_run = l_run * alpha + rs;
   wsum = wsum * alpha + rs;
   m_run = m_new;
-  // the accumulators hold O^T: column pair (2t, 2t+1) = heads 2t and 2t+1, whose statistics live in
-  // the lane quads 2t and 2t+1
-  const float a_lo = __shfl_sync(0xffffffffu, alpha, (2 * t) * 4);
-  const float a_hi = __shfl_sync(0xffffffffu, alpha, (2 * t + 1) * 4);
+  if (__any_sync(0xffffffffu, alpha != 1.f)) {
+    // the accumulators hold O^T: column pair (2t, 2t+1) = heads 2t and 2t+1 (PACK: heads modulo 4),
+    // whose statistics live in the lane quads of those heads
+    const int h0 = PACK ? ((2 * t) & 3) : 2 * t;
+    const float a_lo = __shfl_sync(0xffffffffu, alpha, h0 * 4);
+    const float a_hi = __shfl_sync(0xffffffffu, alpha, (h0 + 1) * 4);
 #pragma unroll
-  for (int i = 0; i < MT; ++i) {
-    o[i][0] *= a_lo; o[i][1] *= a_hi; o[i][2] *= a_lo; o[i][3] *= a_hi;
+    for (int i = 0; i < MT; ++i) {
+      o[i][0] *= a_lo; o[i][1] *= a_hi; o[i][2] *= a_lo; o[i][3] *= a_hi;
+    }
   }
   split_pair<T>(p[0][0], p[0][1], pa[0][0], pb[0][0]);
   split_pair<T>(p[1][0], p[1][1], pa[0][1], pb[0][1]);
   split_pair<T>(p[2][0], p[2][1], pa[1][0], pb[1][0]);
   split_pair<T>(p[3][0], p[3][1], pa[1][1], pb[1][1]);
+  if (PACK) {
+    // heads live in rows 0..3; the lanes of rows 4..7 feed the residuals of head (row - 4) as extra
+    // N columns of the same product
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const uint32_t below = __shfl_sync(0xffffffffu, pb[ks][r], (lane + 16) & 31);
+        if (lane >= 16) pa[ks][r] = below;
+      }
+    }
+  }
 }
 
-template <class T, int D, int BITS, int GROUP, int TILES>
-__global__ void __launch_bounds__(DECODE_WARPS * 32) decode_attn_kernel(const DecodeParams p) {
+template <class T, int D, int BITS, int GROUP, int TILES, bool PACK>
+__global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const DecodeParams p) {
   using TT = DecodeTraits<T, D, BITS, GROUP, TILES>;
   constexpr int KS = TT::KS, MT = TT::MT;
+  extern __shared__ __align__(128) unsigned char smem[];
   const int s = blockIdx.x, hk = blockIdx.y, ul = blockIdx.z;
   const int u = p.unit0 + ul;
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  auto ld = [](const uint4* ptr) { return ld_stream16(ptr); };
+  const uint32_t ring = smem_u32(smem) + wid * NSLOT * TT::SLOT_BYTES;
+  const uint32_t bars = smem_u32(smem) + TT::RING_BYTES + wid * NSLOT * 8;
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < NSLOT; ++i) mbar_init(bars + i * 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
 
   // query fragments: row g of the A operand = head hk*G + g (rows >= G are zero)
   uint32_t qa[KS][2];
@@ -258,76 +349,155 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32) decode_attn_kernel(const De
   const int n_live = p.n_live[u];
   const int fill = p.open_fill[u];
   const int stride = p.S * DECODE_WARPS;
-  for (int e = s * DECODE_WARPS + wid; e < n_live; e += stride) {
-    const uint2 ent = p.entries[(size_t)u * p.EMAX + e];
-    const uint32_t kind = ent.x >> ENTRY_KIND_SHIFT;
-    const int page = (int)ent.y;
+  const int first = s * DECODE_WARPS + wid;
+  // this warp's entries, one per lane (the host picks S so that a warp never owns more than 32)
+  const int my_n = first < n_live ? min(32, (n_live - first + stride - 1) / stride) : 0;
+  uint2 my_ent = make_uint2(0u, 0u);
+  if (lane < my_n) my_ent = p.entries[(size_t)u * p.EMAX + first + (size_t)lane * stride];
+
+  // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
+  // piece counts: full-precision tile = 4 (K lo, K hi, V lo, V hi), quantized tile = 2 (K part, V part)
+  int n_pieces;
+  {
+    int mine = lane < my_n ? (((my_ent.x >> ENTRY_KIND_SHIFT) == KIND_Q) ? 2 : 4) * TILES : 0;
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o2);
+    n_pieces = mine;
+  }
+  int pr_ci = 0, pr_tile = 0, pr_part = 0, issued = 0, consumed = 0;
+  bool dead = false;
+  auto issue_next = [&]() {  // warp-collective
+    if (issued >= n_pieces || dead) return;
+    const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, pr_ci), ey = __shfl_sync(0xffffffffu, my_ent.y, pr_ci);
+    const bool isq = (ex >> ENTRY_KIND_SHIFT) == KIND_Q;
+    if (lane == 0) {
+      const int slot = issued % NSLOT;
+      const uint32_t dst = ring + slot * TT::SLOT_BYTES, bar = bars + slot * 8;
+      if (!isq) {
+        const char* src = p.fp_pool + ((size_t)u * p.PF + ey) * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES +
+                          (size_t)pr_tile * 2 * TT::FP_TILE_BYTES + (size_t)pr_part * TT::SLOT_BYTES;
+        mbar_expect_tx(bar, TT::SLOT_BYTES);
+        bulk_g2s(dst, src, TT::SLOT_BYTES, bar);
+      } else {
+        const char* base = p.q_pool + ((size_t)u * p.PQ + ey) * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
+        const char* tb = base + (size_t)pr_tile * TT::Q_TILE_STRIDE;
+        if (pr_part == 0) {
+          mbar_expect_tx(bar, TT::KC_BYTES + TT::KP_BYTES);
+          bulk_g2s(dst, tb, TT::KC_BYTES, bar);
+          bulk_g2s(dst + TT::KC_BYTES, base + TT::KP_OFF + (size_t)((pr_tile * 32) / GROUP) * TT::KP_BYTES, TT::KP_BYTES, bar);
+        } else {
+          mbar_expect_tx(bar, TT::VC_BYTES + TT::VP_BYTES);
+          bulk_g2s(dst, tb + TT::KC_BYTES, TT::VC_BYTES + TT::VP_BYTES, bar);
+        }
+      }
+    }
+    ++issued;
+    if (++pr_part == (isq ? 2 : 4)) {
+      pr_part = 0;
+      if (++pr_tile == TILES) { pr_tile = 0; ++pr_ci; }
+    }
+  };
+  // wait for the next piece in order; returns its slot address
+  auto acquire = [&]() -> uint32_t {
+    const int slot = consumed % NSLOT;
+    if (!dead && !mbar_wait(bars + slot * 8, (consumed / NSLOT) & 1)) {
+      dead = true;
+      if (lane == 0) record_check(p.status, CHECK_COPY_TIMEOUT);
+    }
+    return ring + slot * TT::SLOT_BYTES;
+  };
+  auto release = [&]() {  // all lanes have read the slot: hand it back to the producer
+    ++consumed;
+    __syncwarp();
+    issue_next();
+  };
+#pragma unroll 1
+  for (int i = 0; i < NSLOT; ++i) issue_next();
+
+#pragma unroll 1
+  for (int ci = 0; ci < my_n; ++ci) {
+    const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, ci);
+    const uint32_t kind = ex >> ENTRY_KIND_SHIFT;
+    const int e = first + ci * stride;
     const int valid = (kind == KIND_OPEN) ? fill : TT::W;
     float wsum = 0.f;
-    if (kind != KIND_Q) {
-      const char* base = p.fp_pool + ((size_t)u * p.PF + page) * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES;
 #pragma unroll 1
-      for (int tile = 0; tile < TILES; ++tile) {
-        const int ntok = valid - 32 * tile;
-        if (ntok <= 0) break;
-        const uint4* kt = reinterpret_cast<const uint4*>(base + (size_t)tile * 2 * TT::FP_TILE_BYTES);
-        const uint4* vt = kt + TT::FP_TILE_BYTES / 16;
-        float sacc[4][4];
+    for (int tile = 0; tile < TILES; ++tile) {
+      const int ntok = min(32, valid - 32 * tile);
+      float sacc[4][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
-        qk_fp_tile<T, D>(sacc, qa, kt, lane, ld);
-        uint32_t pa[2][2], pb[2][2];
-        softmax_tile<T, MT>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
-        pv_fp_tile<T, D>(o, pa, pb, vt, lane, ld);
-      }
-    } else {
-      const char* base = p.q_pool + ((size_t)u * p.PQ + page) * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
-#pragma unroll 1
-      for (int tile = 0; tile < TILES; ++tile) {
-        const char* tb = base + (size_t)tile * TT::Q_TILE_STRIDE;
-        const uint4* kc = reinterpret_cast<const uint4*>(tb);
-        const uint4* vc = reinterpret_cast<const uint4*>(tb + TT::KC_BYTES);
-        const uint4* vp = reinterpret_cast<const uint4*>(tb + TT::KC_BYTES + TT::VC_BYTES);
-        const uint4* kp = reinterpret_cast<const uint4*>(base + TT::KP_OFF + (size_t)((tile * 32) / GROUP) * TT::KP_BYTES);
-        float sacc[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
-        qk_q_tile<T, D, BITS>(sacc, qa, kc, kp, lane, ld);
-        uint32_t pa[2][2], pb[2][2];
-        softmax_tile<T, MT>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
-        pv_q_tile<T, D, BITS, GROUP>(o, pa, pb, vc, vp, lane, ld);
+      for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
+      uint32_t pa[2][2], pb[2][2];
+      if (kind != KIND_Q) {
+        uint32_t sl = acquire();
+        if (!dead && ntok > 0) qk_fp_half<T, D>(sacc, 0, qa, sl, lane);
+        release();
+        sl = acquire();
+        if (!dead && ntok > 0) {
+          qk_fp_half<T, D>(sacc, 2, qa, sl, lane);
+          softmax_tile<T, MT, PACK>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+        }
+        release();
+        sl = acquire();
+        if (!dead && ntok > 0) pv_fp_half<T, D, PACK>(o, 0, pa, pb, sl, lane);
+        release();
+        sl = acquire();
+        if (!dead && ntok > 0) pv_fp_half<T, D, PACK>(o, MT / 2, pa, pb, sl, lane);
+        release();
+      } else {
+        uint32_t sl = acquire();
+        if (!dead) {
+          qk_q_tile<T, D, BITS>(sacc, qa, sl, lane);
+          softmax_tile<T, MT, PACK>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+        }
+        release();
+        sl = acquire();
+        if (!dead) pv_q_tile<T, D, BITS, GROUP, PACK>(o, pa, pb, sl, lane);
+        release();
       }
     }
     if (t == 0 && g < p.G) {
       p.wrec[((size_t)u * p.Hq + (size_t)hk * p.G + g) * p.EMAX + e] = make_float2(wsum, m_run);
     }
   }
+  if (dead) {
+    // give the copies still in flight a bounded time to land before the shared memory is reused
+    for (int k = consumed; k < issued; ++k) mbar_wait(bars + (k % NSLOT) * 8, (k / NSLOT) & 1);
+  }
 
-  // ---- merge the four warps, write the split's partial ------------------------------------------
-  __shared__ float sm_m[DECODE_WARPS][8];
-  __shared__ float sm_l[DECODE_WARPS][8];
-  __shared__ float sm_o[DECODE_WARPS][8][D + 4];
-  if (t == 0) { sm_m[wid][g] = m_run; sm_l[wid][g] = l_run; }
+  // ---- merge the four warps (each parks its state in its own, now idle, ring), write the partial ------
+  // per-warp layout: float o[8][D + 4], then float m[8], float l[8]
+  constexpr int OSTR = D + 4;
+  float* my_o = reinterpret_cast<float*>(smem + wid * NSLOT * TT::SLOT_BYTES);
+  float* my_ml = my_o + 8 * OSTR;
+  if (t == 0) { my_ml[g] = m_run; my_ml[8 + g] = l_run; }
 #pragma unroll
   for (int i = 0; i < MT; ++i) {
-    sm_o[wid][2 * t][16 * i + g] = o[i][0];
-    sm_o[wid][2 * t + 1][16 * i + g] = o[i][1];
-    sm_o[wid][2 * t][16 * i + g + 8] = o[i][2];
-    sm_o[wid][2 * t + 1][16 * i + g + 8] = o[i][3];
+    my_o[(2 * t) * OSTR + 16 * i + g] = o[i][0];
+    my_o[(2 * t + 1) * OSTR + 16 * i + g] = o[i][1];
+    my_o[(2 * t) * OSTR + 16 * i + g + 8] = o[i][2];
+    my_o[(2 * t + 1) * OSTR + 16 * i + g + 8] = o[i][3];
   }
   __syncthreads();
   for (int idx = threadIdx.x; idx < p.G * D; idx += DECODE_WARPS * 32) {
     const int h = idx / D, ch = idx - h * D;
-    float mx = sm_m[0][h];
+    float mw[DECODE_WARPS];
+    float mx = -INFINITY;
 #pragma unroll
-    for (int w = 1; w < DECODE_WARPS; ++w) mx = fmaxf(mx, sm_m[w][h]);
+    for (int w = 0; w < DECODE_WARPS; ++w) {
+      const float* wo = reinterpret_cast<const float*>(smem + w * NSLOT * TT::SLOT_BYTES);
+      mw[w] = wo[8 * OSTR + h];
+      mx = fmaxf(mx, mw[w]);
+    }
     float acc = 0.f, l = 0.f;
 #pragma unroll
     for (int w = 0; w < DECODE_WARPS; ++w) {
-      const float mw = sm_m[w][h];
-      const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mx);
-      acc += sm_o[w][h][ch] * sc;
-      l += sm_l[w][h] * sc;
+      const float* wo = reinterpret_cast<const float*>(smem + w * NSLOT * TT::SLOT_BYTES);
+      const float sc = (mw[w] == -INFINITY) ? 0.f : ex2(mw[w] - mx);
+      float ov = wo[h * OSTR + ch];
+      if (PACK) ov += wo[(h + 4) * OSTR + ch];  // residual columns
+      acc += ov * sc;
+      l += wo[8 * OSTR + 8 + h] * sc;
     }
     const size_t ph = ((size_t)u * p.Hq + (size_t)hk * p.G + h) * MAX_SPLITS + s;
     p.o_part[ph * D + ch] = acc;
@@ -335,29 +505,41 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32) decode_attn_kernel(const De
   }
 }
 
-template <class T, int D, int BITS, int GROUP, int TILES>
+template <class T, int D, int BITS, int GROUP, int TILES, bool PACK>
 cudaError_t launch_decode_attn(const DecodeParams& p, int n_units, cudaStream_t stream) {
+  using TT = DecodeTraits<T, D, BITS, GROUP, TILES>;
+  static bool prepared = false;
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TT::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
   dim3 grid(p.S, p.Hkv, n_units);
-  decode_attn_kernel<T, D, BITS, GROUP, TILES><<<grid, DECODE_WARPS * 32, 0, stream>>>(p);
+  decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK><<<grid, DECODE_WARPS * 32, TT::SMEM_BYTES, stream>>>(p);
   return cudaGetLastError();
 }
 
 // explicit dispatch table entry points, one per (dtype, D) translation unit
 typedef cudaError_t (*decode_launch_fn)(const DecodeParams&, int, cudaStream_t);
-decode_launch_fn decode_dispatch_h64(int bits, int group, int tiles);
-decode_launch_fn decode_dispatch_h128(int bits, int group, int tiles);
-decode_launch_fn decode_dispatch_b64(int bits, int group, int tiles);
-decode_launch_fn decode_dispatch_b128(int bits, int group, int tiles);
+decode_launch_fn decode_dispatch_h64(int bits, int group, int tiles, int heads_per_kv);
+decode_launch_fn decode_dispatch_h128(int bits, int group, int tiles, int heads_per_kv);
+decode_launch_fn decode_dispatch_b64(int bits, int group, int tiles, int heads_per_kv);
+decode_launch_fn decode_dispatch_b128(int bits, int group, int tiles, int heads_per_kv);
 
-#define QEVICT_DECODE_DISPATCH(NAME, T, D)                                            \
-  decode_launch_fn NAME(int bits, int group, int tiles) {                             \
-    if (bits == 4 && group == 32 && tiles == 1) return launch_decode_attn<T, D, 4, 32, 1>; \
-    if (bits == 2 && group == 32 && tiles == 1) return launch_decode_attn<T, D, 2, 32, 1>; \
-    if (bits == 4 && group == 32 && tiles == 2) return launch_decode_attn<T, D, 4, 32, 2>; \
-    if (bits == 2 && group == 32 && tiles == 2) return launch_decode_attn<T, D, 2, 32, 2>; \
-    if (bits == 4 && group == 64 && tiles == 2) return launch_decode_attn<T, D, 4, 64, 2>; \
-    if (bits == 2 && group == 64 && tiles == 2) return launch_decode_attn<T, D, 2, 64, 2>; \
-    return nullptr;                                                                   \
+#define QEVICT_DECODE_CASE(T, D, B, G, TL)    \
+  if (bits == B && group == G && tiles == TL) \
+    return heads_per_kv <= 4 ? launch_decode_attn<T, D, B, G, TL, true> : launch_decode_attn<T, D, B, G, TL, false>;
+
+#define QEVICT_DECODE_DISPATCH(NAME, T, D)                                  \
+  decode_launch_fn NAME(int bits, int group, int tiles, int heads_per_kv) { \
+    QEVICT_DECODE_CASE(T, D, 4, 32, 1)                                      \
+    QEVICT_DECODE_CASE(T, D, 2, 32, 1)                                      \
+    QEVICT_DECODE_CASE(T, D, 4, 32, 2)                                      \
+    QEVICT_DECODE_CASE(T, D, 2, 32, 2)                                      \
+    QEVICT_DECODE_CASE(T, D, 4, 64, 2)                                      \
+    QEVICT_DECODE_CASE(T, D, 2, 64, 2)                                      \
+    return nullptr;                                                         \
   }
 
 }  // namespace qevict
