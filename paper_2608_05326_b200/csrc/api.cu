@@ -417,7 +417,7 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   QE_CUDA(h, launch_prefill_init(a, n_prompt, window_scores, s));
   QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
   QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kf, s));
-  QE_CUDA(h, launch_quantize(a, k, v, ctx_tokens, g.Kq, s));
+  QE_CUDA(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));
   h->launches += 2 + (g.Kf > 0) + (g.Kq > 0);
   for (int l = l0; l < l1; ++l) {
     h->layers[l].prefilled = true;
@@ -468,11 +468,11 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   cudaStream_t s = (cudaStream_t)stream;
   const KernelArgs a = make_args(h, l0, l1);
   QE_CUDA(h, launch_route(a, 0, next_pow2(g.Kf + g.Kq + g.aged_cap + 1), s));
-  // quantizations read full-precision pages that promotions may overwrite: quantize first
-  QE_CUDA(h, launch_quantize(a, nullptr, nullptr, 0, g.Kq > 0 ? g.PF : 0, s));
+  // quantizations and promotions of the event in one launch (linked where they share a page)
   const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
-  QE_CUDA(h, launch_promote(a, max_promote, s));
-  h->launches += 1 + (g.Kq > 0) + (max_promote > 0);
+  const int max_items = (g.Kq > 0 ? g.PF : 0) + max_promote;
+  QE_CUDA(h, launch_migrate(a, nullptr, nullptr, 0, max_items, s));
+  h->launches += 1 + (max_items > 0);
   for (int l = l0; l < l1; ++l) h->layers[l].aged = 0;
   return QEVICT_OK;
 }

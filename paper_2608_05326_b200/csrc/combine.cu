@@ -55,9 +55,18 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   const float2* wrec = a.st.wrec + (size_t)u * g.Hq * g.EMAX;
   for (int e = e0 + tid; e < e1; e += COMBINE_THREADS) {
     float acc = 0.f;
-    for (int h = 0; h < g.Hq; ++h) {
-      const float2 r = wrec[(size_t)h * g.EMAX + e];
-      acc += r.x * exp2f(r.y - s_m[h]) * s_invl[h];
+    // heads in ascending order (fixed summation order); records are fetched eight at a time so that the
+    // loads overlap
+    for (int h0 = 0; h0 < g.Hq; h0 += 8) {
+      float2 r[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        r[k] = (h0 + k < g.Hq) ? wrec[(size_t)(h0 + k) * g.EMAX + e] : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (h0 + k < g.Hq) acc += r[k].x * exp2f(r[k].y - s_m[h0 + k]) * s_invl[h0 + k];
+      }
     }
     const uint32_t w = a.st.entries[(size_t)u * g.EMAX + e].x & ENTRY_WINDOW_MASK;
     a.st.importance[(size_t)u * g.NW + w] += acc;

@@ -23,11 +23,11 @@ cudaError_t launch_combine(const KernelArgs& a, int n_splits, void* out, cudaStr
 cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt_windows, const float* scores, cudaStream_t s);
 // A3 + A4 + A7: rank, assign tiers, release / allocate pages, build migration lists and the work list.
 cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_capacity, cudaStream_t s);
-// A5: quantize the windows of the quantization list (source: their full-precision page, or the prompt).
-cudaError_t launch_quantize(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx,
-                            int max_items, cudaStream_t s);
-// A6: dequantize the windows of the promotion list into their new full-precision page.
-cudaError_t launch_promote(const KernelArgs& a, int max_items, cudaStream_t s);
+// A5 + A6: quantize the windows of the quantization list (source: their full-precision page, or the
+// prompt) and dequantize the windows of the promotion list into their new full-precision page; a
+// promotion that takes over the page a quantization reads runs after it in the same CTA.
+cudaError_t launch_migrate(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
+                           cudaStream_t s);
 // P0 (second half): copy the prompt windows of the copy list into their full-precision page.
 cudaError_t launch_copy_prompt(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx,
                                int max_items, cudaStream_t s);

@@ -14,6 +14,7 @@ namespace qevict {
 namespace {
 
 constexpr int PAGE_THREADS = 128;
+constexpr int MIGRATE_THREADS = 256;
 
 template <class T>
 __device__ __forceinline__ void group_params(float mn, float mx, int qmax, T& s_out, T& z_out, float& s_f, bool& bad) {
@@ -34,167 +35,202 @@ __device__ __forceinline__ uint32_t quant_code(float x, float z, float s, int qm
   return (uint32_t)c;
 }
 
-// One CTA per (list item, KV head).  Shared memory: K and V of the window in plain [W][D] order,
-// the packed code words, and the parameters as floats.
+// ---- quantize one half (keys or values) of one window of one KV head ------------------------------------
+// Shared memory: the half in plain [W][D] order and its parameters as floats.  Every thread then builds
+// whole 32-bit code words (no atomics) and stores them straight into the page.
 template <class T>
-__global__ void __launch_bounds__(PAGE_THREADS) quantize_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
-                                                                const T* __restrict__ v_prompt, int ctx) {
-  const Geometry& g = a.geo;
-  const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y, item = blockIdx.x, tid = threadIdx.x;
-  if (item >= a.st.n_quant[u]) return;
-  const int4 it = a.st.quant_list[(size_t)u * (g.PF + g.Kq) + item];
-  const int w = it.x, src = it.y, dst = it.z;
-  const int W = g.W, D = g.D, G = g.group, qmax = (1 << g.bits) - 1;
+__device__ void quantize_part(const Geometry& g, int part, const T* __restrict__ rows /* prompt rows or null */,
+                              const char* __restrict__ fp_head /* source page head or null */, char* qb,
+                              unsigned char* smem_raw) {
+  const int tid = threadIdx.x, W = g.W, D = g.D, G = g.group, qmax = (1 << g.bits) - 1;
+  T* sx = reinterpret_cast<T*>(smem_raw);                       // [W][D]
+  float* sf = reinterpret_cast<float*>(sx + W * D);             // scale (or -1 if the group is degenerate)
+  float* zf = sf + (part == 0 ? (W / G) * D : W * (D / G));     // zero
+  const int KG = D / 32;
 
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* sk = reinterpret_cast<T*>(smem_raw);                   // [W][D]
-  T* sv = sk + W * D;                                       // [W][D]
-  uint32_t* kw = reinterpret_cast<uint32_t*>(sv + W * D);   // [tiles][kc words]
-  const int words_per_tile = g.q_kc_bytes / 4;
-  uint32_t* vw = kw + g.tiles * words_per_tile;             // [tiles][vc words]
-  float* ksf = reinterpret_cast<float*>(vw + g.tiles * words_per_tile);  // [W/G][D] scale (or -1 if bad)
-  float* kzf = ksf + (W / G) * D;
-  float* vsf = kzf + (W / G) * D;                           // [W][D/G]
-  float* vzf = vsf + W * (D / G);
-
-  // ---- stage the window in plain order -----------------------------------------------------------
-  if (src < 0) {
-    const T* kr = k_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * W) * D;
-    const T* vr = v_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * W) * D;
-    const uint4* k4 = reinterpret_cast<const uint4*>(kr);
-    const uint4* v4 = reinterpret_cast<const uint4*>(vr);
-    for (int i = tid; i < W * D / 8; i += PAGE_THREADS) {
-      reinterpret_cast<uint4*>(sk)[i] = k4[i];
-      reinterpret_cast<uint4*>(sv)[i] = v4[i];
-    }
+  // ---- stage the half in plain order ---------------------------------------------------------------
+  if (rows) {
+    const uint4* r4 = reinterpret_cast<const uint4*>(rows);
+    for (int i = tid; i < W * D / 8; i += MIGRATE_THREADS) reinterpret_cast<uint4*>(sx)[i] = r4[i];
   } else {
-    const char* hb = a.st.fp_pool + ((size_t)u * g.PF + src) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
+    // the page is fragment-major: 16-byte loads (many in flight), each vector scattered to plain positions
+    const int nvec = 32 * D / 8;
     for (int tile = 0; tile < g.tiles; ++tile) {
-      const T* kt = reinterpret_cast<const T*>(hb + (size_t)tile * 2 * g.fp_tile_bytes);
-      const T* vt = reinterpret_cast<const T*>(hb + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes);
-      for (int i = tid; i < 32 * D; i += PAGE_THREADS) {
-        const int tk = i / D, ch = i - tk * D;
-        sk[(tile * 32 + tk) * D + ch] = kt[fpk_off(tk, ch, D)];
-        sv[(tile * 32 + tk) * D + ch] = vt[fpv_off(tk, ch)];
+      const uint4* src = reinterpret_cast<const uint4*>(fp_head + (size_t)tile * 2 * g.fp_tile_bytes + (part ? g.fp_tile_bytes : 0));
+#pragma unroll 4
+      for (int v = tid; v < nvec; v += MIGRATE_THREADS) {
+        const uint4 x = src[v];
+        const int ln = v & 31, vec = v >> 5, gg = ln >> 2, tt = ln & 3;
+        const T* xe = reinterpret_cast<const T*>(&x);
+#pragma unroll
+        for (int el = 0; el < 8; ++el) {
+          const int a1 = el >> 2, a2 = (el >> 1) & 1, e = el & 1;
+          int tk, ch;
+          if (part == 0) { const int kj = vec / KG, kc = vec - kj * KG; tk = 8 * kj + gg; ch = 32 * kc + 16 * a1 + 8 * a2 + 2 * tt + e; }
+          else { const int vi = vec >> 1, vks = vec & 1; tk = 16 * vks + 8 * a1 + 2 * tt + e; ch = 16 * vi + 8 * a2 + gg; }
+          sx[(tile * 32 + tk) * D + ch] = xe[el];
+        }
       }
     }
   }
-  for (int i = tid; i < 2 * g.tiles * words_per_tile; i += PAGE_THREADS) kw[i] = 0u;
   __syncthreads();
 
-  char* qb = a.st.q_pool + ((size_t)u * g.PQ + dst) * g.q_page_bytes + (size_t)hk * g.q_head_bytes;
-
-  // ---- parameters --------------------------------------------------------------------------------
-  for (int i = tid; i < (W / G) * D; i += PAGE_THREADS) {  // keys: (token block, channel)
-    const int blk = i / D, ch = i - blk * D;
-    float mn = INFINITY, mx = -INFINITY;
-    for (int tk = blk * G; tk < (blk + 1) * G; ++tk) {
-      const float x = Tr<T>::to_float(sk[tk * D + ch]);
-      mn = fminf(mn, x); mx = fmaxf(mx, x);
+  // ---- parameters ----------------------------------------------------------------------------------
+  if (part == 0) {  // keys: one group per (block of G tokens, channel)
+    for (int i = tid; i < (W / G) * D; i += MIGRATE_THREADS) {
+      const int blk = i / D, ch = i - blk * D;
+      float mn = INFINITY, mx = -INFINITY;
+      for (int tk = blk * G; tk < (blk + 1) * G; ++tk) {
+        const float x = Tr<T>::to_float(sx[tk * D + ch]);
+        mn = fminf(mn, x); mx = fmaxf(mx, x);
+      }
+      T st, zt; float s; bool bad;
+      group_params<T>(mn, mx, qmax, st, zt, s, bad);
+      sf[i] = bad ? -1.f : s;
+      zf[i] = mn;
+      T* kp = reinterpret_cast<T*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes);
+      kp[kparam_off(ch, 0)] = st;
+      kp[kparam_off(ch, 1)] = zt;
     }
-    T st, zt; float sf; bool bad;
-    group_params<T>(mn, mx, qmax, st, zt, sf, bad);
-    ksf[i] = bad ? -1.f : sf;
-    kzf[i] = mn;
-    T* kp = reinterpret_cast<T*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes);
-    kp[kparam_off(ch, 0)] = st;
-    kp[kparam_off(ch, 1)] = zt;
-  }
-  for (int i = tid; i < W * (D / G); i += PAGE_THREADS) {  // values: (token, channel block)
-    const int tk = i / (D / G), gc = i - tk * (D / G);
-    float mn = INFINITY, mx = -INFINITY;
-    for (int ch = gc * G; ch < (gc + 1) * G; ++ch) {
-      const float x = Tr<T>::to_float(sv[tk * D + ch]);
-      mn = fminf(mn, x); mx = fmaxf(mx, x);
-    }
-    T st, zt; float sf; bool bad;
-    group_params<T>(mn, mx, qmax, st, zt, sf, bad);
-    vsf[i] = bad ? -1.f : sf;
-    vzf[i] = mn;
-    const int tile = tk >> 5;
-    T* vp = reinterpret_cast<T*>(qb + (size_t)tile * g.q_tile_stride + g.q_kc_bytes + g.q_vc_bytes);
-    vp[vparam_off(tk & 31, gc, 0)] = st;
-    vp[vparam_off(tk & 31, gc, 1)] = zt;
-  }
-  __syncthreads();
-
-  // ---- codes -------------------------------------------------------------------------------------
-  for (int i = tid; i < W * D; i += PAGE_THREADS) {
-    const int tk = i / D, ch = i - tk * D;
-    const int tile = tk >> 5, tkk = tk & 31;
-    {
-      const int pi = (tk / G) * D + ch;
-      const float s = ksf[pi];
-      const uint32_t c = quant_code(Tr<T>::to_float(sk[i]), kzf[pi], s, qmax, s < 0.f);
-      const CodePos p = kcode_pos(tkk, ch, D, g.bits);
-      atomicOr(&kw[tile * words_per_tile + p.word], c << p.shift);
-    }
-    {
-      const int pi = tk * (D / G) + ch / G;
-      const float s = vsf[pi];
-      const uint32_t c = quant_code(Tr<T>::to_float(sv[i]), vzf[pi], s, qmax, s < 0.f);
-      const CodePos p = vcode_pos(tkk, ch, g.bits);
-      atomicOr(&vw[tile * words_per_tile + p.word], c << p.shift);
+  } else {  // values: one group per (token, block of G channels)
+    const int ng = D / G;
+    for (int i = tid; i < W * ng; i += MIGRATE_THREADS) {
+      const int gc = i / W, tk = i - gc * W;  // consecutive threads take consecutive tokens
+      float mn = INFINITY, mx = -INFINITY;
+      for (int k = 0; k < G; ++k) {
+        const int ch = gc * G + ((k + tk) & (G - 1));  // rotated start: spreads the threads over the banks
+        const float x = Tr<T>::to_float(sx[tk * D + ch]);
+        mn = fminf(mn, x); mx = fmaxf(mx, x);
+      }
+      T st, zt; float s; bool bad;
+      group_params<T>(mn, mx, qmax, st, zt, s, bad);
+      sf[tk * ng + gc] = bad ? -1.f : s;
+      zf[tk * ng + gc] = mn;
+      T* vp = reinterpret_cast<T*>(qb + (size_t)(tk >> 5) * g.q_tile_stride + g.q_kc_bytes + g.q_vc_bytes);
+      vp[vparam_off(tk & 31, gc, 0)] = st;
+      vp[vparam_off(tk & 31, gc, 1)] = zt;
     }
   }
   __syncthreads();
+
+  // ---- codes: one 32-bit word (8 or 16 codes) per thread and iteration ----------------------------------
+  const int words_per_tile = g.q_kc_bytes / 4;
+  const int cpw = 32 / g.bits;  // codes per word
   for (int tile = 0; tile < g.tiles; ++tile) {
-    uint4* kc = reinterpret_cast<uint4*>(qb + (size_t)tile * g.q_tile_stride);
-    uint4* vc = reinterpret_cast<uint4*>(qb + (size_t)tile * g.q_tile_stride + g.q_kc_bytes);
-    for (int i = tid; i < words_per_tile / 4; i += PAGE_THREADS) {
-      kc[i] = reinterpret_cast<const uint4*>(kw + tile * words_per_tile)[i];
-      vc[i] = reinterpret_cast<const uint4*>(vw + tile * words_per_tile)[i];
+    uint32_t* dstw = reinterpret_cast<uint32_t*>(qb + (size_t)tile * g.q_tile_stride + (part ? g.q_kc_bytes : 0));
+    for (int wo = tid; wo < words_per_tile; wo += MIGRATE_THREADS) {
+      // word offset -> (word index of the lane, lane)
+      const int q4 = wo >> 2, ln = q4 & 31, widx = (q4 >> 5) * 4 + (wo & 3), gg = ln >> 2, tt = ln & 3;
+      uint32_t word = 0u;
+      for (int k = 0; k < cpw; ++k) {
+        // slot k of the word: sub-word (2-bit only), register m / a, element e
+        const int e = k & 1, m = (k >> 1) & 3, sub = k >> 3;
+        int tk, ch;
+        if (part == 0) {
+          const int per_j = g.bits == 4 ? KG : KG / 2;
+          const int j = widx / per_j, c = (widx - j * per_j) * (g.bits == 4 ? 1 : 2) + sub;
+          tk = 8 * j + gg;
+          ch = 32 * c + 16 * (m >> 1) + 8 * (m & 1) + 2 * tt + e;
+        } else {
+          const int i = g.bits == 4 ? (widx >> 1) : widx;
+          const int ks = g.bits == 4 ? (widx & 1) : sub;
+          tk = 16 * ks + 8 * (m >> 1) + 2 * tt + e;
+          ch = 16 * i + 8 * (m & 1) + gg;
+        }
+        const int row = tile * 32 + tk;
+        const int pi = part == 0 ? (row / G) * D + ch : row * (D / G) + ch / G;
+        const float s = sf[pi];
+        const uint32_t code = quant_code(Tr<T>::to_float(sx[row * D + ch]), zf[pi], s, qmax, s < 0.f);
+        word |= code << (g.bits * (sub * 4 + m) + 16 * e);
+      }
+      dstw[wo] = word;
     }
   }
 }
 
-// One CTA per (list item, KV head): rebuild the window from its codes into a full-precision page,
-// producing exactly the operand registers the decode kernel forms in flight.
+// ---- dequantize one half of one window of one KV head into a full-precision page -----------------------
+// Produces exactly the operand registers the decode kernel forms in flight.
 template <class T>
-__global__ void __launch_bounds__(PAGE_THREADS) promote_kernel(const KernelArgs a) {
-  const Geometry& g = a.geo;
-  const int u = a.unit0 + blockIdx.z, hk = blockIdx.y, item = blockIdx.x;
-  if (item >= a.st.n_promote[u]) return;
-  const int4 it = a.st.promote_list[(size_t)u * g.Kf + item];
-  const int srcq = it.y, dst = it.z;
+__device__ void promote_part(const Geometry& g, int part, const char* __restrict__ qb, char* fb) {
   const int D = g.D, KG = D / 32, MT = D / 16, bits = g.bits;
   const uint32_t mask = bits == 4 ? 0x000F000Fu : 0x00030003u, MG = Tr<T>::MAGIC;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, t = lane & 3, nwarps = PAGE_THREADS / 32;
-  const char* qb = a.st.q_pool + ((size_t)u * g.PQ + srcq) * g.q_page_bytes + (size_t)hk * g.q_head_bytes;
-  char* fb = a.st.fp_pool + ((size_t)u * g.PF + dst) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, t = lane & 3, nwarps = MIGRATE_THREADS / 32;
   for (int tile = 0; tile < g.tiles; ++tile) {
-    const uint32_t* kc = reinterpret_cast<const uint32_t*>(qb + (size_t)tile * g.q_tile_stride);
-    const uint32_t* vc = reinterpret_cast<const uint32_t*>(qb + (size_t)tile * g.q_tile_stride + g.q_kc_bytes);
-    const uint4* vp = reinterpret_cast<const uint4*>(qb + (size_t)tile * g.q_tile_stride + g.q_kc_bytes + g.q_vc_bytes);
-    const uint4* kp = reinterpret_cast<const uint4*>(qb + g.q_kp_off + (size_t)((tile * 32) / g.group) * g.q_kp_bytes);
-    uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
-    uint4* vt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes);
-    for (int v = wid; v < 4 * KG; v += nwarps) {  // key vectors (j, c)
-      const int j = v / KG, c = v - j * KG;
-      const int widx = bits == 4 ? j * KG + c : j * (KG / 2) + (c >> 1);
-      const int sh = bits == 4 ? 0 : (c & 1) * 8;
-      const uint32_t w = kc[code_word_off(widx, lane)];
-      const uint4 p0 = kp[(c * 2 + 0) * 4 + t], p1 = kp[(c * 2 + 1) * 4 + t];
-      uint4 r;
-      r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, p0.x, p0.y);
-      r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, p0.z, p0.w);
-      r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, p1.x, p1.y);
-      r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, p1.z, p1.w);
-      kt[v * 32 + lane] = r;
+    const char* tb = qb + (size_t)tile * g.q_tile_stride;
+    if (part == 0) {
+      const uint32_t* kc = reinterpret_cast<const uint32_t*>(tb);
+      const uint4* kp = reinterpret_cast<const uint4*>(qb + g.q_kp_off + (size_t)((tile * 32) / g.group) * g.q_kp_bytes);
+      uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
+      for (int v = wid; v < 4 * KG; v += nwarps) {  // key vectors (j, c)
+        const int j = v / KG, c = v - j * KG;
+        const int widx = bits == 4 ? j * KG + c : j * (KG / 2) + (c >> 1);
+        const int sh = bits == 4 ? 0 : (c & 1) * 8;
+        const uint32_t w = kc[code_word_off(widx, lane)];
+        const uint4 p0 = kp[(c * 2 + 0) * 4 + t], p1 = kp[(c * 2 + 1) * 4 + t];
+        uint4 r;
+        r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, p0.x, p0.y);
+        r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, p0.z, p0.w);
+        r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, p1.x, p1.y);
+        r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, p1.z, p1.w);
+        kt[v * 32 + lane] = r;
+      }
+    } else {
+      const uint32_t* vc = reinterpret_cast<const uint32_t*>(tb + g.q_kc_bytes);
+      const uint4* vp = reinterpret_cast<const uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes);
+      uint4* vt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes);
+      for (int v = wid; v < 2 * MT; v += nwarps) {  // value vectors (i, ks)
+        const int i = v >> 1, ks = v & 1;
+        const int widx = bits == 4 ? i * 2 + ks : i;
+        const int sh = bits == 4 ? 0 : ks * 8;
+        const uint32_t w = vc[code_word_off(widx, lane)];
+        const int gc = (16 * i) / g.group;
+        const uint4 pr = vp[(gc * 2 + ks) * 4 + t];
+        uint4 r;
+        r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, pr.x, pr.y);
+        r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, pr.x, pr.y);
+        r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, pr.z, pr.w);
+        r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, pr.z, pr.w);
+        vt[v * 32 + lane] = r;
+      }
     }
-    for (int v = wid; v < 2 * MT; v += nwarps) {  // value vectors (i, ks)
-      const int i = v >> 1, ks = v & 1;
-      const int widx = bits == 4 ? i * 2 + ks : i;
-      const int sh = bits == 4 ? 0 : ks * 8;
-      const uint32_t w = vc[code_word_off(widx, lane)];
-      const int gc = (16 * i) / g.group;
-      const uint4 pr = vp[(gc * 2 + ks) * 4 + t];
-      uint4 r;
-      r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, pr.x, pr.y);
-      r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, pr.x, pr.y);
-      r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, pr.z, pr.w);
-      r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, pr.z, pr.w);
-      vt[v * 32 + lane] = r;
+  }
+}
+
+// Migration kernel.  CTA = (list slot, KV head x {keys, values}, unit); it walks the unit's quantization
+// list and then the promotions nobody else handles.  A promotion whose new full-precision page is the
+// page a quantization of the same event reads from is linked to that quantization and runs in the same
+// CTA right after it, so no page is overwritten before it has been read.
+template <class T>
+__global__ void __launch_bounds__(MIGRATE_THREADS) migrate_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
+                                                                  const T* __restrict__ v_prompt, int ctx) {
+  const Geometry& g = a.geo;
+  const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y >> 1, part = blockIdx.y & 1;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int n_quant = a.st.n_quant[u], n_promote = a.st.n_promote[u];
+  const int4* quant_list = a.st.quant_list + (size_t)u * (g.PF + g.Kq);
+  const int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
+  auto promote = [&](int k) {
+    const int4 it = promote_list[k];
+    promote_part<T>(g, part, a.st.q_pool + ((size_t)u * g.PQ + it.y) * g.q_page_bytes + (size_t)hk * g.q_head_bytes,
+                    a.st.fp_pool + ((size_t)u * g.PF + it.z) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes);
+  };
+  for (int item = blockIdx.x; item < n_quant + n_promote; item += gridDim.x) {
+    if (item < n_quant) {
+      const int4 it = quant_list[item];  // {window, source page (-1: prompt), destination page, linked promotion}
+      const T* rows = nullptr;
+      const char* fp_head = nullptr;
+      if (it.y < 0) rows = (part ? v_prompt : k_prompt) + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)it.x * g.W) * g.D;
+      else fp_head = a.st.fp_pool + ((size_t)u * g.PF + it.y) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
+      __syncthreads();  // the staging buffer is reused from item to item
+      quantize_part<T>(g, part, rows, fp_head,
+                       a.st.q_pool + ((size_t)u * g.PQ + it.z) * g.q_page_bytes + (size_t)hk * g.q_head_bytes, smem_raw);
+      if (it.w >= 0) {
+        __syncthreads();  // every thread has finished reading the source page
+        promote(it.w);
+      }
+    } else {
+      const int k = item - n_quant;
+      if (promote_list[k].w == 0) promote(k);  // not linked to a quantization
     }
   }
 }
@@ -204,8 +240,9 @@ template <class T>
 __global__ void __launch_bounds__(PAGE_THREADS) copy_prompt_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
                                                                    const T* __restrict__ v_prompt, int ctx) {
   const Geometry& g = a.geo;
-  const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y, item = blockIdx.x;
-  if (item >= a.st.n_copy[u]) return;
+  const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y;
+  const int n_items = a.st.n_copy[u];
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
   const int4 it = a.st.copy_list[(size_t)u * g.Kf + item];
   const int w = it.x, dst = it.y, D = g.D;
   const T* kr = k_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * g.W) * D;
@@ -219,6 +256,7 @@ __global__ void __launch_bounds__(PAGE_THREADS) copy_prompt_kernel(const KernelA
       kt[fpk_off(tk, ch, D)] = kr[(size_t)(tile * 32 + tk) * D + ch];
       vt[fpv_off(tk, ch)] = vr[(size_t)(tile * 32 + tk) * D + ch];
     }
+  }
   }
 }
 
@@ -266,40 +304,41 @@ __global__ void export_q_page_kernel(const KernelArgs a, int u, int page, uint8_
   }
 }
 
-size_t quantize_smem_bytes(const Geometry& g) {
-  return (size_t)2 * g.W * g.D * 2 + (size_t)2 * g.tiles * g.q_kc_bytes +
-         (size_t)(2 * (g.W / g.group) * g.D + 2 * g.W * (g.D / g.group)) * 4;
+size_t migrate_smem_bytes(const Geometry& g) {
+  const size_t params = (size_t)((g.W / g.group) * g.D > g.W * (g.D / g.group) ? (g.W / g.group) * g.D : g.W * (g.D / g.group));
+  return (size_t)g.W * g.D * 2 + 2 * params * 4;
 }
 
 }  // namespace
 
+// CTAs per (unit, KV head) that walk a migration list: as many as there can be items, but no more
+// than keeps the whole launch near two thousand CTAs (lists are mostly short or empty at decode time).
+static int items_grid(int max_items, const KernelArgs& a) {
+  const int pairs = a.geo.Hkv * 2 * a.n_units;
+  int per = 2048 / (pairs > 0 ? pairs : 1);
+  if (per < 1) per = 1;
+  return max_items < per ? max_items : per;
+}
+
 #define QE_BY_DTYPE(geo, CALL_H, CALL_B) \
   do { if ((geo).dtype == QEVICT_DTYPE_FP16) { CALL_H; } else { CALL_B; } } while (0)
 
-cudaError_t launch_quantize(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
-                            cudaStream_t s) {
+cudaError_t launch_migrate(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
+                           cudaStream_t s) {
   if (max_items <= 0) return cudaSuccess;
-  dim3 grid(max_items, a.geo.Hkv, a.n_units);
-  const size_t sm = quantize_smem_bytes(a.geo);
+  dim3 grid(items_grid(max_items, a), a.geo.Hkv * 2, a.n_units);
+  const size_t sm = migrate_smem_bytes(a.geo);
   QE_BY_DTYPE(a.geo,
-              (quantize_kernel<__half><<<grid, PAGE_THREADS, sm, s>>>(a, (const __half*)k_prompt, (const __half*)v_prompt, ctx)),
-              (quantize_kernel<__nv_bfloat16><<<grid, PAGE_THREADS, sm, s>>>(a, (const __nv_bfloat16*)k_prompt,
-                                                                          (const __nv_bfloat16*)v_prompt, ctx)));
-  return cudaGetLastError();
-}
-
-cudaError_t launch_promote(const KernelArgs& a, int max_items, cudaStream_t s) {
-  if (max_items <= 0) return cudaSuccess;
-  dim3 grid(max_items, a.geo.Hkv, a.n_units);
-  QE_BY_DTYPE(a.geo, (promote_kernel<__half><<<grid, PAGE_THREADS, 0, s>>>(a)),
-              (promote_kernel<__nv_bfloat16><<<grid, PAGE_THREADS, 0, s>>>(a)));
+              (migrate_kernel<__half><<<grid, MIGRATE_THREADS, sm, s>>>(a, (const __half*)k_prompt, (const __half*)v_prompt, ctx)),
+              (migrate_kernel<__nv_bfloat16><<<grid, MIGRATE_THREADS, sm, s>>>(a, (const __nv_bfloat16*)k_prompt,
+                                                                         (const __nv_bfloat16*)v_prompt, ctx)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_copy_prompt(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
                                cudaStream_t s) {
   if (max_items <= 0) return cudaSuccess;
-  dim3 grid(max_items, a.geo.Hkv, a.n_units);
+  dim3 grid(items_grid(max_items, a), a.geo.Hkv, a.n_units);
   QE_BY_DTYPE(a.geo,
               (copy_prompt_kernel<__half><<<grid, PAGE_THREADS, 0, s>>>(a, (const __half*)k_prompt, (const __half*)v_prompt, ctx)),
               (copy_prompt_kernel<__nv_bfloat16><<<grid, PAGE_THREADS, 0, s>>>(a, (const __nv_bfloat16*)k_prompt,

@@ -17,16 +17,10 @@ __device__ __forceinline__ uint32_t mono_bits(float f) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Stable, deterministic block-wide stream compaction: calls emit(i, rank) for every i in [0, n)
-// with pred(i), rank = number of smaller i with pred.  Returns the total.  pred must be pure until
-// emit(i) has run.  scratch: 33 ints of shared memory.
-template <class Pred, class Emit>
-__device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
+// Block-wide exclusive prefix sum of one int per thread; *total receives the sum.  scratch: 33 ints of
+// shared memory.  Ends with a barrier, so scratch may be reused right away.
+__device__ __forceinline__ int block_exclusive_scan(int cnt, int* scratch, int* total) {
   const int tid = threadIdx.x, nt = blockDim.x;
-  const int chunk = (n + nt - 1) / nt;
-  const int b = min(n, tid * chunk), e = min(n, b + chunk);
-  int cnt = 0;
-  for (int i = b; i < e; ++i) cnt += pred(i) ? 1 : 0;
   const int lane = tid & 31, wid = tid >> 5;
   int inc = cnt;
 #pragma unroll
@@ -48,8 +42,24 @@ __device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
     if (lane == 31) scratch[32] = iv;
   }
   __syncthreads();
-  int rank = scratch[wid] + inc - cnt;
-  const int total = scratch[32];
+  const int rank = scratch[wid] + inc - cnt;
+  *total = scratch[32];
+  __syncthreads();
+  return rank;
+}
+
+// Stable, deterministic block-wide stream compaction: calls emit(i, rank) for every i in [0, n)
+// with pred(i), rank = number of smaller i with pred.  Returns the total.  pred must be pure until
+// emit(i) has run.  scratch: 33 ints of shared memory.
+template <class Pred, class Emit>
+__device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int chunk = (n + nt - 1) / nt;
+  const int b = min(n, tid * chunk), e = min(n, b + chunk);
+  int cnt = 0;
+  for (int i = b; i < e; ++i) cnt += pred(i) ? 1 : 0;
+  int total;
+  int rank = block_exclusive_scan(cnt, scratch, &total);
   for (int i = b; i < e; ++i) {
     if (pred(i)) emit(i, rank++);
   }
@@ -153,15 +163,30 @@ __global__ void prefill_init_kernel(const KernelArgs a, int n_prompt, const floa
 }
 
 // ------------------------------------------------------------------------------------------- route
+// One CTA per unit.  The candidates (Full, Quantized and aged windows) are gathered in ascending window
+// order into shared memory together with the two page-owner tables; ranking, tier assignment, page
+// release and allocation, migration lists and the decode work list all run on those shared copies, and
+// the tables go back to global memory once at the end.  Global memory is waited on three times.
+__device__ __forceinline__ bool is_candidate(uint8_t t) {
+  return t == QEVICT_TIER_FULL || t == QEVICT_TIER_QUANT || t == QEVICT_TIER_AGED;
+}
+
 __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a, int prefill, int sort_cap) {
   const Geometry& g = a.geo;
   const int u = a.unit0 + blockIdx.x, tid = threadIdx.x;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
-  int32_t* free_fp = reinterpret_cast<int32_t*>(keys + sort_cap);            // [PF]
+  int32_t* cw = reinterpret_cast<int32_t*>(keys + sort_cap);                 // [sort_cap] window of candidate c
+  int32_t* cfp = cw + sort_cap;                                              // [sort_cap] its full-precision page
+  int32_t* cq = cfp + sort_cap;                                              // [sort_cap] its quantized page
+  int32_t* ofp = cq + sort_cap;                                              // [PF] owner of each page
+  int32_t* oq = ofp + g.PF;                                                  // [PQ]
+  int32_t* free_fp = oq + g.PQ;                                              // [PF] free page ids, ascending
   int32_t* free_q = free_fp + g.PF;                                          // [PQ]
   int32_t* scratch = free_q + g.PQ;                                          // [40]
-  uint8_t* newt = reinterpret_cast<uint8_t*>(scratch + 40);                  // [NW]
+  uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 40);                 // [sort_cap] state before
+  uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
+  uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
 
   uint8_t* tier = a.st.tier + (size_t)u * g.NW;
   uint8_t* ledger = a.st.ledger + (size_t)u * g.NW;
@@ -171,143 +196,191 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int32_t* fp_owner = a.st.fp_owner + (size_t)u * g.PF;
   int32_t* q_owner = a.st.q_owner + (size_t)u * g.PQ;
   const int nw = a.st.n_windows[u];
+  const int ow = a.st.open_window[u];
 
-  int* s_ncand = scratch + 33;
   int* s_react = scratch + 34;
   int* s_del = scratch + 35;
-  if (tid == 0) { *s_ncand = 0; *s_react = 0; *s_del = 0; }
-  for (int i = tid; i < sort_cap; i += ROUTE_THREADS) keys[i] = KEY_SENTINEL;
-  __syncthreads();
+  if (tid == 0) { *s_react = 0; *s_del = 0; }
+  for (int i = tid; i < g.PF; i += ROUTE_THREADS) ofp[i] = fp_owner[i];
+  for (int i = tid; i < g.PQ; i += ROUTE_THREADS) oq[i] = q_owner[i];
 
-  // candidates = Full, Quantized and aged windows; key orders by score (higher first), then index
-  for (int w = tid; w < nw; w += ROUTE_THREADS) {
-    const uint8_t t = tier[w];
-    newt[w] = t;
-    if (t == QEVICT_TIER_FULL || t == QEVICT_TIER_QUANT || t == QEVICT_TIER_AGED) {
-      const int pos = atomicAdd(s_ncand, 1);
-      if (pos < sort_cap) keys[pos] = ((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)w;
+  // ---- gather the candidates in ascending window order ----------------------------------------------
+  auto emit_candidate = [&](int w, int k, uint8_t t) {
+    if (k >= sort_cap) return;
+    cw[k] = w;
+    ctier[k] = t;
+    cled[k] = ledger[w];
+    cfp[k] = fp_page[w];
+    cq[k] = q_page[w];
+    keys[k] = ((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)k;
+  };
+  int n_all;
+  const int chunk = (nw + ROUTE_THREADS - 1) / ROUTE_THREADS;
+  if (chunk <= 16) {
+    // every thread reads its (up to 16) window states in one go and keeps them in registers
+    uint8_t tc[16];
+    const int b = tid * chunk;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) tc[k] = (k < chunk && b + k < nw) ? tier[b + k] : (uint8_t)QEVICT_TIER_NONE;
+    int cnt = 0;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) cnt += is_candidate(tc[k]) ? 1 : 0;
+    int rank = block_exclusive_scan(cnt, scratch, &n_all);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if (is_candidate(tc[k])) emit_candidate(b + k, rank++, tc[k]);
     }
+    __syncthreads();
+  } else {
+    n_all = block_compact(nw, scratch, [&](int w) { return is_candidate(tier[w]); },
+                          [&](int w, int k) { emit_candidate(w, k, tier[w]); });
   }
-  __syncthreads();
-  const int n_cand = min(*s_ncand, sort_cap);
-  int n_sort = 2;
-  while (n_sort < n_cand) n_sort <<= 1;
-  for (int k = 2; k <= n_sort; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n_sort; i += ROUTE_THREADS) {
-        const int ixj = i ^ j;
-        if (ixj > i) {
-          const unsigned long long x = keys[i], y = keys[ixj];
-          const bool asc = (i & k) == 0;
-          if ((x > y) == asc) { keys[i] = y; keys[ixj] = x; }
+  const int n_cand = min(n_all, sort_cap);
+
+  // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
+  // Quantized, remainder -> Evicted -----------------------------------------------------------------
+  if (n_cand <= 1024) {
+    // rank of a key = number of smaller keys (all keys are distinct)
+    for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+      const unsigned long long mine = keys[c];
+      int pos = 0;
+      for (int i = 0; i < n_cand; ++i) pos += keys[i] < mine ? 1 : 0;
+      cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+    }
+  } else {
+    int n_sort = 2;
+    while (n_sort < n_cand) n_sort <<= 1;
+    for (int i = n_cand + tid; i < n_sort; i += ROUTE_THREADS) keys[i] = KEY_SENTINEL;
+    __syncthreads();
+    for (int k = 2; k <= n_sort; k <<= 1) {
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int i = tid; i < n_sort; i += ROUTE_THREADS) {
+          const int ixj = i ^ j;
+          if (ixj > i) {
+            const unsigned long long x = keys[i], y = keys[ixj];
+            const bool asc = (i & k) == 0;
+            if ((x > y) == asc) { keys[i] = y; keys[ixj] = x; }
+          }
         }
+        __syncthreads();
       }
-      __syncthreads();
     }
-  }
-  // TopK_{K_f} -> Full, next TopK_{K_q} -> Quantized, remainder -> Evicted
-  for (int pos = tid; pos < n_cand; pos += ROUTE_THREADS) {
-    const uint32_t w = (uint32_t)keys[pos];
-    newt[w] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+    for (int pos = tid; pos < n_cand; pos += ROUTE_THREADS) {
+      const uint32_t c = (uint32_t)keys[pos];
+      cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+    }
   }
   __syncthreads();
 
-  // releases (page owner tables only; the per-window page ids stay readable until the lists are built)
-  for (int w = tid; w < nw; w += ROUTE_THREADS) {
-    const uint8_t old = tier[w], nt = newt[w];
-    if (old != QEVICT_TIER_FULL && old != QEVICT_TIER_QUANT && old != QEVICT_TIER_AGED) continue;
+  // ---- releases (owner tables only; the candidates' page ids stay readable until the lists are built) --
+  for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+    const uint8_t old = ctier[c], nt = cnew[c];
     if ((nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT) || nt == QEVICT_TIER_EVICTED) {
-      if (fp_page[w] >= 0) fp_owner[fp_page[w]] = -1;
+      if (cfp[c] >= 0) ofp[cfp[c]] = -1;
     }
-    if (nt == QEVICT_TIER_EVICTED && q_page[w] >= 0) q_owner[q_page[w]] = -1;
-    if (nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT && ledger[w] == QEVICT_LEDGER_DORMANT) {
-      ledger[w] = QEVICT_LEDGER_ACTIVE;  // reactivation: the retained codes are reused, no data moves
+    if (nt == QEVICT_TIER_EVICTED && cq[c] >= 0) oq[cq[c]] = -1;
+    if (nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT && cled[c] == QEVICT_LEDGER_DORMANT) {
+      cled[c] = QEVICT_LEDGER_ACTIVE;  // reactivation: the retained codes are reused, no data moves
       atomicAdd(s_react, 1);
     }
   }
   __syncthreads();
 
   // free pages in ascending id
-  const int n_free_fp = block_compact(g.PF, scratch, [&](int pg) { return fp_owner[pg] < 0; },
+  const int n_free_fp = block_compact(g.PF, scratch, [&](int pg) { return ofp[pg] < 0; },
                                       [&](int pg, int k) { free_fp[k] = pg; });
-  const int n_free_q = block_compact(g.PQ, scratch, [&](int pg) { return q_owner[pg] < 0; },
+  const int n_free_q = block_compact(g.PQ, scratch, [&](int pg) { return oq[pg] < 0; },
                                      [&](int pg, int k) { free_q[k] = pg; });
 
+  // first demotions need a quantized page, ascending window index.  reader[p] = index of the
+  // quantization that reads full-precision page p (free_fp is not needed before the next step, reuse
+  // free_q's neighbour array for the map)
+  const int qcap = g.PF + g.Kq;
+  int4* quant_list = a.st.quant_list + (size_t)u * qcap;
+  int32_t* reader = reinterpret_cast<int32_t*>(keys);  // [PF]; the sort keys are no longer needed
+  for (int i = tid; i < g.PF; i += ROUTE_THREADS) reader[i] = -1;
+  __syncthreads();
+  const int n_q_need = block_compact(
+      n_cand, scratch,
+      [&](int c) { return cnew[c] == QEVICT_TIER_QUANT && ctier[c] != QEVICT_TIER_QUANT && cled[c] == QEVICT_LEDGER_NONE; },
+      [&](int c, int k) {
+        if (k >= n_free_q || k >= qcap) { record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED); return; }
+        const int pg = free_q[k];
+        oq[pg] = cw[c];
+        quant_list[k] = make_int4(cw[c], prefill ? -1 : cfp[c], pg, -1);
+        if (!prefill && cfp[c] >= 0) reader[cfp[c]] = k;
+        cq[c] = pg;
+        cled[c] = QEVICT_LEDGER_ACTIVE;
+      });
   // windows entering the Full tier without a full-precision page (promotions; prompt windows at
-  // prefill), ascending window index
+  // prefill), ascending window index.  A promotion that receives a page some quantization of this event
+  // still has to read is linked to that quantization (the migration kernel runs it right after it).
   int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
   int4* copy_list = a.st.copy_list + (size_t)u * g.Kf;
   const int n_fp_need = block_compact(
-      nw, scratch, [&](int w) { return newt[w] == QEVICT_TIER_FULL && tier[w] != QEVICT_TIER_FULL && fp_page[w] < 0; },
-      [&](int w, int k) {
+      n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_FULL && ctier[c] != QEVICT_TIER_FULL && cfp[c] < 0; },
+      [&](int c, int k) {
         if (k >= n_free_fp || k >= g.Kf) { record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED); return; }
         const int pg = free_fp[k];
-        fp_owner[pg] = w;
-        fp_page[w] = pg;
-        if (prefill) copy_list[k] = make_int4(w, pg, 0, 0);
-        else promote_list[k] = make_int4(w, q_page[w], pg, 0);
-      });
-  // first demotions need a quantized page, ascending window index
-  const int qcap = g.PF + g.Kq;
-  int4* quant_list = a.st.quant_list + (size_t)u * qcap;
-  const int n_q_need = block_compact(
-      nw, scratch,
-      [&](int w) {
-        return newt[w] == QEVICT_TIER_QUANT && tier[w] != QEVICT_TIER_QUANT && tier[w] != QEVICT_TIER_EVICTED &&
-               tier[w] != QEVICT_TIER_OPEN && tier[w] != QEVICT_TIER_NONE && ledger[w] == QEVICT_LEDGER_NONE;
-      },
-      [&](int w, int k) {
-        if (k >= n_free_q || k >= qcap) { record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED); return; }
-        const int pg = free_q[k];
-        q_owner[pg] = w;
-        quant_list[k] = make_int4(w, prefill ? -1 : fp_page[w], pg, 0);
-        q_page[w] = pg;
-        ledger[w] = QEVICT_LEDGER_ACTIVE;
+        ofp[pg] = cw[c];
+        cfp[c] = pg;
+        if (prefill) {
+          copy_list[k] = make_int4(cw[c], pg, 0, 0);
+        } else {
+          const int rd = reader[pg];
+          promote_list[k] = make_int4(cw[c], cq[c], pg, rd >= 0 ? 1 : 0);
+          if (rd >= 0) quant_list[rd].w = k;
+        }
       });
 
-  // commit the new states
-  for (int w = tid; w < nw; w += ROUTE_THREADS) {
-    const uint8_t old = tier[w], nt = newt[w];
-    if (old != QEVICT_TIER_FULL && old != QEVICT_TIER_QUANT && old != QEVICT_TIER_AGED) continue;
+  // ---- commit: the candidates' rows and the owner tables go back to global memory --------------------
+  for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+    const uint8_t old = ctier[c], nt = cnew[c];
+    const int w = cw[c];
     if (nt == QEVICT_TIER_FULL) {
-      if (old == QEVICT_TIER_QUANT) ledger[w] = QEVICT_LEDGER_DORMANT;  // codes retained for a later demotion
+      if (old == QEVICT_TIER_QUANT) cled[c] = QEVICT_LEDGER_DORMANT;  // codes retained for a later demotion
     } else if (nt == QEVICT_TIER_QUANT) {
-      if (old != QEVICT_TIER_QUANT) fp_page[w] = -1;
+      if (old != QEVICT_TIER_QUANT) cfp[c] = -1;
     } else {  // evicted: everything released, ledger deleted
-      fp_page[w] = -1;
-      q_page[w] = -1;
-      ledger[w] = QEVICT_LEDGER_NONE;
+      cfp[c] = -1;
+      cq[c] = -1;
+      cled[c] = QEVICT_LEDGER_NONE;
       atomicAdd(s_del, 1);
     }
     tier[w] = nt;
+    ledger[w] = cled[c];
+    fp_page[w] = cfp[c];
+    q_page[w] = cq[c];
   }
+  for (int i = tid; i < g.PF; i += ROUTE_THREADS) fp_owner[i] = ofp[i];
+  for (int i = tid; i < g.PQ; i += ROUTE_THREADS) q_owner[i] = oq[i];
   __syncthreads();
 
-  // decode work list: Full.., Quantized.., open window last
+  // ---- decode work list: Full.., Quantized.., open window last ---------------------------------------
   uint2* entries = a.st.entries + (size_t)u * g.EMAX;
-  const int n_f = block_compact(nw, scratch, [&](int w) { return tier[w] == QEVICT_TIER_FULL; },
-                                [&](int w, int k) {
-                                  if (k < g.EMAX) entries[k] = make_uint2((uint32_t)w | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)fp_page[w]);
+  const int n_f = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_FULL; },
+                                [&](int c, int k) {
+                                  if (k < g.EMAX) entries[k] = make_uint2((uint32_t)cw[c] | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)cfp[c]);
                                 });
-  const int n_q = block_compact(nw, scratch, [&](int w) { return tier[w] == QEVICT_TIER_QUANT; },
-                                [&](int w, int k) {
-                                  if (n_f + k < g.EMAX) entries[n_f + k] = make_uint2((uint32_t)w | (KIND_Q << ENTRY_KIND_SHIFT), (uint32_t)q_page[w]);
+  const int n_q = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_QUANT; },
+                                [&](int c, int k) {
+                                  if (n_f + k < g.EMAX) entries[n_f + k] = make_uint2((uint32_t)cw[c] | (KIND_Q << ENTRY_KIND_SHIFT), (uint32_t)cq[c]);
                                 });
   if (tid == 0) {
     int n = n_f + n_q;
-    const int ow = a.st.open_window[u];
     if (ow >= 0) {
       if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)fp_page[ow]);
       n += 1;
     }
     if (n > g.EMAX) { record_check(a.st.status, CHECK_ENTRY_OVERFLOW); n = g.EMAX; }
     a.st.n_live[u] = n;
-    a.st.n_quant[u] = min(n_q_need, min(n_free_q, qcap));
-    a.st.n_promote[u] = prefill ? 0 : min(n_fp_need, min(n_free_fp, g.Kf));
-    a.st.n_copy[u] = prefill ? min(n_fp_need, min(n_free_fp, g.Kf)) : 0;
+    const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, g.Kf));
+    a.st.n_quant[u] = nq;
+    a.st.n_promote[u] = prefill ? 0 : nfp;
+    a.st.n_copy[u] = prefill ? nfp : 0;
     unsigned long long* c = a.st.counters + (size_t)u * 4;
-    c[0] += prefill ? 0 : (unsigned long long)min(n_fp_need, min(n_free_fp, g.Kf));
-    c[1] += (unsigned long long)min(n_q_need, min(n_free_q, qcap));
+    c[0] += prefill ? 0ull : (unsigned long long)nfp;
+    c[1] += (unsigned long long)nq;
     c[2] += (unsigned long long)*s_react;
     c[3] += (unsigned long long)*s_del;
   }
@@ -326,7 +399,7 @@ __global__ void export_mass_kernel(const KernelArgs a, int u, float* __restrict_
 }  // namespace
 
 size_t route_smem_bytes(const Geometry& g, int sort_cap) {
-  return (size_t)sort_cap * 8 + (size_t)(g.PF + g.PQ + 40) * 4 + (size_t)((g.NW + 15) / 16) * 16;
+  return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(2 * (g.PF + g.PQ) + 40) * 4 + 16;
 }
 
 cudaError_t route_prepare(size_t max_smem) {
