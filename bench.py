@@ -235,7 +235,8 @@ def run_ours(args, rank, world):
     for _ in range(K):
         step(t); t += 1
     torch.cuda.synchronize()
-    kernel_ms, kernel_n = cache.kernel_time()
+    ktimes = cache.kernel_times()
+    kernel_ms, kernel_n = ktimes["decode_attn"]
     cache.set_kernel_timing(False)
     stats = cache.stats()
     # ---- end to end: host buffers through the host entry point ----
@@ -288,6 +289,7 @@ def run_ours(args, rank, world):
             "kernel_share_of_step": k_avg_ms / (ms / K),
             "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
         },
+        "kernel_us_per_step": {k: round(v[0] * 1e3 / K, 2) for k, v in ktimes.items()},
         "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_open", "n_evicted", "promotions",
                                              "quantizations", "reactivations", "deletions")},
     }

@@ -189,11 +189,15 @@ QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, in
  * floating-point summation order. */
 QEVICT_API qevict_status qevict_set_splits(qevict_handle h, int32_t splits);
 
-/* Instrumentation: while enabled, every decode call brackets its attention kernel (the dominant
- * kernel of the path) with CUDA events on the call's stream.  qevict_kernel_time synchronises on the
- * recorded events, returns their summed duration in milliseconds and their count, and forgets them. */
+/* Instrumentation: while enabled, every kernel of the decode and rebalance calls is bracketed with CUDA
+ * events on the call's stream.  qevict_kernel_time synchronises on the recorded events, returns the
+ * summed duration in milliseconds and the launch count of the attention kernel (the dominant kernel of
+ * the path), and forgets all recorded events; qevict_kernel_times does the same for every kernel:
+ * index 0 append, 1 attention, 2 combine, 3 route, 4 migrate (arrays of QEVICT_N_KERNELS). */
+enum { QEVICT_N_KERNELS = 5 };
 QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enable);
 QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches);
+QEVICT_API qevict_status qevict_kernel_times(qevict_handle h, double* total_ms, uint64_t* n_launches);
 
 /* Number of kernels this handle has launched since creation (host counter). */
 QEVICT_API uint64_t qevict_launch_count(qevict_handle h);

@@ -54,6 +54,7 @@ _SIGNATURES = {
     "qevict_set_splits": (C.c_int, [C.c_void_p, C.c_int32]),
     "qevict_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32]),
     "qevict_kernel_time": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
+    "qevict_kernel_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
     "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -166,6 +167,16 @@ def qevict_kernel_time(h):
     return ms.value, n.value
 
 
+KERNEL_NAMES = ("append", "decode_attn", "combine", "route", "migrate")
+
+
+def qevict_kernel_times(h):
+    ms = (C.c_double * len(KERNEL_NAMES))()
+    n = (C.c_uint64 * len(KERNEL_NAMES))()
+    _check(lib().qevict_kernel_times(h, ms, n), h)
+    return {name: (ms[i], n[i]) for i, name in enumerate(KERNEL_NAMES)}
+
+
 def qevict_get_stats(h, layer=-1):
     st = qevict_stats()
     _check(lib().qevict_get_stats(h, layer, C.byref(st)), h)
@@ -231,6 +242,10 @@ class QEvictCache:
     def kernel_time(self):
         """(summed milliseconds, launches) of the attention kernel since the last call."""
         return qevict_kernel_time(self.handle)
+
+    def kernel_times(self):
+        """{kernel name: (summed milliseconds, launches)} since the last call."""
+        return qevict_kernel_times(self.handle)
 
     def stats(self, layer=-1):
         return qevict_get_stats(self.handle, layer)

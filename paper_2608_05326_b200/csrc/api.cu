@@ -48,6 +48,7 @@ struct qevict_ctx {
   int sm_count = SM_COUNT_FALLBACK;
   bool timing = false;
   std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
+  std::vector<int> ev_kind;           // kernel index of each pair
   size_t ev_used = 0;
   char* stage_q = nullptr;    // device staging for the host-buffer entry point
   char* stage_k = nullptr;
@@ -60,6 +61,34 @@ namespace {
 qevict_status fail(qevict_handle h, qevict_status s, const std::string& msg) {
   if (h) h->last_error = msg;
   return s;
+}
+
+// Brackets one kernel launch with events when instrumentation is on.
+template <class F>
+cudaError_t timed_launch(qevict_ctx* h, int kind, cudaStream_t stream, F launch) {
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (h->timing) {
+    if (h->ev_used + 2 > h->ev_pool.size()) {
+      cudaError_t e = cudaEventCreate(&e0);
+      if (e != cudaSuccess) return e;
+      e = cudaEventCreate(&e1);
+      if (e != cudaSuccess) return e;
+      h->ev_pool.push_back(e0);
+      h->ev_pool.push_back(e1);
+      h->ev_kind.push_back(kind);
+    }
+    e0 = h->ev_pool[h->ev_used];
+    e1 = h->ev_pool[h->ev_used + 1];
+    h->ev_kind[h->ev_used / 2] = kind;
+    h->ev_used += 2;
+    cudaError_t e = cudaEventRecord(e0, stream);
+    if (e != cudaSuccess) return e;
+  }
+  cudaError_t e = launch();
+  if (e != cudaSuccess) return e;
+  if (e1) e = cudaEventRecord(e1, stream);
+  h->launches++;
+  return e;
 }
 
 const char* validate(const qevict_config* c) {
@@ -226,8 +255,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   QE_CUDA(h, cudaSetDevice(h->cfg.device));
   const KernelArgs a = make_args(h, l0, l1);
   if (k_new) {
-    QE_CUDA(h, launch_append(a, k_new, v_new, stream));
-    h->launches++;
+    QE_CUDA(h, timed_launch(h, 0, stream, [&] { return launch_append(a, k_new, v_new, stream); }));
     for (int l = l0; l < l1; ++l) {
       LayerMirror& m = h->layers[l];
       if (!m.has_open) { m.has_open = true; m.open_fill = 0; m.n_windows++; }
@@ -239,24 +267,14 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  if (h->timing) {
-    if (h->ev_used + 2 > h->ev_pool.size()) {
-      cudaEvent_t e0, e1;
-      QE_CUDA(h, cudaEventCreate(&e0));
-      QE_CUDA(h, cudaEventCreate(&e1));
-      h->ev_pool.push_back(e0);
-      h->ev_pool.push_back(e1);
-    }
-    ev0 = h->ev_pool[h->ev_used]; ev1 = h->ev_pool[h->ev_used + 1];
-    h->ev_used += 2;
-    QE_CUDA(h, cudaEventRecord(ev0, stream));
+  QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
+  int e_bound = 1;  // upper bound of every unit's work-list length, from the host's mirror of the window counts
+  for (int l = l0; l < l1; ++l) {
+    const LayerMirror& m = h->layers[l];
+    const int e = g.Kf + g.Kq + m.aged + (m.has_open ? 1 : 0);
+    if (e > e_bound) e_bound = e;
   }
-  QE_CUDA(h, h->decode_fn(p, a.n_units, stream));
-  if (ev1) QE_CUDA(h, cudaEventRecord(ev1, stream));
-  h->launches++;
-  QE_CUDA(h, launch_combine(a, p.S, out, stream));
-  h->launches++;
+  QE_CUDA(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
   h->decode_steps++;
   return QEVICT_OK;
 }
@@ -378,18 +396,29 @@ QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enabl
   return QEVICT_OK;
 }
 
-QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches) {
+QEVICT_API qevict_status qevict_kernel_times(qevict_handle h, double* total_ms, uint64_t* n_launches) {
   if (!h || !total_ms || !n_launches) return QEVICT_ERR_INVALID_ARG;
-  double sum = 0.0;
+  for (int k = 0; k < QEVICT_N_KERNELS; ++k) { total_ms[k] = 0.0; n_launches[k] = 0; }
   for (size_t i = 0; i + 1 < h->ev_used; i += 2) {
     QE_CUDA(h, cudaEventSynchronize(h->ev_pool[i + 1]));
     float ms = 0.f;
     QE_CUDA(h, cudaEventElapsedTime(&ms, h->ev_pool[i], h->ev_pool[i + 1]));
-    sum += ms;
+    const int k = h->ev_kind[i / 2];
+    total_ms[k] += ms;
+    n_launches[k] += 1;
   }
-  *total_ms = sum;
-  *n_launches = h->ev_used / 2;
   h->ev_used = 0;
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches) {
+  if (!h || !total_ms || !n_launches) return QEVICT_ERR_INVALID_ARG;
+  double ms[QEVICT_N_KERNELS];
+  uint64_t n[QEVICT_N_KERNELS];
+  const qevict_status st = qevict_kernel_times(h, ms, n);
+  if (st != QEVICT_OK) return st;
+  *total_ms = ms[1];
+  *n_launches = n[1];
   return QEVICT_OK;
 }
 
@@ -467,12 +496,11 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   QE_CUDA(h, cudaSetDevice(h->cfg.device));
   cudaStream_t s = (cudaStream_t)stream;
   const KernelArgs a = make_args(h, l0, l1);
-  QE_CUDA(h, launch_route(a, 0, next_pow2(g.Kf + g.Kq + g.aged_cap + 1), s));
+  QE_CUDA(h, timed_launch(h, 3, s, [&] { return launch_route(a, 0, next_pow2(g.Kf + g.Kq + g.aged_cap + 1), s); }));
   // quantizations and promotions of the event in one launch (linked where they share a page)
   const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
   const int max_items = (g.Kq > 0 ? g.PF : 0) + max_promote;
-  QE_CUDA(h, launch_migrate(a, nullptr, nullptr, 0, max_items, s));
-  h->launches += 1 + (max_items > 0);
+  if (max_items > 0) QE_CUDA(h, timed_launch(h, 4, s, [&] { return launch_migrate(a, nullptr, nullptr, 0, max_items, s); }));
   for (int l = l0; l < l1; ++l) h->layers[l].aged = 0;
   return QEVICT_OK;
 }

@@ -140,6 +140,31 @@ __device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
 
 __device__ __forceinline__ void record_check(int32_t* status, int code) { atomicCAS(status, 0, code); }
 
+// Programmatic dependent launch: the kernels of a step are enqueued with launch_pdl and begin with
+// pdl_prologue().  The prologue first lets the next kernel of the stream start scheduling its CTAs, then
+// waits until every earlier kernel has completed and its writes are visible -- so launch latency and CTA
+// ramp-up of kernel n+1 overlap the tail of kernel n, while all data dependencies stay intact.
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // ---- kernels launched by the host API (defined in the .cu files) -------------------------------
 struct LaunchCtx {
   Geometry geo;

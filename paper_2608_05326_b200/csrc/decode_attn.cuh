@@ -319,6 +319,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const uint32_t ring = smem_u32(smem) + wid * NSLOT * TT::SLOT_BYTES;
   const uint32_t bars = smem_u32(smem) + TT::RING_BYTES + wid * NSLOT * 8;
+  pdl_prologue();
   if (lane == 0) {
 #pragma unroll
     for (int i = 0; i < NSLOT; ++i) mbar_init(bars + i * 8, 1);
@@ -516,8 +517,7 @@ cudaError_t launch_decode_attn(const DecodeParams& p, int n_units, cudaStream_t 
     prepared = true;
   }
   dim3 grid(p.S, p.Hkv, n_units);
-  decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK><<<grid, DECODE_WARPS * 32, TT::SMEM_BYTES, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK>, grid, dim3(DECODE_WARPS * 32), TT::SMEM_BYTES, stream, p);
 }
 
 // explicit dispatch table entry points, one per (dtype, D) translation unit

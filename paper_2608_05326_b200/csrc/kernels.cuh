@@ -16,7 +16,7 @@ struct KernelArgs {
 // A0: append one token per unit to its open window (opens one first if needed, zeroing the page).
 cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s);
 // A2: merge the split partials into `out`, add each window's mass to its score in fixed head order.
-cudaError_t launch_combine(const KernelArgs& a, int n_splits, void* out, cudaStream_t s);
+cudaError_t launch_combine(const KernelArgs& a, int n_splits, int e_bound, void* out, cudaStream_t s);
 
 // routing event ---------------------------------------------------------------------------------------
 // P0 (first half): every prompt window becomes an aged candidate with the given score.

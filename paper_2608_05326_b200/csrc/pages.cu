@@ -206,6 +206,7 @@ __global__ void __launch_bounds__(MIGRATE_THREADS) migrate_kernel(const KernelAr
   const Geometry& g = a.geo;
   const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y >> 1, part = blockIdx.y & 1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_prologue();
   const int n_quant = a.st.n_quant[u], n_promote = a.st.n_promote[u];
   const int4* quant_list = a.st.quant_list + (size_t)u * (g.PF + g.Kq);
   const int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
@@ -315,7 +316,7 @@ size_t migrate_smem_bytes(const Geometry& g) {
 // than keeps the whole launch near two thousand CTAs (lists are mostly short or empty at decode time).
 static int items_grid(int max_items, const KernelArgs& a) {
   const int pairs = a.geo.Hkv * 2 * a.n_units;
-  int per = 2048 / (pairs > 0 ? pairs : 1);
+  int per = 1024 / (pairs > 0 ? pairs : 1);
   if (per < 1) per = 1;
   return max_items < per ? max_items : per;
 }
@@ -328,11 +329,10 @@ cudaError_t launch_migrate(const KernelArgs& a, const void* k_prompt, const void
   if (max_items <= 0) return cudaSuccess;
   dim3 grid(items_grid(max_items, a), a.geo.Hkv * 2, a.n_units);
   const size_t sm = migrate_smem_bytes(a.geo);
-  QE_BY_DTYPE(a.geo,
-              (migrate_kernel<__half><<<grid, MIGRATE_THREADS, sm, s>>>(a, (const __half*)k_prompt, (const __half*)v_prompt, ctx)),
-              (migrate_kernel<__nv_bfloat16><<<grid, MIGRATE_THREADS, sm, s>>>(a, (const __nv_bfloat16*)k_prompt,
-                                                                         (const __nv_bfloat16*)v_prompt, ctx)));
-  return cudaGetLastError();
+  if (a.geo.dtype == QEVICT_DTYPE_FP16)
+    return launch_pdl(migrate_kernel<__half>, grid, dim3(MIGRATE_THREADS), sm, s, a, (const __half*)k_prompt, (const __half*)v_prompt, ctx);
+  return launch_pdl(migrate_kernel<__nv_bfloat16>, grid, dim3(MIGRATE_THREADS), sm, s, a, (const __nv_bfloat16*)k_prompt,
+                    (const __nv_bfloat16*)v_prompt, ctx);
 }
 
 cudaError_t launch_copy_prompt(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,

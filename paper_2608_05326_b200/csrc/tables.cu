@@ -68,84 +68,117 @@ __device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
 }
 
 // ------------------------------------------------------------------------------------------ append
+// One CTA per unit.  Global memory is waited on twice: the unit's scalars together with the new token,
+// then the open window's page id; everything else is stores.
 template <class T>
 __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T* __restrict__ k_new,
                                                      const T* __restrict__ v_new) {
   const Geometry& g = a.geo;
   const int ul = blockIdx.x, u = a.unit0 + ul, tid = threadIdx.x;
-  __shared__ int s_page, s_slot, s_new, s_window;
-  if (tid == 0) {
-    int ow = a.st.open_window[u];
-    int page = -1, is_new = 0, slot = 0;
-    if (ow < 0) {
-      const int w = a.st.n_windows[u];
-      if (w >= g.NW) {
-        record_check(a.st.status, CHECK_WINDOW_OVERFLOW);
-      } else {
-        int32_t* owner = a.st.fp_owner + (size_t)u * g.PF;
-        for (int pg = 0; pg < g.PF; ++pg) {
-          if (owner[pg] < 0) { page = pg; break; }
-        }
-        const int e = a.st.n_live[u];
-        if (page < 0) {
-          record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED);
-        } else if (e >= g.EMAX) {
-          record_check(a.st.status, CHECK_ENTRY_OVERFLOW);
-          page = -1;
-        } else {
-          owner[page] = w;
-          const size_t wi = (size_t)u * g.NW + w;
-          a.st.fp_page[wi] = page;
-          a.st.q_page[wi] = -1;
-          a.st.tier[wi] = QEVICT_TIER_OPEN;
-          a.st.ledger[wi] = QEVICT_LEDGER_NONE;
-          a.st.importance[wi] = 0.f;
-          a.st.n_windows[u] = w + 1;
-          a.st.open_window[u] = w;
-          a.st.entries[(size_t)u * g.EMAX + e] = make_uint2((uint32_t)w | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)page);
-          a.st.n_live[u] = e + 1;
-          ow = w;
-          is_new = 1;
-        }
-      }
-    } else {
-      page = a.st.fp_page[(size_t)u * g.NW + ow];
-      slot = a.st.open_fill[u];
+  __shared__ int s_page;
+  pdl_prologue();
+  // every thread reads the scalars itself (same addresses: one broadcast transaction each)
+  const int ow0 = a.st.open_window[u];
+  const int fill0 = a.st.open_fill[u];
+  const int n_live0 = a.st.n_live[u];
+  const int n_win0 = a.st.n_windows[u];
+  // the token: 16-byte pieces of the [H_kv][d] rows, in flight while the tables are being looked at
+  constexpr int MAXV = 4;  // pieces per thread kept in registers (H_kv * d <= 4096 elements)
+  const int nvec = g.Hkv * g.D / 8;
+  uint4 kx[MAXV], vx[MAXV];
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int v = tid + i * 128;
+    if (v < nvec) {
+      kx[i] = __ldg(reinterpret_cast<const uint4*>(k_new + (size_t)ul * g.Hkv * g.D) + v);
+      vx[i] = __ldg(reinterpret_cast<const uint4*>(v_new + (size_t)ul * g.Hkv * g.D) + v);
     }
-    s_page = page; s_slot = slot; s_new = is_new; s_window = ow;
   }
-  __syncthreads();
-  const int page = s_page, slot = s_slot;
-  if (page < 0) return;
+  int page, slot, window;
+  const bool is_new = ow0 < 0;
+  if (is_new) {
+    // open a window: it takes the lowest free full-precision page
+    window = n_win0;
+    slot = 0;
+    if (tid < 32) {
+      int found = -1;
+      const int32_t* owner = a.st.fp_owner + (size_t)u * g.PF;
+      for (int base = 0; base < g.PF && found < 0; base += 32) {
+        const int pg = base + tid;
+        const bool free_pg = pg < g.PF && owner[pg] < 0;
+        const unsigned m = __ballot_sync(0xffffffffu, free_pg);
+        if (m) found = base + __ffs(m) - 1;
+      }
+      if (tid == 0) s_page = found;
+    }
+    __syncthreads();
+    page = s_page;
+    if (window >= g.NW || page < 0 || n_live0 >= g.EMAX) {
+      if (tid == 0)
+        record_check(a.st.status, window >= g.NW ? CHECK_WINDOW_OVERFLOW : (page < 0 ? CHECK_FP_POOL_EXHAUSTED : CHECK_ENTRY_OVERFLOW));
+      return;
+    }
+  } else {
+    window = ow0;
+    slot = fill0;
+    page = a.st.fp_page[(size_t)u * g.NW + ow0];
+  }
   char* pbase = a.st.fp_pool + ((size_t)u * g.PF + page) * g.fp_page_bytes;
-  if (s_new) {
+  if (is_new) {
     // unfilled token slots of the open window must hold finite values (they are multiplied by a zero
     // probability in the PV product)
     uint4* z = reinterpret_cast<uint4*>(pbase);
-    for (uint32_t i = tid; i < g.fp_page_bytes / 16; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (uint32_t i = tid; i < g.fp_page_bytes / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
   }
   const int tile = slot >> 5, tk = slot & 31;
-  for (int idx = tid; idx < g.Hkv * g.D; idx += blockDim.x) {
-    const int h = idx / g.D, ch = idx - h * g.D;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int v = tid + i * 128;
+    if (v < nvec) {
+      const int h = (v * 8) / g.D, ch0 = v * 8 - h * g.D;
+      T* kt = reinterpret_cast<T*>(pbase + (size_t)h * g.fp_head_bytes + (size_t)tile * 2 * g.fp_tile_bytes);
+      T* vt = reinterpret_cast<T*>(reinterpret_cast<char*>(kt) + g.fp_tile_bytes);
+      const T* ke = reinterpret_cast<const T*>(&kx[i]);
+      const T* ve = reinterpret_cast<const T*>(&vx[i]);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        kt[fpk_off(tk, ch0 + e, g.D)] = ke[e];
+        vt[fpv_off(tk, ch0 + e)] = ve[e];
+      }
+    }
+  }
+  for (int v = tid + MAXV * 128; v < nvec; v += 128) {  // wider rows than the register buffer holds
+    const uint4 kk = __ldg(reinterpret_cast<const uint4*>(k_new + (size_t)ul * g.Hkv * g.D) + v);
+    const uint4 vv = __ldg(reinterpret_cast<const uint4*>(v_new + (size_t)ul * g.Hkv * g.D) + v);
+    const int h = (v * 8) / g.D, ch0 = v * 8 - h * g.D;
     T* kt = reinterpret_cast<T*>(pbase + (size_t)h * g.fp_head_bytes + (size_t)tile * 2 * g.fp_tile_bytes);
     T* vt = reinterpret_cast<T*>(reinterpret_cast<char*>(kt) + g.fp_tile_bytes);
-    kt[fpk_off(tk, ch, g.D)] = k_new[((size_t)ul * g.Hkv + h) * g.D + ch];
-    vt[fpv_off(tk, ch)] = v_new[((size_t)ul * g.Hkv + h) * g.D + ch];
-  }
-  __syncthreads();
-  if (tid == 0) {
-    const int fill = slot + 1;
-    if (fill == g.W) {
-      const int w = s_window;
-      a.st.tier[(size_t)u * g.NW + w] = QEVICT_TIER_AGED;
-      const int e = a.st.n_live[u] - 1;  // the open window is always the last entry
-      a.st.entries[(size_t)u * g.EMAX + e] = make_uint2((uint32_t)w | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)page);
-      a.st.open_window[u] = -1;
-      a.st.open_fill[u] = 0;
-    } else {
-      a.st.open_fill[u] = fill;
+    const T* ke = reinterpret_cast<const T*>(&kk);
+    const T* ve = reinterpret_cast<const T*>(&vv);
+    for (int e = 0; e < 8; ++e) {
+      kt[fpk_off(tk, ch0 + e, g.D)] = ke[e];
+      vt[fpv_off(tk, ch0 + e)] = ve[e];
     }
+  }
+  if (tid == 0) {
+    const size_t wi = (size_t)u * g.NW + window;
+    const int e_idx = is_new ? n_live0 : n_live0 - 1;  // the open window is always the last entry
+    const bool full = slot + 1 == g.W;
+    if (is_new) {
+      a.st.fp_owner[(size_t)u * g.PF + page] = window;
+      a.st.fp_page[wi] = page;
+      a.st.q_page[wi] = -1;
+      a.st.ledger[wi] = QEVICT_LEDGER_NONE;
+      a.st.importance[wi] = 0.f;
+      a.st.n_windows[u] = window + 1;
+      a.st.n_live[u] = n_live0 + 1;
+    }
+    a.st.tier[wi] = full ? QEVICT_TIER_AGED : QEVICT_TIER_OPEN;
+    a.st.entries[(size_t)u * g.EMAX + e_idx] =
+        make_uint2((uint32_t)window | ((full ? KIND_FP : KIND_OPEN) << ENTRY_KIND_SHIFT), (uint32_t)page);
+    a.st.open_window[u] = full ? -1 : window;
+    a.st.open_fill[u] = full ? 0 : slot + 1;
   }
 }
 
@@ -187,6 +220,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 40);                 // [sort_cap] state before
   uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
   uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
+  pdl_prologue();
 
   uint8_t* tier = a.st.tier + (size_t)u * g.NW;
   uint8_t* ledger = a.st.ledger + (size_t)u * g.NW;
@@ -409,10 +443,9 @@ cudaError_t route_prepare(size_t max_smem) {
 
 cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s) {
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
-    append_kernel<__half><<<a.n_units, 128, 0, s>>>(a, (const __half*)k_new, (const __half*)v_new);
-  else
-    append_kernel<__nv_bfloat16><<<a.n_units, 128, 0, s>>>(a, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
-  return cudaGetLastError();
+    return launch_pdl(append_kernel<__half>, dim3(a.n_units), dim3(128), 0, s, a, (const __half*)k_new, (const __half*)v_new);
+  return launch_pdl(append_kernel<__nv_bfloat16>, dim3(a.n_units), dim3(128), 0, s, a, (const __nv_bfloat16*)k_new,
+                    (const __nv_bfloat16*)v_new);
 }
 
 cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt, const float* scores, cudaStream_t s) {
@@ -422,8 +455,7 @@ cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt, const float* 
 }
 
 cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_cap, cudaStream_t s) {
-  route_kernel<<<a.n_units, ROUTE_THREADS, route_smem_bytes(a.geo, sort_cap), s>>>(a, prefill, sort_cap);
-  return cudaGetLastError();
+  return launch_pdl(route_kernel, dim3(a.n_units), dim3(ROUTE_THREADS), route_smem_bytes(a.geo, sort_cap), s, a, prefill, sort_cap);
 }
 
 cudaError_t launch_export_mass(const KernelArgs& a, int unit, float* mass, cudaStream_t s) {
