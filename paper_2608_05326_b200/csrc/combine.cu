@@ -19,7 +19,9 @@ constexpr int MAX_HQ = 128;
 template <class T>
 __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelArgs a, int S, int e_bound, T* __restrict__ out) {
   const Geometry& g = a.geo;
-  const int hk = blockIdx.x, ul = blockIdx.y, u = a.unit0 + ul, tid = threadIdx.x;
+  // blockIdx.x = chunk * Hkv + KV head: chunk 0 of every KV head also merges the attention output;
+  // every CTA owns 4 * NE consecutive work-list entries for the mass update
+  const int hk = blockIdx.x % a.geo.Hkv, ul = blockIdx.y, u = a.unit0 + ul, tid = threadIdx.x;
   const int lane = tid & 31, wid = tid >> 5;
   pdl_prologue();
   constexpr int NE = 8;  // work-list entries a warp keeps in registers at a time
@@ -28,10 +30,9 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   const float2* wrec = a.st.wrec + (size_t)u * g.Hq * g.EMAX;
   const uint2* entries = a.st.entries + (size_t)u * g.EMAX;
 
-  // This CTA's slice of the work list (bounds from the host's upper bound, so that nothing here waits
-  // for the list length); warp `wid` takes entries e0 + wid, e0 + wid + 4, ...; lane = query head.
-  const int per = (e_bound + g.Hkv - 1) / g.Hkv;
-  const int e0 = hk * per, e1 = min(min(e_bound, g.EMAX), e0 + per);
+  // This CTA's slice of the work list (the grid covers the host's upper bound of the list length, so
+  // nothing here waits for the length); warp `wid` takes entries e0 + wid, e0 + wid + 4, ...; lane = head.
+  const int e0 = blockIdx.x * (4 * NE), e1 = min(min(e_bound, g.EMAX), e0 + 4 * NE);
   const int n = a.st.n_live[u];
   float2 rec[NE];
   uint32_t ewin[NE];
@@ -70,7 +71,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
 
   // attention output of the heads of this KV head
   const float* op = a.st.o_part + (size_t)u * g.Hq * MAX_SPLITS * g.D;
-  for (int idx = tid; idx < g.G * g.D; idx += COMBINE_THREADS) {
+  for (int idx = tid; idx < g.G * g.D && blockIdx.x < g.Hkv; idx += COMBINE_THREADS) {
     const int hl = idx / g.D, ch = idx - hl * g.D, h = hk * g.G + hl;
     const float2* mlh = reinterpret_cast<const float2*>(ml) + (size_t)h * MAX_SPLITS;
     const float mx = s_m[h];
@@ -120,20 +121,13 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
       a.st.mass_e[(size_t)u * g.EMAX + e] = mass[k];
     }
   }
-  for (int e = e0 + wid + 4 * NE; e < e1 && e < n; e += 4) {  // slices longer than 4 * NE entries
-    const float2 r = (lane < g.Hq) ? __ldg(wrec + (size_t)lane * g.EMAX + e) : make_float2(0.f, 0.f);
-    const float m1 = head_sum(r, e);
-    if (lane == 0) {
-      a.st.importance[(size_t)u * g.NW + (__ldg(&entries[e].x) & ENTRY_WINDOW_MASK)] += m1;
-      a.st.mass_e[(size_t)u * g.EMAX + e] = m1;
-    }
-  }
 }
 
 }  // namespace
 
 cudaError_t launch_combine(const KernelArgs& a, int n_splits, int e_bound, void* out, cudaStream_t s) {
-  dim3 grid(a.geo.Hkv, a.n_units);
+  const int chunks = (e_bound + 31) / 32;  // 4 warps x 8 entries per CTA
+  dim3 grid(chunks > a.geo.Hkv ? chunks : a.geo.Hkv, a.n_units);
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
     return launch_pdl(combine_kernel<__half>, grid, dim3(COMBINE_THREADS), 0, s, a, n_splits, e_bound, (__half*)out);
   return launch_pdl(combine_kernel<__nv_bfloat16>, grid, dim3(COMBINE_THREADS), 0, s, a, n_splits, e_bound, (__nv_bfloat16*)out);

@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
 
   // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
   // Quantized, remainder -> Evicted -----------------------------------------------------------------
-  if (n_cand <= 1024) {
+  if (n_cand <= 512) {
     // rank of a key = number of smaller keys (all keys are distinct)
     for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
       const unsigned long long mine = keys[c];

@@ -103,7 +103,8 @@ def compare_state(cache, layer, seq, orc, wl, check_pages=None, what=""):
 class LockstepRun:
     """One workload instance on the GPU (all its units in one cache) and oracles for a subset of units."""
 
-    def __init__(self, wl, oracle_units=None, score_mode="observation", rebalance_interval=None, device="cuda"):
+    def __init__(self, wl, oracle_units=None, score_mode="observation", rebalance_interval=None, device="cuda",
+                 gen_device="cpu"):
         self.wl = wl
         self.R = wl.rebalance_interval if rebalance_interval is None else rebalance_interval
         self.units = list(range(wl.n_units)) if oracle_units is None else list(oracle_units)
@@ -112,26 +113,30 @@ class LockstepRun:
         ocfg = oracle_config(wl, aged_capacity(wl, self.R))
         self.oracles = {u: UnitOracle(ocfg) for u in self.units}
         self.k_prompt, self.scores, self.queries, self.new_kv = {}, {}, {}, {}
-        ks, vs, ss = [], [], []
-        for u in range(wl.n_units):
-            k, v = workloads.gen_prompt_kv(wl, u)
-            if u in self.oracles and score_mode == "observation":
-                s = observation_scores(wl, u, k.double().numpy())
-            else:
-                s = workloads.synthetic_window_scores(wl, u)
-            s = workloads.place_planted(s, workloads.planted_windows(wl, u), wl.fp_budget_windows, wl.q_budget_windows)
-            ks.append(k); vs.append(v); ss.append(s)
-            self.scores[u] = s
-            self.queries[u] = workloads.gen_queries(wl, u, k, s)
-            self.new_kv[u] = workloads.gen_new_kv(wl, u)
-            if u in self.oracles:
-                self.oracles[u].prefill_assign(k.double().numpy(), v.double().numpy(), s.numpy())
-        shape = (wl.n_layers, wl.batch, wl.n_kv_heads, wl.context, wl.head_dim)
-        kd = torch.stack(ks).reshape(shape).to(self.dev)
-        vd = torch.stack(vs).reshape(shape).to(self.dev)
-        sd = torch.stack(ss).reshape(wl.n_layers, wl.batch, -1).contiguous().to(self.dev)
-        self.cache.prefill_assign(-1, kd, vd, sd)
-        torch.cuda.synchronize()
+        # prompts are generated (on `gen_device`) and handed to the cache layer by layer; only the units
+        # that have an oracle are copied to the host
+        for layer in range(wl.n_layers):
+            ks, vs, ss = [], [], []
+            for u in range(layer * wl.batch, (layer + 1) * wl.batch):
+                k, v = workloads.gen_prompt_kv(wl, u, device=gen_device)
+                if u in self.oracles and score_mode == "observation":
+                    s = observation_scores(wl, u, k.cpu().double().numpy())
+                else:
+                    s = workloads.synthetic_window_scores(wl, u)
+                s = workloads.place_planted(s, workloads.planted_windows(wl, u), wl.fp_budget_windows,
+                                            wl.q_budget_windows)
+                ks.append(k); vs.append(v); ss.append(s)
+                self.scores[u] = s
+                self.queries[u] = workloads.gen_queries(wl, u, k, s)
+                self.new_kv[u] = workloads.gen_new_kv(wl, u)
+                if u in self.oracles:
+                    self.oracles[u].prefill_assign(k.cpu().double().numpy(), v.cpu().double().numpy(), s.numpy())
+            kd = torch.stack(ks).to(self.dev)
+            vd = torch.stack(vs).to(self.dev)
+            sd = torch.stack(ss).contiguous().to(self.dev)
+            self.cache.prefill_assign(layer, kd, vd, sd)
+            torch.cuda.synchronize()
+            del ks, vs, kd, vd
         self.step_idx = 0
 
     def unit_ls(self, u):

@@ -1,0 +1,61 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the whole workload
+runs on the GPU, the oracle follows a sample of its units step by step (outputs, per-window mass, tiers,
+page tables, codes), and properties that hold at any size are checked on every unit."""
+
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_05326_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, oracle_units, steps, rebalance_interval=1, check_all_units_mass=True):
+    import lockstep
+    wl = replace(wl, steps=steps)
+    run = lockstep.LockstepRun(wl, oracle_units=oracle_units, score_mode="synthetic",
+                               rebalance_interval=rebalance_interval, gen_device="cuda")
+    run.check_state({u: list(range(0, wl.n_prompt_windows, max(1, wl.n_prompt_windows // 40))) for u in oracle_units},
+                    "after prefill")
+    for t in range(steps):
+        run.step(append=True)
+        if check_all_units_mass and t % 4 == 0:
+            for u in range(wl.n_units):
+                m = run.cache.export_last_mass(u // wl.batch, u % wl.batch).double().sum().item()
+                assert abs(m - wl.n_q_heads) < 1e-4 * wl.n_q_heads, (u, m)
+    run.rebalance(full_check=False)
+    st = run.cache.stats()
+    assert st["n_full"] <= wl.n_units * wl.fp_budget_windows and st["n_quant"] <= wl.n_units * wl.q_budget_windows
+    for u in oracle_units:
+        o = run.oracles[u]
+        tab = run.cache.export_tables(u // wl.batch, u % wl.batch)
+        assert np.array_equal(tab["tier"].numpy()[: o.n_windows], o.tier[: o.n_windows])
+    run.close()
+    return st
+
+
+def test_config1_llama_32k_x32_layers_sampled_units():
+    wl = workloads.config(1, n_layers=32)
+    st = _run(wl, oracle_units=[0, 13, 31], steps=40)
+    assert st["n_full"] == 32 * 64 and st["n_quant"] == 32 * 128
+
+
+def test_config2_stacked_2bit_sampled_units():
+    # 16 sequences x 4 of the 32 layers (the per-unit work is the full-size one; fewer layers keep the
+    # test short), 2-bit codes, rebalance every step
+    wl = workloads.config(2, n_layers=4)
+    _run(wl, oracle_units=[5, 37, 63], steps=36)
+
+
+def test_config3_long_context_window64_sampled_unit():
+    wl = workloads.config(3)
+    _run(wl, oracle_units=[2], steps=70, check_all_units_mass=True)
+
+
+@pytest.mark.parametrize("bits,fp_frac", [(4, 0.10), (2, 0.20)])
+def test_config4_qwen_gqa7_sampled_unit(bits, fp_frac):
+    wl = workloads.config(4, bits=bits, fp_frac=fp_frac)
+    _run(wl, oracle_units=[3], steps=34, rebalance_interval=2)
