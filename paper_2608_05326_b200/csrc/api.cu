@@ -8,22 +8,11 @@
 #include <string>
 #include <vector>
 
-#include "decode_attn.cuh"
-#include "kernels.cuh"
+#include "ctx.h"
 
 using namespace qevict;
 
 namespace {
-
-struct LayerMirror {  // what the host must know without reading device memory (same for every sequence)
-  bool prefilled = false;
-  bool has_open = false;
-  int open_fill = 0;
-  int n_windows = 0;
-  int aged = 0;  // filled windows waiting for a routing event
-};
-
-constexpr int SM_COUNT_FALLBACK = 148;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -34,27 +23,6 @@ int next_pow2(int x) {
 }
 
 }  // namespace
-
-struct qevict_ctx {
-  qevict_config cfg;
-  Geometry geo;
-  State st;
-  std::vector<LayerMirror> layers;
-  std::string last_error;
-  uint64_t launches = 0;
-  uint64_t decode_steps = 0;
-  decode_launch_fn decode_fn = nullptr;
-  int forced_splits = 0;
-  int sm_count = SM_COUNT_FALLBACK;
-  bool timing = false;
-  std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
-  std::vector<int> ev_kind;           // kernel index of each pair
-  size_t ev_used = 0;
-  char* stage_q = nullptr;    // device staging for the host-buffer entry point
-  char* stage_k = nullptr;
-  char* stage_v = nullptr;
-  char* stage_out = nullptr;
-};
 
 namespace {
 
@@ -205,9 +173,11 @@ KernelArgs make_args(qevict_handle h, int l0, int l1) {
   return a;
 }
 
+}  // namespace
+
 // Splits per (unit, KV head): enough CTAs to fill the GPU in whole waves while every warp still walks
 // several windows.
-int choose_splits(const qevict_ctx* h, int n_units) {
+int qevict::choose_splits(const qevict_ctx* h, int n_units) {
   const Geometry& g = h->geo;
   // a warp holds its work-list entries one per lane: at most 32 entries per warp
   const int smin = (g.EMAX + 32 * DECODE_WARPS - 1) / (32 * DECODE_WARPS);
@@ -230,6 +200,8 @@ int choose_splits(const qevict_ctx* h, int n_units) {
   }
   return best;
 }
+
+namespace {
 
 #define QE_CUDA(h, expr)                                                                  \
   do {                                                                                    \

@@ -1,0 +1,50 @@
+// Private definition of the cache handle, shared by the translation units of the host API.
+#pragma once
+
+#include <string>
+#include <vector>
+
+#include "decode_attn.cuh"
+#include "kernels.cuh"
+
+namespace qevict {
+
+struct LayerMirror {  // what the host must know without reading device memory (same for every sequence)
+  bool prefilled = false;
+  bool has_open = false;
+  int open_fill = 0;
+  int n_windows = 0;
+  int aged = 0;  // filled windows waiting for a routing event
+};
+
+constexpr int SM_COUNT_FALLBACK = 148;
+
+}  // namespace qevict
+
+struct qevict_ctx {
+  qevict_config cfg;
+  qevict::Geometry geo;
+  qevict::State st;
+  std::vector<qevict::LayerMirror> layers;
+  std::string last_error;
+  uint64_t launches = 0;
+  uint64_t decode_steps = 0;
+  qevict::decode_launch_fn decode_fn = nullptr;
+  int forced_splits = 0;
+  int sm_count = qevict::SM_COUNT_FALLBACK;
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
+  std::vector<int> ev_kind;           // kernel index of each pair
+  size_t ev_used = 0;
+  char* stage_q = nullptr;    // device staging for the host-buffer entry point
+  char* stage_k = nullptr;
+  char* stage_v = nullptr;
+  char* stage_out = nullptr;
+};
+
+namespace qevict {
+
+// Splits per (unit, KV head) of the attention kernel for a call over `n_units` units.
+int choose_splits(const qevict_ctx* h, int n_units);
+
+}  // namespace qevict
