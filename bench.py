@@ -26,14 +26,17 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2608_05326_b200 import workloads  # noqa: E402
+from paper_2608_05326_b200 import sharding, workloads  # noqa: E402
 
 METRIC = "decode_steps_per_sec"
 UNIT = "steps/s"
 HBM_FALLBACK_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures
 # summarised under profiles/ (bytes per launch, keyed by workload name); None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/decode_attn_c1x32.md: 440.83 MB read + 6.50 MB written per launch
+    "c1-llama3-8b-32k": 447_330_000,
+}
 
 
 def parse_args():
@@ -183,7 +186,7 @@ def run_ours(args, rank, world):
     phases = 2 + (0 if args.no_e2e else 1)
     total_steps = W + phases * K
     wl = make_workload(args, total_steps)
-    wl = replace(wl, seed=wl.seed + rank)  # every rank owns its own sequences (weak scaling, no exchange)
+    wl = sharding.rank_workload(wl, rank)  # every rank owns its own sequences (weak scaling, no exchange)
     cfg = binding.make_config(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window,
                               wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
                               rebalance_interval_hint=args.rebalance_interval, device=dev.index)
@@ -255,12 +258,9 @@ def run_ours(args, rank, world):
         h2d = qh[0].numel() * 2 + (2 * knh[0].numel() * 2 if append else 0)
         e2e = {"seconds": e2e_s, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": outh.numel() * 2}
 
-    if world > 1:
-        tm = torch.tensor([ms, e2e["seconds"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(tm, op=torch.distributed.ReduceOp.MAX)
-        ms = float(tm[0]);
-        if e2e:
-            e2e["seconds"] = float(tm[1])
+    ms, e2e_s = sharding.max_over_ranks([ms, e2e["seconds"] if e2e else 0.0], device=dev)
+    if e2e:
+        e2e["seconds"] = e2e_s
     if rank != 0:
         cache.close()
         return None
@@ -269,7 +269,7 @@ def run_ours(args, rank, world):
     k_avg_ms = kernel_ms / max(kernel_n, 1)
     achieved = kbytes / (k_avg_ms * 1e-3) / 1e9 if k_avg_ms > 0 else 0.0
     line = {
-        "metric": METRIC, "value": world * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "metric": METRIC, "value": sharding.aggregate_steps_per_second(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
         "data": "synthetic",
         "config": {
