@@ -150,6 +150,31 @@ QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer,
                                       const void* k_new_host, const void* v_new_host, void* out_host,
                                       void* stream);
 
+/* The same decode step for callers that must not allocate device memory (the paper has no counterpart:
+ * this is a deployment variant of qevict_decode_attn, not a step of the method).
+ *
+ * Who needs it: code that runs under a fixed device-memory plan.  A serving process that hands all of
+ * HBM to its own pool at start-up has nothing left for a library to allocate from; a latency-critical
+ * thread must not enter the CUDA allocator, which can block behind other work on the device.  Such a
+ * caller can still build a cache inside memory it already owns (qevict_create takes the buffer), but the
+ * attention kernel also wants scratch for its per-split partial results.  This entry point keeps that
+ * scratch in a fixed array of QEVICT_NOALLOC_SCRATCH_BYTES that is part of the library's device image:
+ * every GPU that loads the library holds those bytes until the process exits, and nothing is allocated
+ * or freed by the call (no cudaMalloc / cudaFree, no allocating library routine).
+ *
+ * Arguments, results and state changes are those of qevict_decode_attn.  Differences:
+ *   - A call whose scratch (partials for all units up to the last unit of the call) does not fit the
+ *     array returns QEVICT_ERR_NO_MEMORY and enqueues nothing; qevict_last_error states the size needed.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) before it
+ *     launches anything.  Make that first call before any stream capture begins.
+ *   - All calls, on all handles and streams of a device, share the one array, which keeps the last
+ *     call's contents.  Nothing in it has to start at zero -- every slot a call reads it has written
+ *     first -- but two calls that overlap on the GPU race on it: keep them in one stream, or order them
+ *     with events. */
+#define QEVICT_NOALLOC_SCRATCH_BYTES (8u << 20)
+QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, int32_t layer, const void* q, const void* k_new,
+                                                    const void* v_new, void* out, void* stream);
+
 /* One routing event [Algorithm 1].  Candidates = Full, Quantized and aged windows, ranked by score
  * (float32, higher first, lower window index first among equals); the first K_f become Full, the next
  * K_q Quantized, the rest Evicted.  Pages are released, then handed out in ascending page id to the

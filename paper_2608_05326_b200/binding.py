@@ -58,6 +58,7 @@ _SIGNATURES = {
     "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_decode_attn_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_rebalance": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "qevict_get_stats": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(qevict_stats)]),
     "qevict_export_tables": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 7),
@@ -147,6 +148,12 @@ def qevict_decode_attn(h, layer, q, k_new, v_new, out, stream=None):
 def qevict_decode_attn_host(h, layer, q, k_new, v_new, out, stream=None):
     """q, k_new, v_new, out: HOST tensors (pinned or pageable)."""
     _check(lib().qevict_decode_attn_host(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
+
+
+def qevict_decode_attn_noalloc(h, layer, q, k_new, v_new, out, stream=None):
+    """qevict_decode_attn with the attention scratch in the library's built-in device array: for callers
+    that must not allocate device memory.  Raises QEvictError(NO_MEMORY) if the call's scratch does not fit."""
+    _check(lib().qevict_decode_attn_noalloc(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
 
 
 def qevict_rebalance(h, layer, stream=None):
