@@ -30,6 +30,11 @@ Readings taken where the paper is silent (each is listed in the design notes):
     routing event, windows that need a page take the free page ids in ascending
     order, in ascending window index; a newly opened window takes the lowest
     free full-precision page.
+
+Parity unpinned: the page-id assignment order above is this build's own rule (the
+paper never speaks of pages), so nothing outside this file fixes it; and the
+prefill window scores are an input here (the paper only says that prompt attention
+initialises them), so their definition is pinned by nothing beyond Eq. 1's form.
 """
 
 from dataclasses import dataclass
