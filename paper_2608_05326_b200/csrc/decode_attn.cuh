@@ -132,37 +132,38 @@ __device__ __forceinline__ void qk_fp_half(float (&s)[4][4], int j0, const uint3
   }
 }
 
-// Key part of a quantized tile: codes at `slot`, parameters at `slot + KC_BYTES`.
+// Key part of a quantized tile: codes at `slot`, parameters at `slot + KC_BYTES`.  The codes of one
+// channel group (two k-steps; four with 2-bit codes) for all four token blocks are one 16-byte vector, so
+// only four code words are live at a time.
 template <class T, int D, int BITS>
 __device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
   constexpr int KG = D / 32;
-  constexpr int WPL = 32 * D * BITS / 8 / 128;
   constexpr uint32_t KC_BYTES = 32 * D * BITS / 8;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
+  constexpr int CPV = (BITS == 4) ? 1 : 2;  // channel groups per code vector
   const int t = lane & 3;
-  uint32_t cw[WPL];
-#pragma unroll
-  for (int v = 0; v < WPL / 4; ++v) {
-    const uint4 x = lds16(slot + (v * 32 + lane) * 16);
-    cw[4 * v] = x.x; cw[4 * v + 1] = x.y; cw[4 * v + 2] = x.z; cw[4 * v + 3] = x.w;
-  }
   const uint32_t kp = slot + KC_BYTES;
 #pragma unroll
-  for (int c = 0; c < KG; ++c) {
-    const uint4 p0 = lds16(kp + ((c * 2 + 0) * 4 + t) * 16);  // k-step 2c:   {s,z} low / high channel octet
-    const uint4 p1 = lds16(kp + ((c * 2 + 1) * 4 + t) * 16);  // k-step 2c+1
+  for (int v = 0; v < KG / CPV; ++v) {
+    const uint4 cv = lds16(slot + (v * 32 + lane) * 16);  // token blocks j = 0..3
+    const uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t w;
-      int sh;
-      if (BITS == 4) { w = cw[j * KG + c]; sh = 0; } else { w = cw[j * (KG / 2) + (c >> 1)]; sh = (c & 1) * 8; }
-      const uint32_t b0 = dequant2<T>(((w >> (sh + 0 * BITS)) & MASK) | MG, p0.x, p0.y);
-      const uint32_t b1 = dequant2<T>(((w >> (sh + 1 * BITS)) & MASK) | MG, p0.z, p0.w);
-      const uint32_t b2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, p1.x, p1.y);
-      const uint32_t b3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, p1.z, p1.w);
-      mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, b0, b1);
-      mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, b2, b3);
+    for (int cc = 0; cc < CPV; ++cc) {
+      const int c = v * CPV + cc;
+      const int sh = cc * 8;
+      const uint4 p0 = lds16(kp + ((c * 2 + 0) * 4 + t) * 16);  // k-step 2c:   {s,z} low / high channel octet
+      const uint4 p1 = lds16(kp + ((c * 2 + 1) * 4 + t) * 16);  // k-step 2c+1
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t w = cw[j];
+        const uint32_t b0 = dequant2<T>(((w >> (sh + 0 * BITS)) & MASK) | MG, p0.x, p0.y);
+        const uint32_t b1 = dequant2<T>(((w >> (sh + 1 * BITS)) & MASK) | MG, p0.z, p0.w);
+        const uint32_t b2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, p1.x, p1.y);
+        const uint32_t b3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, p1.z, p1.w);
+        mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, b0, b1);
+        mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, b2, b3);
+      }
     }
   }
 }
@@ -183,35 +184,36 @@ __device__ __forceinline__ void pv_fp_half(float (&o)[D / 16][4], int i0, const 
   }
 }
 
-// Value part of a quantized tile: codes at `slot`, parameters at `slot + VC_BYTES`.
+// Value part of a quantized tile: codes at `slot`, parameters at `slot + VC_BYTES`.  One 16-byte code
+// vector covers two channel blocks (four with 2-bit codes) and is fetched right before it is used.
 template <class T, int D, int BITS, int GROUP, bool PACK>
 __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2], const uint32_t (&pb)[2][2],
                                           uint32_t slot, int lane) {
-  constexpr int WPL = 32 * D * BITS / 8 / 128;
+  constexpr int MT = D / 16;
   constexpr uint32_t VC_BYTES = 32 * D * BITS / 8;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
+  constexpr int IPV = (BITS == 4) ? 2 : 4;  // channel blocks (of 16) per code vector
   const int t = lane & 3;
-  uint32_t vw[WPL];
-#pragma unroll
-  for (int v = 0; v < WPL / 4; ++v) {
-    const uint4 x = lds16(slot + (v * 32 + lane) * 16);
-    vw[4 * v] = x.x; vw[4 * v + 1] = x.y; vw[4 * v + 2] = x.z; vw[4 * v + 3] = x.w;
-  }
   const uint32_t vp = slot + VC_BYTES;
+  uint4 pr0 = make_uint4(0u, 0u, 0u, 0u), pr1 = pr0;
 #pragma unroll
-  for (int gc = 0; gc < D / GROUP; ++gc) {
-    const uint4 pr0 = lds16(vp + ((gc * 2 + 0) * 4 + t) * 16);  // tokens 0..15:  {s,z} low octet, {s,z} high octet
-    const uint4 pr1 = lds16(vp + ((gc * 2 + 1) * 4 + t) * 16);  // tokens 16..31
+  for (int v = 0; v < MT / IPV; ++v) {
+    const uint4 cv = lds16(slot + (v * 32 + lane) * 16);
+    const uint32_t vw[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-    for (int ii = 0; ii < GROUP / 16; ++ii) {
-      const int i = gc * (GROUP / 16) + ii;
+    for (int ii = 0; ii < IPV; ++ii) {
+      const int i = v * IPV + ii;
+      if ((16 * i) % GROUP == 0) {  // a new channel group starts: its per-token parameters
+        const int gc = (16 * i) / GROUP;
+        pr0 = lds16(vp + ((gc * 2 + 0) * 4 + t) * 16);  // tokens 0..15:  {s,z} low octet, {s,z} high octet
+        pr1 = lds16(vp + ((gc * 2 + 1) * 4 + t) * 16);  // tokens 16..31
+      }
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         const uint4 pr = ks ? pr1 : pr0;
-        uint32_t w;
-        int sh;
-        if (BITS == 4) { w = vw[i * 2 + ks]; sh = 0; } else { w = vw[i]; sh = ks * 8; }
+        const uint32_t w = (BITS == 4) ? vw[ii * 2 + ks] : vw[ii];
+        const int sh = (BITS == 4) ? 0 : ks * 8;
         const uint32_t a0 = dequant2<T>(((w >> (sh + 0 * BITS)) & MASK) | MG, pr.x, pr.y);
         const uint32_t a1 = dequant2<T>(((w >> (sh + 1 * BITS)) & MASK) | MG, pr.x, pr.y);
         const uint32_t a2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, pr.z, pr.w);

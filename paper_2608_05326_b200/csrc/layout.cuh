@@ -58,11 +58,13 @@ QE_HD CodePos kcode_pos(int tk, int ch, int D, int bits) {
   const int lane = g * 4 + t;
   const int m = ks * 2 + hi;
   CodePos p;
+  // word index = channel-group * 4 + token block: one 16-byte vector holds the four token blocks of a
+  // channel group, so the attention kernel fetches the codes of one k-step pair at a time
   if (bits == 4) {
-    p.word = code_word_off(j * (D >> 5) + c, lane);
+    p.word = code_word_off(c * 4 + j, lane);
     p.shift = 4 * m + 16 * e;
   } else {
-    p.word = code_word_off(j * (D >> 6) + (c >> 1), lane);
+    p.word = code_word_off((c >> 1) * 4 + j, lane);
     p.shift = 2 * ((c & 1) * 4 + m) + 16 * e;
   }
   return p;

@@ -127,8 +127,7 @@ __device__ void quantize_part(const Geometry& g, int part, const T* __restrict__
         const int e = k & 1, m = (k >> 1) & 3, sub = k >> 3;
         int tk, ch;
         if (part == 0) {
-          const int per_j = g.bits == 4 ? KG : KG / 2;
-          const int j = widx / per_j, c = (widx - j * per_j) * (g.bits == 4 ? 1 : 2) + sub;
+          const int j = widx & 3, c = (widx >> 2) * (g.bits == 4 ? 1 : 2) + sub;  // widx = channel group * 4 + j
           tk = 8 * j + gg;
           ch = 32 * c + 16 * (m >> 1) + 8 * (m & 1) + 2 * tt + e;
         } else {
@@ -163,7 +162,7 @@ __device__ void promote_part(const Geometry& g, int part, const char* __restrict
       uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
       for (int v = wid; v < 4 * KG; v += nwarps) {  // key vectors (j, c)
         const int j = v / KG, c = v - j * KG;
-        const int widx = bits == 4 ? j * KG + c : j * (KG / 2) + (c >> 1);
+        const int widx = (bits == 4 ? c : (c >> 1)) * 4 + j;
         const int sh = bits == 4 ? 0 : (c & 1) * 8;
         const uint32_t w = kc[code_word_off(widx, lane)];
         const uint4 p0 = kp[(c * 2 + 0) * 4 + t], p1 = kp[(c * 2 + 1) * 4 + t];
