@@ -12,7 +12,7 @@
 //
 // Data movement: every warp owns a ring of NSLOT shared-memory slots.  Lane 0 streams the warp's
 // pages into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on one
-// mbarrier per slot) NSLOT-1 pieces ahead of the math; a page is stored fragment-major (layout.cuh),
+// mbarrier per slot) one piece ahead of the math; a page is stored fragment-major (layout.cuh),
 // so a piece is one contiguous run in global memory and every lane reads its operands from shared
 // memory with conflict-free 16-byte loads.  Waits on the mbarriers are bounded: a wait that runs out
 // records CHECK_COPY_TIMEOUT, the warp stops issuing, drains what it has in flight and returns.
@@ -46,7 +46,7 @@ struct DecodeParams {
   float scale_log2;
 };
 
-static constexpr int NSLOT = 4;                   // ring slots per warp
+static constexpr int NSLOT = 2;                   // ring slots per warp
 static constexpr uint32_t WAIT_LIMIT = 1u << 20;  // mbarrier try_wait attempts before giving up
 
 template <class T, int D, int BITS, int GROUP, int TILES>
@@ -64,12 +64,12 @@ struct DecodeTraits {
   static constexpr uint32_t KP_BYTES = D * 4;
   static constexpr uint32_t KP_OFF = TILES * Q_TILE_STRIDE;
   static constexpr uint32_t Q_HEAD_BYTES = KP_OFF + (W / GROUP) * KP_BYTES;
-  // a ring slot holds half of a full-precision key or value tile, or the key part (codes + params)
-  // or the value part (codes + params) of a quantized tile
-  static constexpr uint32_t SLOT_BYTES = FP_TILE_BYTES / 2;
+  // a ring slot holds a full-precision key tile or value tile, or a whole quantized tile
+  // (key codes, value codes, value params as they lie in the page, then the key params)
+  static constexpr uint32_t SLOT_BYTES = FP_TILE_BYTES;
   static constexpr uint32_t RING_BYTES = DECODE_WARPS * NSLOT * SLOT_BYTES;
   static constexpr uint32_t SMEM_BYTES = RING_BYTES + DECODE_WARPS * NSLOT * 8;
-  static_assert(KC_BYTES + KP_BYTES <= SLOT_BYTES && VC_BYTES + VP_BYTES <= SLOT_BYTES, "quantized part must fit a slot");
+  static_assert(Q_TILE_STRIDE + KP_BYTES <= SLOT_BYTES, "a quantized tile must fit a slot");
   static_assert(8 * (D + 4) * 4 + 64 <= NSLOT * SLOT_BYTES, "merge buffer must fit the warp's ring");
 };
 
@@ -116,34 +116,32 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // ---- S = Q K^T -----------------------------------------------------------------------------------------
-// Half of a full-precision key tile (16 tokens: score blocks j0, j0+1) from a ring slot.
+// A full-precision key tile (32 tokens) from a ring slot.
 template <class T, int D>
-__device__ __forceinline__ void qk_fp_half(float (&s)[4][4], int j0, const uint32_t (&qa)[D / 16][2], uint32_t slot,
-                                           int lane) {
+__device__ __forceinline__ void qk_fp_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
   constexpr int KG = D / 32;
 #pragma unroll
-  for (int jj = 0; jj < 2; ++jj) {
+  for (int c = 0; c < KG; ++c) {
 #pragma unroll
-    for (int c = 0; c < KG; ++c) {
-      const uint4 kv = lds16(slot + ((jj * KG + c) * 32 + lane) * 16);
-      mma16816<T>(s[j0 + jj], qa[2 * c][0], 0u, qa[2 * c][1], 0u, kv.x, kv.y);
-      mma16816<T>(s[j0 + jj], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, kv.z, kv.w);
+    for (int j = 0; j < 4; ++j) {
+      const uint4 kv = lds16(slot + ((j * KG + c) * 32 + lane) * 16);
+      mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, kv.x, kv.y);
+      mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, kv.z, kv.w);
     }
   }
 }
 
-// Key part of a quantized tile: codes at `slot`, parameters at `slot + KC_BYTES`.  The codes of one
+// Key part of a quantized tile: codes at `codes`, parameters at `kp`.  The codes of one
 // channel group (two k-steps; four with 2-bit codes) for all four token blocks are one 16-byte vector, so
 // only four code words are live at a time.
 template <class T, int D, int BITS>
-__device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
+__device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
+                                          int lane) {
   constexpr int KG = D / 32;
-  constexpr uint32_t KC_BYTES = 32 * D * BITS / 8;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
   constexpr int CPV = (BITS == 4) ? 1 : 2;  // channel groups per code vector
   const int t = lane & 3;
-  const uint32_t kp = slot + KC_BYTES;
 #pragma unroll
   for (int v = 0; v < KG / CPV; ++v) {
     const uint4 cv = lds16(slot + (v * 32 + lane) * 16);  // token blocks j = 0..3
@@ -169,17 +167,17 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)
 }
 
 // ---- O^T += V^T P^T ----------------------------------------------------------------------------------------
-// Half of a full-precision value tile (channel blocks i0 .. i0 + MT/2 - 1) from a ring slot.
+// A full-precision value tile from a ring slot.
 template <class T, int D, bool PACK>
-__device__ __forceinline__ void pv_fp_half(float (&o)[D / 16][4], int i0, const uint32_t (&pa)[2][2],
-                                           const uint32_t (&pb)[2][2], uint32_t slot, int lane) {
+__device__ __forceinline__ void pv_fp_tile(float (&o)[D / 16][4], const uint32_t (&pa)[2][2], const uint32_t (&pb)[2][2],
+                                           uint32_t slot, int lane) {
 #pragma unroll
-  for (int ii = 0; ii < D / 32; ++ii) {
+  for (int ks = 0; ks < 2; ++ks) {
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      const uint4 vv = lds16(slot + ((ii * 2 + ks) * 32 + lane) * 16);
-      mma16816<T>(o[i0 + ii], vv.x, vv.y, vv.z, vv.w, pa[ks][0], pa[ks][1]);
-      if (!PACK) mma16816<T>(o[i0 + ii], vv.x, vv.y, vv.z, vv.w, pb[ks][0], pb[ks][1]);
+    for (int i = 0; i < D / 16; ++i) {
+      const uint4 vv = lds16(slot + ((i * 2 + ks) * 32 + lane) * 16);
+      mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pa[ks][0], pa[ks][1]);
+      if (!PACK) mma16816<T>(o[i], vv.x, vv.y, vv.z, vv.w, pb[ks][0], pb[ks][1]);
     }
   }
 }
@@ -359,43 +357,40 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   if (lane < my_n) my_ent = p.entries[(size_t)u * p.EMAX + first + (size_t)lane * stride];
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
-  // piece counts: full-precision tile = 4 (K lo, K hi, V lo, V hi), quantized tile = 2 (K part, V part)
+  // pieces per tile: full precision = 2 (key tile, value tile), quantized = 1 (the whole tile)
   int n_pieces;
   {
-    int mine = lane < my_n ? (((my_ent.x >> ENTRY_KIND_SHIFT) == KIND_Q) ? 2 : 4) * TILES : 0;
+    int mine = lane < my_n ? (((my_ent.x >> ENTRY_KIND_SHIFT) == KIND_Q) ? 1 : 2) * TILES : 0;
 #pragma unroll
     for (int o2 = 16; o2 > 0; o2 >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o2);
     n_pieces = mine;
   }
   int pr_ci = 0, pr_tile = 0, pr_part = 0, issued = 0, consumed = 0;
-  bool dead = false;
+  bool dead = false, pr_isq = false;
+  const char* pr_base = nullptr;  // page of the producer's current entry (this KV head), set on its first piece
+  const char* const fp_unit = p.fp_pool + (size_t)u * p.PF * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES;
+  const char* const q_unit = p.q_pool + (size_t)u * p.PQ * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
   auto issue_next = [&]() {  // warp-collective
     if (issued >= n_pieces || dead) return;
-    const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, pr_ci), ey = __shfl_sync(0xffffffffu, my_ent.y, pr_ci);
-    const bool isq = (ex >> ENTRY_KIND_SHIFT) == KIND_Q;
+    if (pr_tile == 0 && pr_part == 0) {
+      const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, pr_ci), ey = __shfl_sync(0xffffffffu, my_ent.y, pr_ci);
+      pr_isq = (ex >> ENTRY_KIND_SHIFT) == KIND_Q;
+      pr_base = pr_isq ? q_unit + (size_t)ey * p.q_page_bytes : fp_unit + (size_t)ey * p.fp_page_bytes;
+    }
     if (lane == 0) {
       const int slot = issued % NSLOT;
       const uint32_t dst = ring + slot * TT::SLOT_BYTES, bar = bars + slot * 8;
-      if (!isq) {
-        const char* src = p.fp_pool + ((size_t)u * p.PF + ey) * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES +
-                          (size_t)pr_tile * 2 * TT::FP_TILE_BYTES + (size_t)pr_part * TT::SLOT_BYTES;
-        mbar_expect_tx(bar, TT::SLOT_BYTES);
-        bulk_g2s(dst, src, TT::SLOT_BYTES, bar);
+      if (!pr_isq) {
+        mbar_expect_tx(bar, TT::FP_TILE_BYTES);
+        bulk_g2s(dst, pr_base + (size_t)(pr_tile * 2 + pr_part) * TT::FP_TILE_BYTES, TT::FP_TILE_BYTES, bar);
       } else {
-        const char* base = p.q_pool + ((size_t)u * p.PQ + ey) * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
-        const char* tb = base + (size_t)pr_tile * TT::Q_TILE_STRIDE;
-        if (pr_part == 0) {
-          mbar_expect_tx(bar, TT::KC_BYTES + TT::KP_BYTES);
-          bulk_g2s(dst, tb, TT::KC_BYTES, bar);
-          bulk_g2s(dst + TT::KC_BYTES, base + TT::KP_OFF + (size_t)((pr_tile * 32) / GROUP) * TT::KP_BYTES, TT::KP_BYTES, bar);
-        } else {
-          mbar_expect_tx(bar, TT::VC_BYTES + TT::VP_BYTES);
-          bulk_g2s(dst, tb + TT::KC_BYTES, TT::VC_BYTES + TT::VP_BYTES, bar);
-        }
+        mbar_expect_tx(bar, TT::Q_TILE_STRIDE + TT::KP_BYTES);
+        bulk_g2s(dst, pr_base + (size_t)pr_tile * TT::Q_TILE_STRIDE, TT::Q_TILE_STRIDE, bar);
+        bulk_g2s(dst + TT::Q_TILE_STRIDE, pr_base + TT::KP_OFF + (size_t)((pr_tile * 32) / GROUP) * TT::KP_BYTES, TT::KP_BYTES, bar);
       }
     }
     ++issued;
-    if (++pr_part == (isq ? 2 : 4)) {
+    if (++pr_part == (pr_isq ? 1 : 2)) {
       pr_part = 0;
       if (++pr_tile == TILES) { pr_tile = 0; ++pr_ci; }
     }
@@ -433,29 +428,21 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
       uint32_t pa[2][2], pb[2][2];
       if (kind != KIND_Q) {
         uint32_t sl = acquire();
-        if (!dead && ntok > 0) qk_fp_half<T, D>(sacc, 0, qa, sl, lane);
-        release();
-        sl = acquire();
         if (!dead && ntok > 0) {
-          qk_fp_half<T, D>(sacc, 2, qa, sl, lane);
+          qk_fp_tile<T, D>(sacc, qa, sl, lane);
           softmax_tile<T, MT, PACK>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
         }
         release();
         sl = acquire();
-        if (!dead && ntok > 0) pv_fp_half<T, D, PACK>(o, 0, pa, pb, sl, lane);
-        release();
-        sl = acquire();
-        if (!dead && ntok > 0) pv_fp_half<T, D, PACK>(o, MT / 2, pa, pb, sl, lane);
+        if (!dead && ntok > 0) pv_fp_tile<T, D, PACK>(o, pa, pb, sl, lane);
         release();
       } else {
-        uint32_t sl = acquire();
+        const uint32_t sl = acquire();
         if (!dead) {
-          qk_q_tile<T, D, BITS>(sacc, qa, sl, lane);
+          qk_q_tile<T, D, BITS>(sacc, qa, sl, sl + TT::Q_TILE_STRIDE, lane);
           softmax_tile<T, MT, PACK>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+          pv_q_tile<T, D, BITS, GROUP, PACK>(o, pa, pb, sl + TT::KC_BYTES, lane);
         }
-        release();
-        sl = acquire();
-        if (!dead) pv_q_tile<T, D, BITS, GROUP, PACK>(o, pa, pb, sl, lane);
         release();
       }
     }
