@@ -96,6 +96,13 @@ template <class T2> __device__ __forceinline__ T2 as_t2(uint32_t x) {
 }
 template <class T2> __device__ __forceinline__ uint32_t as_u32(T2 x) { return *reinterpret_cast<uint32_t*>(&x); }
 
+// (a & b) | c in one LOP3: pulls two codes out of a packed word and plants them in the significands of MAGIC.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;\n" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
 // Dequantize two codes held in the low bits of each 16-bit half of `x` (already OR-ed with MAGIC):
 // value = RNE_T(code * s + z), one correctly rounded fused multiply-add in the execution datatype.
 template <class T> __device__ __forceinline__ uint32_t dequant2(uint32_t x, uint32_t s2, uint32_t z2) {

@@ -155,10 +155,10 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint32_t w = cw[j];
-        const uint32_t b0 = dequant2<T>(((w >> (sh + 0 * BITS)) & MASK) | MG, p0.x, p0.y);
-        const uint32_t b1 = dequant2<T>(((w >> (sh + 1 * BITS)) & MASK) | MG, p0.z, p0.w);
-        const uint32_t b2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, p1.x, p1.y);
-        const uint32_t b3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, p1.z, p1.w);
+        const uint32_t b0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), p0.x, p0.y);
+        const uint32_t b1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), p0.z, p0.w);
+        const uint32_t b2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), p1.x, p1.y);
+        const uint32_t b3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), p1.z, p1.w);
         mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, b0, b1);
         mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, b2, b3);
       }
@@ -212,10 +212,10 @@ __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t 
         const uint4 pr = ks ? pr1 : pr0;
         const uint32_t w = (BITS == 4) ? vw[ii * 2 + ks] : vw[ii];
         const int sh = (BITS == 4) ? 0 : ks * 8;
-        const uint32_t a0 = dequant2<T>(((w >> (sh + 0 * BITS)) & MASK) | MG, pr.x, pr.y);
-        const uint32_t a1 = dequant2<T>(((w >> (sh + 1 * BITS)) & MASK) | MG, pr.x, pr.y);
-        const uint32_t a2 = dequant2<T>(((w >> (sh + 2 * BITS)) & MASK) | MG, pr.z, pr.w);
-        const uint32_t a3 = dequant2<T>(((w >> (sh + 3 * BITS)) & MASK) | MG, pr.z, pr.w);
+        const uint32_t a0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
+        const uint32_t a1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
+        const uint32_t a2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
+        const uint32_t a3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
         mma16816<T>(o[i], a0, a1, a2, a3, pa[ks][0], pa[ks][1]);
         if (!PACK) mma16816<T>(o[i], a0, a1, a2, a3, pb[ks][0], pb[ks][1]);
       }

@@ -167,10 +167,10 @@ __device__ void promote_part(const Geometry& g, int part, const char* __restrict
         const uint32_t w = kc[code_word_off(widx, lane)];
         const uint4 p0 = kp[(c * 2 + 0) * 4 + t], p1 = kp[(c * 2 + 1) * 4 + t];
         uint4 r;
-        r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, p0.x, p0.y);
-        r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, p0.z, p0.w);
-        r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, p1.x, p1.y);
-        r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, p1.z, p1.w);
+        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), p0.x, p0.y);
+        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), p0.z, p0.w);
+        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), p1.x, p1.y);
+        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), p1.z, p1.w);
         kt[v * 32 + lane] = r;
       }
     } else {
@@ -185,10 +185,10 @@ __device__ void promote_part(const Geometry& g, int part, const char* __restrict
         const int gc = (16 * i) / g.group;
         const uint4 pr = vp[(gc * 2 + ks) * 4 + t];
         uint4 r;
-        r.x = dequant2<T>(((w >> (sh + 0 * bits)) & mask) | MG, pr.x, pr.y);
-        r.y = dequant2<T>(((w >> (sh + 1 * bits)) & mask) | MG, pr.x, pr.y);
-        r.z = dequant2<T>(((w >> (sh + 2 * bits)) & mask) | MG, pr.z, pr.w);
-        r.w = dequant2<T>(((w >> (sh + 3 * bits)) & mask) | MG, pr.z, pr.w);
+        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), pr.x, pr.y);
+        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), pr.x, pr.y);
+        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), pr.z, pr.w);
+        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), pr.z, pr.w);
         vt[v * 32 + lane] = r;
       }
     }
