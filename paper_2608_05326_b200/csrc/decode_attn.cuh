@@ -17,9 +17,10 @@
 // memory with conflict-free 16-byte loads.  Waits on the mbarriers are bounded: a wait that runs out
 // records CHECK_COPY_TIMEOUT, the warp stops issuing, drains what it has in flight and returns.
 //
-// Per 32-token tile:  S = Q K^T with the (<= 8) grouped heads on the M side of mma.m16n8k16 and
-// tokens on N, softmax in fp32 in the log2 domain, O^T += V^T P^T with channels on M, tokens on K and
-// heads on N, so the probability fragments feed the second product without any transposition.  The
+// Per 32-token tile:  S^T = K Q^T with tokens on the M side of mma.m16n8k16, channels on K and the (<= 8)
+// grouped heads on N (all 16 rows of every product are useful), softmax in fp32 in the log2 domain,
+// O^T += V^T P^T with channels on M, tokens on K and heads on N; the probability fragments are turned
+// from (token, head) into (head, token) operands by 8x8 register transposes (movmatrix).  The
 // probabilities enter it as a 16-bit value plus its rounding residual; with at most 4 heads per KV
 // head the residuals ride in the unused N columns 4..7 of the same product (PACK), otherwise they take
 // a second product.  A quantized tile is read as packed words, and codes become operands in
@@ -115,52 +116,49 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// ---- S = Q K^T -----------------------------------------------------------------------------------------
+// ---- S^T = K Q^T ---------------------------------------------------------------------------------------
+// Tokens on M (two blocks of 16), channels on K, the (<= 8) grouped heads on N.  s[mt] = {(token g, head 2t),
+// (token g, head 2t+1), (token g+8, head 2t), (token g+8, head 2t+1)} of token block mt.
 // A full-precision key tile (32 tokens) from a ring slot.
 template <class T, int D>
-__device__ __forceinline__ void qk_fp_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
-  constexpr int KG = D / 32;
+__device__ __forceinline__ void qk_fp_tile(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, int lane) {
 #pragma unroll
-  for (int c = 0; c < KG; ++c) {
+  for (int ks = 0; ks < D / 16; ++ks) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint4 kv = lds16(slot + ((j * KG + c) * 32 + lane) * 16);
-      mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, kv.x, kv.y);
-      mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, kv.z, kv.w);
+    for (int mt = 0; mt < 2; ++mt) {
+      const uint4 kv = lds16(slot + ((ks * 2 + mt) * 32 + lane) * 16);
+      mma16816<T>(s[mt], kv.x, kv.y, kv.z, kv.w, qa[ks][0], qa[ks][1]);
     }
   }
 }
 
-// Key part of a quantized tile: codes at `codes`, parameters at `kp`.  The codes of one
-// channel group (two k-steps; four with 2-bit codes) for all four token blocks are one 16-byte vector, so
-// only four code words are live at a time.
+// Key part of a quantized tile: codes at `slot`, parameters at `kp`.  One 16-byte code vector covers two
+// k-steps (four with 2-bit codes) for both token blocks and is fetched right before it is used.
 template <class T, int D, int BITS>
-__device__ __forceinline__ void qk_q_tile(float (&s)[4][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
+__device__ __forceinline__ void qk_q_tile(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
                                           int lane) {
-  constexpr int KG = D / 32;
+  constexpr int KS = D / 16;
   constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
   constexpr uint32_t MG = Tr<T>::MAGIC;
-  constexpr int CPV = (BITS == 4) ? 1 : 2;  // channel groups per code vector
+  constexpr int KPV = (BITS == 4) ? 2 : 4;  // k-steps per code vector
   const int t = lane & 3;
 #pragma unroll
-  for (int v = 0; v < KG / CPV; ++v) {
-    const uint4 cv = lds16(slot + (v * 32 + lane) * 16);  // token blocks j = 0..3
+  for (int v = 0; v < KS / KPV; ++v) {
+    const uint4 cv = lds16(slot + (v * 32 + lane) * 16);
     const uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-    for (int cc = 0; cc < CPV; ++cc) {
-      const int c = v * CPV + cc;
-      const int sh = cc * 8;
-      const uint4 p0 = lds16(kp + ((c * 2 + 0) * 4 + t) * 16);  // k-step 2c:   {s,z} low / high channel octet
-      const uint4 p1 = lds16(kp + ((c * 2 + 1) * 4 + t) * 16);  // k-step 2c+1
+    for (int kk = 0; kk < KPV; ++kk) {
+      const int ks = v * KPV + kk;
+      const uint4 pr = lds16(kp + (ks * 4 + t) * 16);  // {s,z} of channels 2t,2t+1 and of channels 2t+8,2t+9
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t w = cw[j];
-        const uint32_t b0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), p0.x, p0.y);
-        const uint32_t b1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), p0.z, p0.w);
-        const uint32_t b2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), p1.x, p1.y);
-        const uint32_t b3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), p1.z, p1.w);
-        mma16816<T>(s[j], qa[2 * c][0], 0u, qa[2 * c][1], 0u, b0, b1);
-        mma16816<T>(s[j], qa[2 * c + 1][0], 0u, qa[2 * c + 1][1], 0u, b2, b3);
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint32_t w = (BITS == 4) ? cw[kk * 2 + mt] : cw[kk];
+        const int sh = (BITS == 4) ? 0 : mt * 8;
+        const uint32_t a0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
+        const uint32_t a1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
+        const uint32_t a2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
+        const uint32_t a3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
+        mma16816<T>(s[mt], a0, a1, a2, a3, qa[ks][0], qa[ks][1]);
       }
     }
   }
@@ -237,73 +235,94 @@ template <> __device__ __forceinline__ void split_pair<__nv_bfloat16>(float lo, 
   res = as_u32(__floats2bfloat162_rn(lo - __low2float(m), hi - __high2float(m)));
 }
 
-// Online softmax update for one tile; leaves the probability fragments for the PV product in pa / pb.
+// Transpose an 8x8 block of 16-bit elements held one row pair per lane (row = lane / 4, columns
+// 2 * (lane % 4) and +1): turns probabilities indexed (token, head) into the (head, token) operand of PV.
+__device__ __forceinline__ uint32_t transpose8x8(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
+  return y;
+}
+
+// Online softmax update for one tile.  A lane owns heads 2t and 2t+1 (index 0 / 1 of m_run, l_run, wsum)
+// and tokens g, g+8, g+16, g+24 of the tile; the statistics of a head are replicated over the 8 lanes of
+// equal t.  Leaves the probability fragments for the PV product in pa / pb.
 template <class T, int MT, bool PACK>
-__device__ __forceinline__ void softmax_tile(float (&s)[4][4], int ntok, float scale_log2, int lane, float& m_run,
-                                             float& l_run, float& wsum, float (&o)[MT][4], uint32_t (&pa)[2][2],
-                                             uint32_t (&pb)[2][2]) {
-  const int t = lane & 3;
-  float x[4][2];
-  float tmax = -INFINITY;
+__device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float scale_log2, int lane, float (&m_run)[2],
+                                             float (&l_run)[2], float (&wsum)[2], float (&o)[MT][4],
+                                             uint32_t (&pa)[2][2], uint32_t (&pb)[2][2]) {
+  const int g = lane >> 2;
+  float x[2][2][2];  // [token block][row half][head]
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-    for (int e = 0; e < 2; ++e) x[j][e] = s[j][e] * scale_log2;
+    for (int r = 0; r < 2; ++r) {
+      x[mt][r][0] = s[mt][2 * r] * scale_log2;
+      x[mt][r][1] = s[mt][2 * r + 1] * scale_log2;
+    }
   }
   if (ntok < 32) {  // only the open window has unfilled token slots
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        if (8 * j + 2 * t + e >= ntok) x[j][e] = -INFINITY;
+      for (int r = 0; r < 2; ++r) {
+        if (16 * mt + 8 * r + g >= ntok) { x[mt][r][0] = -INFINITY; x[mt][r][1] = -INFINITY; }
       }
     }
   }
+  float alpha[2], p[2][2][2];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) tmax = fmaxf(tmax, fmaxf(x[j][0], x[j][1]));
-  tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-  tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-  const float m_new = fmaxf(m_run, tmax);  // finite: the caller guarantees ntok >= 1
-  const float alpha = ex2(m_run - m_new);
-  float rs = 0.f;
-  float p[4][2];
+  for (int h = 0; h < 2; ++h) {
+    float tmax = fmaxf(fmaxf(x[0][0][h], x[0][1][h]), fmaxf(x[1][0][h], x[1][1][h]));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+    const float m_new = fmaxf(m_run[h], tmax);  // finite: the caller guarantees ntok >= 1
+    alpha[h] = ex2(m_run[h] - m_new);
+    float rs = 0.f;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      p[j][e] = ex2(x[j][e] - m_new);
-      rs += p[j][e];
-    }
-  }
-  rs += __shfl_xor_sync(0xffffffffu, rs, 1);
-  rs += __shfl_xor_sync(0xffffffffu, rs, 2);
-  l_run = l_run * alpha + rs;
-  wsum = wsum * alpha + rs;
-  m_run = m_new;
-  if (__any_sync(0xffffffffu, alpha != 1.f)) {
-    // the accumulators hold O^T: column pair (2t, 2t+1) = heads 2t and 2t+1 (PACK: heads modulo 4),
-    // whose statistics live in the lane quads of those heads
-    const int h0 = PACK ? ((2 * t) & 3) : 2 * t;
-    const float a_lo = __shfl_sync(0xffffffffu, alpha, h0 * 4);
-    const float a_hi = __shfl_sync(0xffffffffu, alpha, (h0 + 1) * 4);
-#pragma unroll
-    for (int i = 0; i < MT; ++i) {
-      o[i][0] *= a_lo; o[i][1] *= a_hi; o[i][2] *= a_lo; o[i][3] *= a_hi;
-    }
-  }
-  split_pair<T>(p[0][0], p[0][1], pa[0][0], pb[0][0]);
-  split_pair<T>(p[1][0], p[1][1], pa[0][1], pb[0][1]);
-  split_pair<T>(p[2][0], p[2][1], pa[1][0], pb[1][0]);
-  split_pair<T>(p[3][0], p[3][1], pa[1][1], pb[1][1]);
-  if (PACK) {
-    // heads live in rows 0..3; the lanes of rows 4..7 feed the residuals of head (row - 4) as extra
-    // N columns of the same product
-#pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
+    for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
-        const uint32_t below = __shfl_sync(0xffffffffu, pb[ks][r], (lane + 16) & 31);
-        if (lane >= 16) pa[ks][r] = below;
+        p[mt][r][h] = ex2(x[mt][r][h] - m_new);
+        rs += p[mt][r][h];
+      }
+    }
+    rs += __shfl_xor_sync(0xffffffffu, rs, 4);
+    rs += __shfl_xor_sync(0xffffffffu, rs, 8);
+    rs += __shfl_xor_sync(0xffffffffu, rs, 16);
+    l_run[h] = l_run[h] * alpha[h] + rs;
+    wsum[h] = wsum[h] * alpha[h] + rs;
+    m_run[h] = m_new;
+  }
+  if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+    // the accumulators hold O^T with the lane's own two heads as its columns; with PACK the columns of
+    // lanes t >= 2 hold the residual products of heads 2(t-2), 2(t-2)+1
+    float a0 = alpha[0], a1 = alpha[1];
+    if (PACK) {
+      const float b0 = __shfl_sync(0xffffffffu, a0, (lane - 2) & 31), b1 = __shfl_sync(0xffffffffu, a1, (lane - 2) & 31);
+      if ((lane & 3) >= 2) { a0 = b0; a1 = b1; }
+    }
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+      o[i][0] *= a0; o[i][1] *= a1; o[i][2] *= a0; o[i][3] *= a1;
+    }
+  }
+  // probabilities as (token, head) pairs -> 16-bit value + residual -> transposed into the B operand
+  // (k = token, n = head): block (mt, r) becomes register r of k-step mt
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      uint32_t main, res;
+      split_pair<T>(p[mt][r][0], p[mt][r][1], main, res);
+      if (PACK) {
+        // heads live in columns 0..3; columns 4..7 carry the residuals of heads 0..3 in the same product
+        const uint32_t left = __shfl_sync(0xffffffffu, res, (lane - 2) & 31);
+        if ((lane & 3) >= 2) main = left;
+        pa[mt][r] = transpose8x8(main);
+      } else {
+        pa[mt][r] = transpose8x8(main);
+        pb[mt][r] = transpose8x8(res);
       }
     }
   }
@@ -342,7 +361,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
     }
   }
 
-  float m_run = -INFINITY, l_run = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // heads 2t and 2t+1
   float o[MT][4];
 #pragma unroll
   for (int i = 0; i < MT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -418,13 +437,13 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
     const uint32_t kind = ex >> ENTRY_KIND_SHIFT;
     const int e = first + ci * stride;
     const int valid = (kind == KIND_OPEN) ? fill : TT::W;
-    float wsum = 0.f;
+    float wsum[2] = {0.f, 0.f};
 #pragma unroll 1
     for (int tile = 0; tile < TILES; ++tile) {
       const int ntok = min(32, valid - 32 * tile);
-      float sacc[4][4];
+      float sacc[2][4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
+      for (int j = 0; j < 2; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
       uint32_t pa[2][2], pb[2][2];
       if (kind != KIND_Q) {
         uint32_t sl = acquire();
@@ -446,8 +465,11 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
         release();
       }
     }
-    if (t == 0 && g < p.G) {
-      p.wrec[((size_t)u * p.Hq + (size_t)hk * p.G + g) * p.EMAX + e] = make_float2(wsum, m_run);
+    if (g == 0) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (2 * t + h < p.G) p.wrec[((size_t)u * p.Hq + (size_t)hk * p.G + 2 * t + h) * p.EMAX + e] = make_float2(wsum[h], m_run[h]);
+      }
     }
   }
   if (dead) {
@@ -460,7 +482,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   constexpr int OSTR = D + 4;
   float* my_o = reinterpret_cast<float*>(smem + wid * NSLOT * TT::SLOT_BYTES);
   float* my_ml = my_o + 8 * OSTR;
-  if (t == 0) { my_ml[g] = m_run; my_ml[8 + g] = l_run; }
+  if (g == 0) { my_ml[2 * t] = m_run[0]; my_ml[2 * t + 1] = m_run[1]; my_ml[8 + 2 * t] = l_run[0]; my_ml[8 + 2 * t + 1] = l_run[1]; }
 #pragma unroll
   for (int i = 0; i < MT; ++i) {
     my_o[(2 * t) * OSTR + 16 * i + g] = o[i][0];

@@ -2,12 +2,12 @@
 //
 // A page is stored in the order in which the decode kernel's tensor-core fragments consume it, so
 // that every warp-wide 16-byte load is one contiguous 512-byte run and lands in registers (or
-// shared memory) already in mma.m16n8k16 operand order.  A 32-token tile of keys is the B operand of
-// S = Q K^T (k = channel, n = token); a 32-token tile of values is the A operand of O^T = V^T P^T
+// shared memory) already in mma.m16n8k16 operand order.  A 32-token tile of keys is the A operand of
+// S^T = K Q^T (m = token, k = channel); a 32-token tile of values is the A operand of O^T = V^T P^T
 // (m = channel, k = token).  With lane = 4*g + t:
 //
-//   key tile, 16-byte vector (j, c), j = token/8, c = channel/32:
-//       lane holds token 8j+g, channels 32c + 16*ks + 8*hi + 2t + e   at element ks*4 + hi*2 + e
+//   key tile, 16-byte vector (ks, mt), ks = channel/16, mt = token/16:
+//       lane holds tokens 16mt + 8*rh + g, channels 16ks + 8*hi + 2t + e at element (hi*2 + rh)*2 + e
 //   value tile, 16-byte vector (i, ks), i = channel/16, ks = token/16:
 //       lane holds channel 16i + 8*ah + g, tokens 16ks + 8*hi + 2t + e at element (hi*2 + ah)*2 + e
 //
@@ -28,11 +28,11 @@ namespace qevict {
 
 // element offset inside a full-precision key tile
 QE_HD int fpk_off(int tk, int ch, int D) {
-  const int j = tk >> 3, g = tk & 7;
-  const int c = ch >> 5, r = ch & 31;
-  const int ks = r >> 4, hi = (r >> 3) & 1, t = (r & 7) >> 1, e = r & 1;
+  (void)D;
+  const int mt = tk >> 4, rh = (tk >> 3) & 1, g = tk & 7;
+  const int ks = ch >> 4, hi = (ch >> 3) & 1, t = (ch & 7) >> 1, e = ch & 1;
   const int lane = g * 4 + t;
-  return ((j * (D >> 5) + c) * 32 + lane) * 8 + ks * 4 + hi * 2 + e;
+  return ((ks * 2 + mt) * 32 + lane) * 8 + (hi * 2 + rh) * 2 + e;
 }
 
 // element offset inside a full-precision value tile
@@ -52,20 +52,18 @@ QE_HD int code_word_off(int widx, int lane) { return ((widx >> 2) * 32 + lane) *
 
 // key codes of a tile
 QE_HD CodePos kcode_pos(int tk, int ch, int D, int bits) {
-  const int j = tk >> 3, g = tk & 7;
-  const int c = ch >> 5, r = ch & 31;
-  const int ks = r >> 4, hi = (r >> 3) & 1, t = (r & 7) >> 1, e = r & 1;
+  (void)D;
+  const int mt = tk >> 4, rh = (tk >> 3) & 1, g = tk & 7;
+  const int ks = ch >> 4, hi = (ch >> 3) & 1, t = (ch & 7) >> 1, e = ch & 1;
   const int lane = g * 4 + t;
-  const int m = ks * 2 + hi;
+  const int a = hi * 2 + rh;
   CodePos p;
-  // word index = channel-group * 4 + token block: one 16-byte vector holds the four token blocks of a
-  // channel group, so the attention kernel fetches the codes of one k-step pair at a time
   if (bits == 4) {
-    p.word = code_word_off(c * 4 + j, lane);
-    p.shift = 4 * m + 16 * e;
+    p.word = code_word_off(ks * 2 + mt, lane);
+    p.shift = 4 * a + 16 * e;
   } else {
-    p.word = code_word_off((c >> 1) * 4 + j, lane);
-    p.shift = 2 * ((c & 1) * 4 + m) + 16 * e;
+    p.word = code_word_off(ks, lane);
+    p.shift = 2 * (mt * 4 + a) + 16 * e;
   }
   return p;
 }
@@ -89,9 +87,8 @@ QE_HD CodePos vcode_pos(int tk, int ch, int bits) {
 
 // key parameters of one group of tokens: element offsets (16-bit units) of scale and zero of channel ch
 QE_HD int kparam_off(int ch, int is_zero) {
-  const int c = ch >> 5, r = ch & 31;
-  const int ks = r >> 4, hi = (r >> 3) & 1, t = (r & 7) >> 1, e = r & 1;
-  return ((c * 2 + ks) * 4 + t) * 8 + (hi * 2 + is_zero) * 2 + e;
+  const int ks = ch >> 4, hi = (ch >> 3) & 1, t = (ch & 7) >> 1, e = ch & 1;
+  return (ks * 4 + t) * 8 + (hi * 2 + is_zero) * 2 + e;
 }
 
 // value parameters of a tile: scale and zero of (token tk, channel group gc)

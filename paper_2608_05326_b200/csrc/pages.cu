@@ -66,7 +66,8 @@ __device__ void quantize_part(const Geometry& g, int part, const T* __restrict__
         for (int el = 0; el < 8; ++el) {
           const int a1 = el >> 2, a2 = (el >> 1) & 1, e = el & 1;
           int tk, ch;
-          if (part == 0) { const int kj = vec / KG, kc = vec - kj * KG; tk = 8 * kj + gg; ch = 32 * kc + 16 * a1 + 8 * a2 + 2 * tt + e; }
+          // element el of a vector = register (a1*2 + a2), half e
+          if (part == 0) { const int kks = vec >> 1, kmt = vec & 1; tk = 16 * kmt + 8 * a2 + gg; ch = 16 * kks + 8 * a1 + 2 * tt + e; }
           else { const int vi = vec >> 1, vks = vec & 1; tk = 16 * vks + 8 * a1 + 2 * tt + e; ch = 16 * vi + 8 * a2 + gg; }
           sx[(tile * 32 + tk) * D + ch] = xe[el];
         }
@@ -127,9 +128,10 @@ __device__ void quantize_part(const Geometry& g, int part, const T* __restrict__
         const int e = k & 1, m = (k >> 1) & 3, sub = k >> 3;
         int tk, ch;
         if (part == 0) {
-          const int j = widx & 3, c = (widx >> 2) * (g.bits == 4 ? 1 : 2) + sub;  // widx = channel group * 4 + j
-          tk = 8 * j + gg;
-          ch = 32 * c + 16 * (m >> 1) + 8 * (m & 1) + 2 * tt + e;
+          const int ks = g.bits == 4 ? (widx >> 1) : widx;
+          const int mt = g.bits == 4 ? (widx & 1) : sub;
+          tk = 16 * mt + 8 * (m & 1) + gg;
+          ch = 16 * ks + 8 * (m >> 1) + 2 * tt + e;
         } else {
           const int i = g.bits == 4 ? (widx >> 1) : widx;
           const int ks = g.bits == 4 ? (widx & 1) : sub;
@@ -160,17 +162,17 @@ __device__ void promote_part(const Geometry& g, int part, const char* __restrict
       const uint32_t* kc = reinterpret_cast<const uint32_t*>(tb);
       const uint4* kp = reinterpret_cast<const uint4*>(qb + g.q_kp_off + (size_t)((tile * 32) / g.group) * g.q_kp_bytes);
       uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
-      for (int v = wid; v < 4 * KG; v += nwarps) {  // key vectors (j, c)
-        const int j = v / KG, c = v - j * KG;
-        const int widx = (bits == 4 ? c : (c >> 1)) * 4 + j;
-        const int sh = bits == 4 ? 0 : (c & 1) * 8;
+      for (int v = wid; v < 2 * (D / 16); v += nwarps) {  // key vectors (ks, mt)
+        const int ks = v >> 1, mt = v & 1;
+        const int widx = bits == 4 ? ks * 2 + mt : ks;
+        const int sh = bits == 4 ? 0 : mt * 8;
         const uint32_t w = kc[code_word_off(widx, lane)];
-        const uint4 p0 = kp[(c * 2 + 0) * 4 + t], p1 = kp[(c * 2 + 1) * 4 + t];
+        const uint4 pr = kp[ks * 4 + t];
         uint4 r;
-        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), p0.x, p0.y);
-        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), p0.z, p0.w);
-        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), p1.x, p1.y);
-        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), p1.z, p1.w);
+        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), pr.x, pr.y);
+        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), pr.x, pr.y);
+        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), pr.z, pr.w);
+        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), pr.z, pr.w);
         kt[v * 32 + lane] = r;
       }
     } else {
