@@ -346,34 +346,22 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   }
   __syncwarp();
 
-  // query fragments: row g of the A operand = head hk*G + g (rows >= G are zero)
-  uint32_t qa[KS][2];
-  {
-    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)ul * p.Hq + (size_t)hk * p.G + g) * D;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      if (g < p.G) {
-        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * t);
-        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * t);
-      } else {
-        qa[ks][0] = 0u; qa[ks][1] = 0u;
-      }
-    }
-  }
-
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // heads 2t and 2t+1
   float o[MT][4];
 #pragma unroll
   for (int i = 0; i < MT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
 
-  const int n_live = p.n_live[u];
-  const int fill = p.open_fill[u];
+  // The work-list entries are fetched without waiting for the list length (the slots exist up to EMAX;
+  // what lies past the end is masked afterwards), so start-up costs one global round trip, not two.
   const int stride = p.S * DECODE_WARPS;
   const int first = s * DECODE_WARPS + wid;
+  uint2 my_ent = make_uint2(0u, 0u);
+  if (first + lane * stride < p.EMAX) my_ent = p.entries[(size_t)u * p.EMAX + first + (size_t)lane * stride];
+  const int n_live = p.n_live[u];
+  const int fill = p.open_fill[u];
   // this warp's entries, one per lane (the host picks S so that a warp never owns more than 32)
   const int my_n = first < n_live ? min(32, (n_live - first + stride - 1) / stride) : 0;
-  uint2 my_ent = make_uint2(0u, 0u);
-  if (lane < my_n) my_ent = p.entries[(size_t)u * p.EMAX + first + (size_t)lane * stride];
+  if (lane >= my_n) my_ent = make_uint2(0u, 0u);
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
   // pieces per tile: full precision = 2 (key tile, value tile), quantized = 1 (the whole tile)
@@ -430,6 +418,22 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   };
 #pragma unroll 1
   for (int i = 0; i < NSLOT; ++i) issue_next();
+
+  // query fragments: row g of the A operand = head hk*G + g (rows >= G are zero)
+  uint32_t qa[KS][2];
+  {
+    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)ul * p.Hq + (size_t)hk * p.G + g) * D;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      if (g < p.G) {
+        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * t);
+        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * t);
+      } else {
+        qa[ks][0] = 0u; qa[ks][1] = 0u;
+      }
+    }
+  }
+
 
 #pragma unroll 1
   for (int ci = 0; ci < my_n; ++ci) {
