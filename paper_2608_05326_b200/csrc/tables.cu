@@ -216,7 +216,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int32_t* oq = ofp + g.PF;                                                  // [PQ]
   int32_t* free_fp = oq + g.PQ;                                              // [PF] free page ids, ascending
   int32_t* free_q = free_fp + g.PF;                                          // [PQ]
-  int32_t* scratch = free_q + g.PQ;                                          // [40]
+  int32_t* reader = free_q + g.PQ;                                           // [PF] quantization that reads a page
+  int32_t* flist = reader + g.PF;                                            // [EMAX] Full, then Quantized candidates
+  int32_t* scratch = flist + g.EMAX;                                         // [40]
   uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 40);                 // [sort_cap] state before
   uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
   uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
@@ -327,11 +329,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
                                      [&](int pg, int k) { free_q[k] = pg; });
 
   // first demotions need a quantized page, ascending window index.  reader[p] = index of the
-  // quantization that reads full-precision page p (free_fp is not needed before the next step, reuse
-  // free_q's neighbour array for the map)
+  // quantization that reads full-precision page p
   const int qcap = g.PF + g.Kq;
   int4* quant_list = a.st.quant_list + (size_t)u * qcap;
-  int32_t* reader = reinterpret_cast<int32_t*>(keys);  // [PF]; the sort keys are no longer needed
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) reader[i] = -1;
   __syncthreads();
   const int n_q_need = block_compact(
@@ -390,16 +390,29 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) q_owner[i] = oq[i];
   __syncthreads();
 
-  // ---- decode work list: Full.., Quantized.., open window last ---------------------------------------
+  // ---- decode work list: Full and Quantized windows (each ascending) interleaved in proportion, so that
+  // every stretch of the list -- and therefore every warp of the attention kernel at every moment --
+  // sees the same mix of 16-bit and low-bit pages; open window last -------------------------------------
   uint2* entries = a.st.entries + (size_t)u * g.EMAX;
   const int n_f = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_FULL; },
-                                [&](int c, int k) {
-                                  if (k < g.EMAX) entries[k] = make_uint2((uint32_t)cw[c] | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)cfp[c]);
-                                });
+                                [&](int c, int k) { if (k < g.EMAX) flist[k] = c; });
+  int32_t* qlist = flist + n_f;
   const int n_q = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_QUANT; },
-                                [&](int c, int k) {
-                                  if (n_f + k < g.EMAX) entries[n_f + k] = make_uint2((uint32_t)cw[c] | (KIND_Q << ENTRY_KIND_SHIFT), (uint32_t)cq[c]);
-                                });
+                                [&](int c, int k) { if (n_f + k < g.EMAX) qlist[k] = c; });
+  {
+    const int n = n_f + n_q;
+    for (int k = tid; k < n && k < g.EMAX; k += ROUTE_THREADS) {
+      const int cf = (int)(((long long)k * n_f) / n);                       // Full windows before position k
+      const bool is_f = (int)(((long long)(k + 1) * n_f) / n) > cf;
+      if (is_f) {
+        const int c = flist[cf];
+        entries[k] = make_uint2((uint32_t)cw[c] | (KIND_FP << ENTRY_KIND_SHIFT), (uint32_t)cfp[c]);
+      } else {
+        const int c = qlist[k - cf];
+        entries[k] = make_uint2((uint32_t)cw[c] | (KIND_Q << ENTRY_KIND_SHIFT), (uint32_t)cq[c]);
+      }
+    }
+  }
   if (tid == 0) {
     int n = n_f + n_q;
     if (ow >= 0) {
@@ -433,7 +446,7 @@ __global__ void export_mass_kernel(const KernelArgs a, int u, float* __restrict_
 }  // namespace
 
 size_t route_smem_bytes(const Geometry& g, int sort_cap) {
-  return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(2 * (g.PF + g.PQ) + 40) * 4 + 16;
+  return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 40) * 4 + 16;
 }
 
 cudaError_t route_prepare(size_t max_smem) {
