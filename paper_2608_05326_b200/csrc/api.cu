@@ -136,12 +136,10 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.open_fill = (int32_t*)take(U * 4);
   s.n_live = (int32_t*)take(U * 4);
   s.entries = (uint2*)take(U * g.EMAX * 8);
-  s.quant_list = (int4*)take(U * (size_t)(g.PF + g.Kq) * 16);
-  s.promote_list = (int4*)take(U * (size_t)(g.Kf > 0 ? g.Kf : 1) * 16);
   s.copy_list = (int4*)take(U * (size_t)(g.Kf > 0 ? g.Kf : 1) * 16);
-  s.n_quant = (int32_t*)take(U * 4);
-  s.n_promote = (int32_t*)take(U * 4);
   s.n_copy = (int32_t*)take(U * 4);
+  s.mig_queue = (int4*)take(U * (size_t)(g.PF + g.Kq + g.Kf) * 32);
+  s.mig_count = (int32_t*)take((size_t)g.n_layers * 2 * 4);
   s.counters = (unsigned long long*)take(U * 4 * 8);
   s.o_part = (float*)take(U * g.Hq * (size_t)MAX_SPLITS * g.D * 4);
   s.ml = (float*)take(U * g.Hq * (size_t)MAX_SPLITS * 2 * 4);
@@ -338,9 +336,8 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
     if (e == cudaSuccess) e = cudaMemset(h->st.open_window, 0xFF, U * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.open_fill, 0, U * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.n_live, 0, U * 4);
-    if (e == cudaSuccess) e = cudaMemset(h->st.n_quant, 0, U * 4);
-    if (e == cudaSuccess) e = cudaMemset(h->st.n_promote, 0, U * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.n_copy, 0, U * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.mig_count, 0, (size_t)g.n_layers * 2 * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.counters, 0, U * 32);
     if (e == cudaSuccess) e = cudaMemset(h->st.mass_e, 0, U * (size_t)g.EMAX * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.status, 0, 256);

@@ -59,12 +59,11 @@ struct State {
   int32_t* open_fill;   // [1]
   int32_t* n_live;      // [1] entries in the work list
   uint2* entries;       // [EMAX] {window | kind << 28, page}
-  int4* quant_list;     // [PF + Kq] {window, src fp page (-1: prompt), dst q page, 0}
-  int4* promote_list;   // [Kf] {window, src q page, dst fp page, 0}
   int4* copy_list;      // [Kf] {window, dst fp page, 0, 0} (prefill only)
-  int32_t* n_quant;
-  int32_t* n_promote;
   int32_t* n_copy;
+  int4* mig_queue;      // [PF + Kq + Kf] records of two int4 per unit; the units of one call share the run
+                        // that starts at its first unit (record format: see the migration kernel)
+  int32_t* mig_count;   // [n_layers][2] (not per unit) {entries queued by the routing event, CTAs finished}
   unsigned long long* counters;  // [4] promotions, quantizations, reactivations, deletions
   char* fp_pool;        // [PF] pages
   char* q_pool;         // [PQ] pages

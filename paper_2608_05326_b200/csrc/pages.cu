@@ -14,7 +14,7 @@ namespace qevict {
 namespace {
 
 constexpr int PAGE_THREADS = 128;
-constexpr int MIGRATE_THREADS = 256;
+constexpr int MIGRATE_THREADS = 128;
 
 template <class T>
 __device__ __forceinline__ void group_params(float mn, float mx, int qmax, T& s_out, T& z_out, float& s_f, bool& bad) {
@@ -28,212 +28,312 @@ __device__ __forceinline__ void group_params(float mn, float mx, int qmax, T& s_
   s_f = s;
 }
 
-__device__ __forceinline__ uint32_t quant_code(float x, float z, float s, int qmax, bool bad) {
+// code = clamp(rint((x - zero) / scale)) on the IEEE float32 quotient.  The quotient is first estimated with
+// the group's reciprocal (error of a few 1e-6 at most for codes up to 15); only when the estimate lies
+// within 1e-3 of a rounding boundary (or is not finite) is the exact division carried out, so the result
+// is the exact-division result in every case.
+__device__ __forceinline__ uint32_t quant_code(float x, float z, float s, float inv_s, int qmax, bool bad) {
   if (bad) return 0u;
-  const float tq = rintf(__fdiv_rn(__fsub_rn(x, z), s));
-  const int c = (int)fminf(fmaxf(tq, 0.f), (float)qmax);
+  const float d = __fsub_rn(x, z);
+  float r = rintf(__fmul_rn(d, inv_s));
+  if (!(fabsf(fabsf(__fmul_rn(d, inv_s) - r) - 0.5f) >= 1e-3f)) r = rintf(__fdiv_rn(d, s));
+  const int c = (int)fminf(fmaxf(r, 0.f), (float)qmax);
   return (uint32_t)c;
 }
 
-// ---- quantize one half (keys or values) of one window of one KV head ------------------------------------
-// Shared memory: the half in plain [W][D] order and its parameters as floats.  Every thread then builds
-// whole 32-bit code words (no atomics) and stores them straight into the page.
+// ---- migration tasks ---------------------------------------------------------------------------------
+// Everything works in the fragment coordinates of the pages.  The members of a quantization group sit in
+// the registers of the 8 lanes that share lane % 4, so a group's minimum and maximum are a few local
+// comparisons and three shuffles, and every lane holds exactly the elements whose codes make up its own
+// 32-bit code words.  A task is one warp's share of one half (keys or values) of a window of one KV head:
+//   keys:   (block of `group` tokens, ks)      -> 16-byte vectors (ks, mt = 0, 1) of the block's tiles
+//   values: (tile, channel group gc, ks)       -> 16-byte vectors (i, ks), i over the group's channels
+// and the promotion task with the same coordinates writes exactly the vectors the quantization task reads
+// (same lanes, same addresses), so a linked pair needs no ordering beyond program order inside the warp.
 template <class T>
-__device__ void quantize_part(const Geometry& g, int part, const T* __restrict__ rows /* prompt rows or null */,
-                              const char* __restrict__ fp_head /* source page head or null */, char* qb,
-                              unsigned char* smem_raw) {
-  const int tid = threadIdx.x, W = g.W, D = g.D, G = g.group, qmax = (1 << g.bits) - 1;
-  T* sx = reinterpret_cast<T*>(smem_raw);                       // [W][D]
-  float* sf = reinterpret_cast<float*>(sx + W * D);             // scale (or -1 if the group is degenerate)
-  float* zf = sf + (part == 0 ? (W / G) * D : W * (D / G));     // zero
-  const int KG = D / 32;
+__device__ __forceinline__ void unpack2(uint32_t u, float& lo, float& hi) {
+  const typename Tr<T>::T2 h2 = *reinterpret_cast<const typename Tr<T>::T2*>(&u);
+  lo = Tr<T>::to_float(h2.x);
+  hi = Tr<T>::to_float(h2.y);
+}
 
-  // ---- stage the half in plain order ---------------------------------------------------------------
-  if (rows) {
-    const uint4* r4 = reinterpret_cast<const uint4*>(rows);
-    for (int i = tid; i < W * D / 8; i += MIGRATE_THREADS) reinterpret_cast<uint4*>(sx)[i] = r4[i];
-  } else {
-    // the page is fragment-major: 16-byte loads (many in flight), each vector scattered to plain positions
-    const int nvec = 32 * D / 8;
-    for (int tile = 0; tile < g.tiles; ++tile) {
-      const uint4* src = reinterpret_cast<const uint4*>(fp_head + (size_t)tile * 2 * g.fp_tile_bytes + (part ? g.fp_tile_bytes : 0));
-#pragma unroll 4
-      for (int v = tid; v < nvec; v += MIGRATE_THREADS) {
-        const uint4 x = src[v];
-        const int ln = v & 31, vec = v >> 5, gg = ln >> 2, tt = ln & 3;
-        const T* xe = reinterpret_cast<const T*>(&x);
+template <class T>
+__device__ __forceinline__ uint32_t pack2(T lo, T hi) {
+  typename Tr<T>::T2 h2;
+  h2.x = lo; h2.y = hi;
+  return *reinterpret_cast<const uint32_t*>(&h2);
+}
+
+// slot k = hi * 2 + e of a lane: folds the registers of one vector (register a = hi * 2 + x) into the
+// running minimum / maximum of the slots
+template <class T>
+__device__ __forceinline__ void fold_minmax(const uint4& v, float (&mn)[4], float (&mx)[4]) {
+  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int el = 0; el < 8; ++el) {
-          const int a1 = el >> 2, a2 = (el >> 1) & 1, e = el & 1;
-          int tk, ch;
-          // element el of a vector = register (a1*2 + a2), half e
-          if (part == 0) { const int kks = vec >> 1, kmt = vec & 1; tk = 16 * kmt + 8 * a2 + gg; ch = 16 * kks + 8 * a1 + 2 * tt + e; }
-          else { const int vi = vec >> 1, vks = vec & 1; tk = 16 * vks + 8 * a1 + 2 * tt + e; ch = 16 * vi + 8 * a2 + gg; }
-          sx[(tile * 32 + tk) * D + ch] = xe[el];
-        }
-      }
-    }
-  }
-  __syncthreads();
-
-  // ---- parameters ----------------------------------------------------------------------------------
-  if (part == 0) {  // keys: one group per (block of G tokens, channel)
-    for (int i = tid; i < (W / G) * D; i += MIGRATE_THREADS) {
-      const int blk = i / D, ch = i - blk * D;
-      float mn = INFINITY, mx = -INFINITY;
-      for (int tk = blk * G; tk < (blk + 1) * G; ++tk) {
-        const float x = Tr<T>::to_float(sx[tk * D + ch]);
-        mn = fminf(mn, x); mx = fmaxf(mx, x);
-      }
-      T st, zt; float s; bool bad;
-      group_params<T>(mn, mx, qmax, st, zt, s, bad);
-      sf[i] = bad ? -1.f : s;
-      zf[i] = mn;
-      T* kp = reinterpret_cast<T*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes);
-      kp[kparam_off(ch, 0)] = st;
-      kp[kparam_off(ch, 1)] = zt;
-    }
-  } else {  // values: one group per (token, block of G channels)
-    const int ng = D / G;
-    for (int i = tid; i < W * ng; i += MIGRATE_THREADS) {
-      const int gc = i / W, tk = i - gc * W;  // consecutive threads take consecutive tokens
-      float mn = INFINITY, mx = -INFINITY;
-      for (int k = 0; k < G; ++k) {
-        const int ch = gc * G + ((k + tk) & (G - 1));  // rotated start: spreads the threads over the banks
-        const float x = Tr<T>::to_float(sx[tk * D + ch]);
-        mn = fminf(mn, x); mx = fmaxf(mx, x);
-      }
-      T st, zt; float s; bool bad;
-      group_params<T>(mn, mx, qmax, st, zt, s, bad);
-      sf[tk * ng + gc] = bad ? -1.f : s;
-      zf[tk * ng + gc] = mn;
-      T* vp = reinterpret_cast<T*>(qb + (size_t)(tk >> 5) * g.q_tile_stride + g.q_kc_bytes + g.q_vc_bytes);
-      vp[vparam_off(tk & 31, gc, 0)] = st;
-      vp[vparam_off(tk & 31, gc, 1)] = zt;
-    }
-  }
-  __syncthreads();
-
-  // ---- codes: one 32-bit word (8 or 16 codes) per thread and iteration ----------------------------------
-  const int words_per_tile = g.q_kc_bytes / 4;
-  const int cpw = 32 / g.bits;  // codes per word
-  for (int tile = 0; tile < g.tiles; ++tile) {
-    uint32_t* dstw = reinterpret_cast<uint32_t*>(qb + (size_t)tile * g.q_tile_stride + (part ? g.q_kc_bytes : 0));
-    for (int wo = tid; wo < words_per_tile; wo += MIGRATE_THREADS) {
-      // word offset -> (word index of the lane, lane)
-      const int q4 = wo >> 2, ln = q4 & 31, widx = (q4 >> 5) * 4 + (wo & 3), gg = ln >> 2, tt = ln & 3;
-      uint32_t word = 0u;
-      for (int k = 0; k < cpw; ++k) {
-        // slot k of the word: sub-word (2-bit only), register m / a, element e
-        const int e = k & 1, m = (k >> 1) & 3, sub = k >> 3;
-        int tk, ch;
-        if (part == 0) {
-          const int ks = g.bits == 4 ? (widx >> 1) : widx;
-          const int mt = g.bits == 4 ? (widx & 1) : sub;
-          tk = 16 * mt + 8 * (m & 1) + gg;
-          ch = 16 * ks + 8 * (m >> 1) + 2 * tt + e;
-        } else {
-          const int i = g.bits == 4 ? (widx >> 1) : widx;
-          const int ks = g.bits == 4 ? (widx & 1) : sub;
-          tk = 16 * ks + 8 * (m >> 1) + 2 * tt + e;
-          ch = 16 * i + 8 * (m & 1) + gg;
-        }
-        const int row = tile * 32 + tk;
-        const int pi = part == 0 ? (row / G) * D + ch : row * (D / G) + ch / G;
-        const float s = sf[pi];
-        const uint32_t code = quant_code(Tr<T>::to_float(sx[row * D + ch]), zf[pi], s, qmax, s < 0.f);
-        word |= code << (g.bits * (sub * 4 + m) + 16 * e);
-      }
-      dstw[wo] = word;
+  for (int a = 0; a < 4; ++a) {
+    float f[2];
+    unpack2<T>(r[a], f[0], f[1]);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int k = (a >> 1) * 2 + e;
+      mn[k] = fminf(mn[k], f[e]);
+      mx[k] = fmaxf(mx[k], f[e]);
     }
   }
 }
 
-// ---- dequantize one half of one window of one KV head into a full-precision page -----------------------
-// Produces exactly the operand registers the decode kernel forms in flight.
+// codes of one vector: returns sum over (a, e) of code << (bits * a + 16 * e)
 template <class T>
-__device__ void promote_part(const Geometry& g, int part, const char* __restrict__ qb, char* fb) {
-  const int D = g.D, KG = D / 32, MT = D / 16, bits = g.bits;
+__device__ __forceinline__ uint32_t vector_codes(const uint4& v, const float (&mn)[4], const float (&sc)[4],
+                                                 const float (&inv)[4], const bool (&bad)[4], int qmax, int bits) {
+  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+  uint32_t w = 0u;
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    float f[2];
+    unpack2<T>(r[a], f[0], f[1]);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int k = (a >> 1) * 2 + e;
+      w |= quant_code(f[e], mn[k], sc[k], inv[k], qmax, bad[k]) << (bits * a + 16 * e);
+    }
+  }
+  return w;
+}
+
+// Minimum / maximum of the four slots over the 8 lanes of equal lane % 4, then the group parameters of
+// each slot; lanes 0..3 store the 16-byte parameter record (layout (hi * 2 + is_zero) * 2 + e).
+template <class T>
+__device__ __forceinline__ void slot_params(float (&mn)[4], float (&mx)[4], int qmax, float (&sc)[4], float (&inv)[4],
+                                            bool (&bad)[4], uint4* param_dst, int lane) {
+#pragma unroll
+  for (int o = 4; o <= 16; o <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      mn[k] = fminf(mn[k], __shfl_xor_sync(0xffffffffu, mn[k], o));
+      mx[k] = fmaxf(mx[k], __shfl_xor_sync(0xffffffffu, mx[k], o));
+    }
+  }
+  T st[4], zt[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    group_params<T>(mn[k], mx[k], qmax, st[k], zt[k], sc[k], bad[k]);
+    inv[k] = __frcp_rn(sc[k]);
+  }
+  if (lane < 4) *param_dst = make_uint4(pack2<T>(st[0], st[1]), pack2<T>(zt[0], zt[1]), pack2<T>(st[2], st[3]), pack2<T>(zt[2], zt[3]));
+}
+
+// two codes of a pair -> two dequantized values (the registers the decode kernel forms in flight)
+template <class T>
+__device__ __forceinline__ uint4 dequant_vector(uint32_t w, int sh, int bits, const uint4& pr) {
   const uint32_t mask = bits == 4 ? 0x000F000Fu : 0x00030003u, MG = Tr<T>::MAGIC;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, t = lane & 3, nwarps = MIGRATE_THREADS / 32;
-  for (int tile = 0; tile < g.tiles; ++tile) {
-    const char* tb = qb + (size_t)tile * g.q_tile_stride;
-    if (part == 0) {
-      const uint32_t* kc = reinterpret_cast<const uint32_t*>(tb);
-      const uint4* kp = reinterpret_cast<const uint4*>(qb + g.q_kp_off + (size_t)((tile * 32) / g.group) * g.q_kp_bytes);
-      uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
-      for (int v = wid; v < 2 * (D / 16); v += nwarps) {  // key vectors (ks, mt)
-        const int ks = v >> 1, mt = v & 1;
-        const int widx = bits == 4 ? ks * 2 + mt : ks;
-        const int sh = bits == 4 ? 0 : mt * 8;
-        const uint32_t w = kc[code_word_off(widx, lane)];
-        const uint4 pr = kp[ks * 4 + t];
-        uint4 r;
-        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), pr.x, pr.y);
-        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), pr.x, pr.y);
-        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), pr.z, pr.w);
-        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), pr.z, pr.w);
-        kt[v * 32 + lane] = r;
+  uint4 r;
+  r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), pr.x, pr.y);
+  r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), pr.x, pr.y);
+  r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), pr.z, pr.w);
+  r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), pr.z, pr.w);
+  return r;
+}
+
+// ---- keys: task (blk, ks) -----------------------------------------------------------------------------
+template <class T>
+__device__ __forceinline__ void quant_key_task(const Geometry& g, int blk, int ks, const T* __restrict__ rows,
+                                               const char* __restrict__ fp_head, char* qb, int lane) {
+  const int D = g.D, bits = g.bits, qmax = (1 << bits) - 1, tpg = g.group >> 5, gq = lane >> 2, t = lane & 3;
+  uint4 x[2][2];  // [tile of the group][mt]; register a = hi * 2 + rh, halves e
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl) {
+    if (tl >= tpg) continue;
+    const int tile = blk * tpg + tl;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      if (fp_head) {
+        x[tl][mt] = reinterpret_cast<const uint4*>(fp_head + (size_t)tile * 2 * g.fp_tile_bytes)[(ks * 2 + mt) * 32 + lane];
+      } else {
+        uint32_t r[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          const int tk = tile * 32 + 16 * mt + 8 * (a & 1) + gq, ch = 16 * ks + 8 * (a >> 1) + 2 * t;
+          r[a] = *reinterpret_cast<const uint32_t*>(rows + (size_t)tk * D + ch);
+        }
+        x[tl][mt] = make_uint4(r[0], r[1], r[2], r[3]);
       }
+    }
+  }
+  float mn[4] = {INFINITY, INFINITY, INFINITY, INFINITY}, mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl) {
+    if (tl >= tpg) continue;
+    fold_minmax<T>(x[tl][0], mn, mx);
+    fold_minmax<T>(x[tl][1], mn, mx);
+  }
+  float sc[4], inv[4]; bool bad[4];
+  slot_params<T>(mn, mx, qmax, sc, inv, bad, reinterpret_cast<uint4*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes) + ks * 4 + t, lane);
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl) {
+    if (tl >= tpg) continue;
+    uint32_t* dstw = reinterpret_cast<uint32_t*>(qb + (size_t)(blk * tpg + tl) * g.q_tile_stride);
+    const uint32_t w0 = vector_codes<T>(x[tl][0], mn, sc, inv, bad, qmax, bits);
+    const uint32_t w1 = vector_codes<T>(x[tl][1], mn, sc, inv, bad, qmax, bits);
+    if (bits == 4) {
+      dstw[code_word_off(ks * 2 + 0, lane)] = w0;
+      dstw[code_word_off(ks * 2 + 1, lane)] = w1;
     } else {
-      const uint32_t* vc = reinterpret_cast<const uint32_t*>(tb + g.q_kc_bytes);
-      const uint4* vp = reinterpret_cast<const uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes);
-      uint4* vt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes);
-      for (int v = wid; v < 2 * MT; v += nwarps) {  // value vectors (i, ks)
-        const int i = v >> 1, ks = v & 1;
-        const int widx = bits == 4 ? i * 2 + ks : i;
-        const int sh = bits == 4 ? 0 : ks * 8;
-        const uint32_t w = vc[code_word_off(widx, lane)];
-        const int gc = (16 * i) / g.group;
-        const uint4 pr = vp[(gc * 2 + ks) * 4 + t];
-        uint4 r;
-        r.x = dequant2<T>(and_or(w >> (sh + 0 * bits), mask, MG), pr.x, pr.y);
-        r.y = dequant2<T>(and_or(w >> (sh + 1 * bits), mask, MG), pr.x, pr.y);
-        r.z = dequant2<T>(and_or(w >> (sh + 2 * bits), mask, MG), pr.z, pr.w);
-        r.w = dequant2<T>(and_or(w >> (sh + 3 * bits), mask, MG), pr.z, pr.w);
-        vt[v * 32 + lane] = r;
-      }
+      dstw[code_word_off(ks, lane)] = w0 | (w1 << 8);
     }
   }
 }
 
-// Migration kernel.  CTA = (list slot, KV head x {keys, values}, unit); it walks the unit's quantization
-// list and then the promotions nobody else handles.  A promotion whose new full-precision page is the
-// page a quantization of the same event reads from is linked to that quantization and runs in the same
-// CTA right after it, so no page is overwritten before it has been read.
+template <class T>
+__device__ __forceinline__ void promote_key_task(const Geometry& g, int blk, int ks, const char* __restrict__ qb, char* fb,
+                                                 int lane) {
+  const int bits = g.bits, tpg = g.group >> 5, t = lane & 3;
+  const uint4 pr = reinterpret_cast<const uint4*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes)[ks * 4 + t];
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl) {
+    if (tl >= tpg) continue;
+    const int tile = blk * tpg + tl;
+    const uint32_t* kc = reinterpret_cast<const uint32_t*>(qb + (size_t)tile * g.q_tile_stride);
+    uint4* kt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes);
+    if (bits == 4) {
+      const uint32_t w0 = kc[code_word_off(ks * 2 + 0, lane)], w1 = kc[code_word_off(ks * 2 + 1, lane)];
+      kt[(ks * 2 + 0) * 32 + lane] = dequant_vector<T>(w0, 0, 4, pr);
+      kt[(ks * 2 + 1) * 32 + lane] = dequant_vector<T>(w1, 0, 4, pr);
+    } else {
+      const uint32_t w = kc[code_word_off(ks, lane)];
+      kt[(ks * 2 + 0) * 32 + lane] = dequant_vector<T>(w, 0, 2, pr);
+      kt[(ks * 2 + 1) * 32 + lane] = dequant_vector<T>(w, 8, 2, pr);
+    }
+  }
+}
+
+// ---- values: task (tile, gc, ks) ------------------------------------------------------------------------
+template <class T>
+__device__ __forceinline__ void quant_value_task(const Geometry& g, int tile, int gc, int ks, const T* __restrict__ rows,
+                                                 const char* __restrict__ fp_head, char* qb, int lane) {
+  const int D = g.D, bits = g.bits, qmax = (1 << bits) - 1, ipg = g.group >> 4, gq = lane >> 2, t = lane & 3;
+  uint4 x[4];  // [i inside the group]; register a = hi * 2 + ah, halves e
+#pragma unroll
+  for (int ii = 0; ii < 4; ++ii) {
+    if (ii >= ipg) continue;
+    const int i = gc * ipg + ii;
+    if (fp_head) {
+      x[ii] = reinterpret_cast<const uint4*>(fp_head + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes)[(i * 2 + ks) * 32 + lane];
+    } else {
+      uint32_t r[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int tk = tile * 32 + 16 * ks + 8 * (a >> 1) + 2 * t, ch = 16 * i + 8 * (a & 1) + gq;
+        r[a] = pack2<T>(rows[(size_t)tk * D + ch], rows[(size_t)(tk + 1) * D + ch]);
+      }
+      x[ii] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+  }
+  float mn[4] = {INFINITY, INFINITY, INFINITY, INFINITY}, mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int ii = 0; ii < 4; ++ii) {
+    if (ii >= ipg) continue;
+    fold_minmax<T>(x[ii], mn, mx);
+  }
+  float sc[4], inv[4]; bool bad[4];
+  char* tb = qb + (size_t)tile * g.q_tile_stride;
+  slot_params<T>(mn, mx, qmax, sc, inv, bad, reinterpret_cast<uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes) + (gc * 2 + ks) * 4 + t, lane);
+  uint32_t* dstw = reinterpret_cast<uint32_t*>(tb + g.q_kc_bytes);
+#pragma unroll
+  for (int ii = 0; ii < 4; ++ii) {
+    if (ii >= ipg) continue;
+    const int i = gc * ipg + ii;
+    const uint32_t w = vector_codes<T>(x[ii], mn, sc, inv, bad, qmax, bits);
+    if (bits == 4) {
+      dstw[code_word_off(i * 2 + ks, lane)] = w;
+    } else {
+      // a 2-bit word holds both token halves (the ks = 0 byte of each 16-bit half below the ks = 1 byte);
+      // the two tasks that share a word write disjoint bytes
+      unsigned char* b = reinterpret_cast<unsigned char*>(dstw + code_word_off(i, lane));
+      b[ks] = (unsigned char)(w & 0xFFu);
+      b[2 + ks] = (unsigned char)((w >> 16) & 0xFFu);
+    }
+  }
+}
+
+template <class T>
+__device__ __forceinline__ void promote_value_task(const Geometry& g, int tile, int gc, int ks, const char* __restrict__ qb,
+                                                   char* fb, int lane) {
+  const int bits = g.bits, ipg = g.group >> 4, t = lane & 3;
+  const char* tb = qb + (size_t)tile * g.q_tile_stride;
+  const uint32_t* vc = reinterpret_cast<const uint32_t*>(tb + g.q_kc_bytes);
+  const uint4 pr = reinterpret_cast<const uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes)[(gc * 2 + ks) * 4 + t];
+  uint4* vt = reinterpret_cast<uint4*>(fb + (size_t)tile * 2 * g.fp_tile_bytes + g.fp_tile_bytes);
+#pragma unroll
+  for (int ii = 0; ii < 4; ++ii) {
+    if (ii >= ipg) continue;
+    const int i = gc * ipg + ii;
+    const uint32_t w = vc[code_word_off(bits == 4 ? i * 2 + ks : i, lane)];
+    vt[(i * 2 + ks) * 32 + lane] = dequant_vector<T>(w, bits == 4 ? 0 : ks * 8, bits, pr);
+  }
+}
+
+// Migration kernel.  The routing event leaves one queue of 32-byte records for the whole call:
+//   {unit, kind, window, src} {dst, link, -, -}
+//   kind 0  first demotion: quantize full-precision page src (-1: the prompt rows of `window`) into
+//           quantized page dst; link >= 0: afterwards dequantize quantized page `link` into page src
+//           (a promotion of the same event that was handed the page being vacated)
+//   kind 1  promotion: dequantize quantized page src into full-precision page dst
+//   kind 2  nothing (a promotion that is linked to a demotion)
+// Every warp of a fixed-size grid takes (record, KV head, keys | values, task) tuples round-robin, so the
+// launch costs the same whether one unit or all of them migrate something, and the tasks are independent
+// (see above), so nothing waits on another warp.  The last CTA to finish empties the queue.
 template <class T>
 __global__ void __launch_bounds__(MIGRATE_THREADS) migrate_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
                                                                   const T* __restrict__ v_prompt, int ctx) {
   const Geometry& g = a.geo;
-  const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y >> 1, part = blockIdx.y & 1;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_prologue();
-  const int n_quant = a.st.n_quant[u], n_promote = a.st.n_promote[u];
-  const int4* quant_list = a.st.quant_list + (size_t)u * (g.PF + g.Kq);
-  const int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
-  auto promote = [&](int k) {
-    const int4 it = promote_list[k];
-    promote_part<T>(g, part, a.st.q_pool + ((size_t)u * g.PQ + it.y) * g.q_page_bytes + (size_t)hk * g.q_head_bytes,
-                    a.st.fp_pool + ((size_t)u * g.PF + it.z) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes);
-  };
-  for (int item = blockIdx.x; item < n_quant + n_promote; item += gridDim.x) {
-    if (item < n_quant) {
-      const int4 it = quant_list[item];  // {window, source page (-1: prompt), destination page, linked promotion}
+  int32_t* cnt = a.st.mig_count + 2 * (a.unit0 / g.batch);
+  const int4* queue = a.st.mig_queue + (size_t)a.unit0 * (g.PF + g.Kq + g.Kf) * 2;
+  const int n_entries = *reinterpret_cast<volatile int32_t*>(cnt);
+  const int lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * (MIGRATE_THREADS / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (MIGRATE_THREADS / 32);
+  const int ks_n = g.D >> 4, ng = g.D / g.group;
+  const int n_kt = (g.W / g.group) * ks_n, n_vt = g.tiles * ng * 2, tpp = n_kt > n_vt ? n_kt : n_vt;
+  const int per_rec = g.Hkv * 2 * tpp, total = n_entries * per_rec;
+  for (int id = gw; id < total; id += n_warps) {
+    const int rec = id / per_rec, rem = id - rec * per_rec, hp = rem / tpp, task = rem - hp * tpp;
+    const int hk = hp >> 1, part = hp & 1;
+    if (task >= (part ? n_vt : n_kt)) continue;
+    const int4 r0 = queue[2 * rec], r1 = queue[2 * rec + 1];
+    const int u = r0.x, kind = r0.y, ul = u - a.unit0;
+    if (kind == 2) continue;
+    char* fp_u = a.st.fp_pool + (size_t)u * g.PF * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
+    char* q_u = a.st.q_pool + (size_t)u * g.PQ * g.q_page_bytes + (size_t)hk * g.q_head_bytes;
+    // task coordinates
+    int c0, c1, c2 = 0;
+    if (part == 0) { c0 = task / ks_n; c1 = task - c0 * ks_n; }                    // (blk, ks)
+    else { c2 = task & 1; c1 = (task >> 1) % ng; c0 = (task >> 1) / ng; }           // (tile, gc, ks)
+    if (kind == 0) {
       const T* rows = nullptr;
       const char* fp_head = nullptr;
-      if (it.y < 0) rows = (part ? v_prompt : k_prompt) + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)it.x * g.W) * g.D;
-      else fp_head = a.st.fp_pool + ((size_t)u * g.PF + it.y) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
-      __syncthreads();  // the staging buffer is reused from item to item
-      quantize_part<T>(g, part, rows, fp_head,
-                       a.st.q_pool + ((size_t)u * g.PQ + it.z) * g.q_page_bytes + (size_t)hk * g.q_head_bytes, smem_raw);
-      if (it.w >= 0) {
-        __syncthreads();  // every thread has finished reading the source page
-        promote(it.w);
+      if (r0.w < 0) rows = (part ? v_prompt : k_prompt) + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)r0.z * g.W) * g.D;
+      else fp_head = fp_u + (size_t)r0.w * g.fp_page_bytes;
+      char* qb = q_u + (size_t)r1.x * g.q_page_bytes;
+      if (part == 0) quant_key_task<T>(g, c0, c1, rows, fp_head, qb, lane);
+      else quant_value_task<T>(g, c0, c1, c2, rows, fp_head, qb, lane);
+      if (r1.y >= 0) {
+        const char* pq = q_u + (size_t)r1.y * g.q_page_bytes;
+        char* pf = fp_u + (size_t)r0.w * g.fp_page_bytes;
+        if (part == 0) promote_key_task<T>(g, c0, c1, pq, pf, lane);
+        else promote_value_task<T>(g, c0, c1, c2, pq, pf, lane);
       }
     } else {
-      const int k = item - n_quant;
-      if (promote_list[k].w == 0) promote(k);  // not linked to a quantization
+      const char* pq = q_u + (size_t)r0.w * g.q_page_bytes;
+      char* pf = fp_u + (size_t)r1.x * g.fp_page_bytes;
+      if (part == 0) promote_key_task<T>(g, c0, c1, pq, pf, lane);
+      else promote_value_task<T>(g, c0, c1, c2, pq, pf, lane);
     }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(cnt + 1, 1) == (int)gridDim.x - 1) { cnt[0] = 0; cnt[1] = 0; }
   }
 }
 
@@ -306,11 +406,6 @@ __global__ void export_q_page_kernel(const KernelArgs a, int u, int page, uint8_
   }
 }
 
-size_t migrate_smem_bytes(const Geometry& g) {
-  const size_t params = (size_t)((g.W / g.group) * g.D > g.W * (g.D / g.group) ? (g.W / g.group) * g.D : g.W * (g.D / g.group));
-  return (size_t)g.W * g.D * 2 + 2 * params * 4;
-}
-
 }  // namespace
 
 // CTAs per (unit, KV head) that walk a migration list: as many as there can be items, but no more
@@ -328,8 +423,11 @@ static int items_grid(int max_items, const KernelArgs& a) {
 cudaError_t launch_migrate(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
                            cudaStream_t s) {
   if (max_items <= 0) return cudaSuccess;
-  dim3 grid(items_grid(max_items, a), a.geo.Hkv * 2, a.n_units);
-  const size_t sm = migrate_smem_bytes(a.geo);
+  // warp tasks there can be at most, capped at a few resident waves of CTAs
+  const int ks_n = a.geo.D >> 4, n_kt = (a.geo.W / a.geo.group) * ks_n, n_vt = a.geo.tiles * (a.geo.D / a.geo.group) * 2;
+  const long long bound = ((long long)max_items * a.n_units * a.geo.Hkv * 2 * (n_kt > n_vt ? n_kt : n_vt) + 3) / 4;
+  dim3 grid((unsigned)(bound < 1184 ? bound : 1184));
+  const size_t sm = 0;
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
     return launch_pdl(migrate_kernel<__half>, grid, dim3(MIGRATE_THREADS), sm, s, a, (const __half*)k_prompt, (const __half*)v_prompt, ctx);
   return launch_pdl(migrate_kernel<__nv_bfloat16>, grid, dim3(MIGRATE_THREADS), sm, s, a, (const __nv_bfloat16*)k_prompt,

@@ -48,6 +48,38 @@ __device__ __forceinline__ int block_exclusive_scan(int cnt, int* scratch, int* 
   return rank;
 }
 
+// The same for three packed counters at once.  scratch: 99 ints.
+__device__ __forceinline__ int3 block_exclusive_scan3(int3 cnt, int* scratch, int3* total) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int lane = tid & 31, wid = tid >> 5;
+  int3 inc = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, inc.x, o), y = __shfl_up_sync(0xffffffffu, inc.y, o),
+              z = __shfl_up_sync(0xffffffffu, inc.z, o);
+    if (lane >= o) { inc.x += x; inc.y += y; inc.z += z; }
+  }
+  if (lane == 31) { scratch[wid] = inc.x; scratch[33 + wid] = inc.y; scratch[66 + wid] = inc.z; }
+  __syncthreads();
+  if (wid < 3) {
+    int* sc = scratch + 33 * wid;
+    const int v = (lane < (nt >> 5)) ? sc[lane] : 0;
+    int iv = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, iv, o);
+      if (lane >= o) iv += x;
+    }
+    sc[lane] = iv - v;
+    if (lane == 31) sc[32] = iv;
+  }
+  __syncthreads();
+  const int3 rank = make_int3(scratch[wid] + inc.x - cnt.x, scratch[33 + wid] + inc.y - cnt.y, scratch[66 + wid] + inc.z - cnt.z);
+  *total = make_int3(scratch[32], scratch[65], scratch[98]);
+  __syncthreads();
+  return rank;
+}
+
 // Stable, deterministic block-wide stream compaction: calls emit(i, rank) for every i in [0, n)
 // with pred(i), rank = number of smaller i with pred.  Returns the total.  pred must be pure until
 // emit(i) has run.  scratch: 33 ints of shared memory.
@@ -209,7 +241,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   const int u = a.unit0 + blockIdx.x, tid = threadIdx.x;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
-  int32_t* cw = reinterpret_cast<int32_t*>(keys + sort_cap);                 // [sort_cap] window of candidate c
+  int4* qrec = reinterpret_cast<int4*>(keys + sort_cap);                      // [PF + Kq] first demotions of this event
+  int4* prec = qrec + (g.PF + g.Kq);                                         // [Kf] promotions of this event
+  int32_t* cw = reinterpret_cast<int32_t*>(prec + (g.Kf > 0 ? g.Kf : 1));     // [sort_cap] window of candidate c
   int32_t* cfp = cw + sort_cap;                                              // [sort_cap] its full-precision page
   int32_t* cq = cfp + sort_cap;                                              // [sort_cap] its quantized page
   int32_t* ofp = cq + sort_cap;                                              // [PF] owner of each page
@@ -218,8 +252,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int32_t* free_q = free_fp + g.PF;                                          // [PQ]
   int32_t* reader = free_q + g.PQ;                                           // [PF] quantization that reads a page
   int32_t* flist = reader + g.PF;                                            // [EMAX] Full, then Quantized candidates
-  int32_t* scratch = flist + g.EMAX;                                         // [40]
-  uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 40);                 // [sort_cap] state before
+  int32_t* scratch = flist + g.EMAX;                                         // [128]
+  uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 128);                 // [sort_cap] state before
   uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
   uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
   pdl_prologue();
@@ -233,9 +267,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int32_t* q_owner = a.st.q_owner + (size_t)u * g.PQ;
   const int nw = a.st.n_windows[u];
   const int ow = a.st.open_window[u];
+  const int ow_page = ow >= 0 ? fp_page[ow] : -1;  // the open window is no candidate: its page does not change here
 
-  int* s_react = scratch + 34;
-  int* s_del = scratch + 35;
+  int* s_react = scratch + 100;
+  int* s_del = scratch + 101;
   if (tid == 0) { *s_react = 0; *s_del = 0; }
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) ofp[i] = fp_owner[i];
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) oq[i] = q_owner[i];
@@ -320,52 +355,86 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
       atomicAdd(s_react, 1);
     }
   }
-  __syncthreads();
-
-  // free pages in ascending id
-  const int n_free_fp = block_compact(g.PF, scratch, [&](int pg) { return ofp[pg] < 0; },
-                                      [&](int pg, int k) { free_fp[k] = pg; });
-  const int n_free_q = block_compact(g.PQ, scratch, [&](int pg) { return oq[pg] < 0; },
-                                     [&](int pg, int k) { free_q[k] = pg; });
-
-  // first demotions need a quantized page, ascending window index.  reader[p] = index of the
-  // quantization that reads full-precision page p
-  const int qcap = g.PF + g.Kq;
-  int4* quant_list = a.st.quant_list + (size_t)u * qcap;
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) reader[i] = -1;
   __syncthreads();
-  const int n_q_need = block_compact(
-      n_cand, scratch,
-      [&](int c) { return cnew[c] == QEVICT_TIER_QUANT && ctier[c] != QEVICT_TIER_QUANT && cled[c] == QEVICT_LEDGER_NONE; },
-      [&](int c, int k) {
-        if (k >= n_free_q || k >= qcap) { record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED); return; }
-        const int pg = free_q[k];
-        oq[pg] = cw[c];
-        quant_list[k] = make_int4(cw[c], prefill ? -1 : cfp[c], pg, -1);
-        if (!prefill && cfp[c] >= 0) reader[cfp[c]] = k;
-        cq[c] = pg;
-        cled[c] = QEVICT_LEDGER_ACTIVE;
-      });
-  // windows entering the Full tier without a full-precision page (promotions; prompt windows at
-  // prefill), ascending window index.  A promotion that receives a page some quantization of this event
-  // still has to read is linked to that quantization (the migration kernel runs it right after it).
-  int4* promote_list = a.st.promote_list + (size_t)u * g.Kf;
+
+  // ---- one packed scan yields six stable compactions at once (all ascending): free full-precision pages,
+  // free quantized pages, first demotions (need a quantized page), windows entering the Full tier without
+  // a page (promotions; prompt windows at prefill), and the Full / Quantized members of the work list ----
+  auto q_needs = [&](int c) { return cnew[c] == QEVICT_TIER_QUANT && ctier[c] != QEVICT_TIER_QUANT && cled[c] == QEVICT_LEDGER_NONE; };
+  auto fp_needs = [&](int c) { return cnew[c] == QEVICT_TIER_FULL && ctier[c] != QEVICT_TIER_FULL && cfp[c] < 0; };
+  int32_t* need_q = reinterpret_cast<int32_t*>(keys);  // the sort keys are dead from here on
+  int32_t* need_fp = need_q + sort_cap;
+  const int ch_f = (g.PF + ROUTE_THREADS - 1) / ROUTE_THREADS, ch_q = (g.PQ + ROUTE_THREADS - 1) / ROUTE_THREADS;
+  const int ch_c = (n_cand + ROUTE_THREADS - 1) / ROUTE_THREADS;
+  const int bf = min(g.PF, tid * ch_f), ef = min(g.PF, bf + ch_f), bq = min(g.PQ, tid * ch_q), eq = min(g.PQ, bq + ch_q);
+  const int bc = min(n_cand, tid * ch_c), ec = min(n_cand, bc + ch_c);
+  int3 cnt = make_int3(0, 0, 0);  // {free fp | free q << 16, need q | need fp << 16, Full | Quantized << 16}
+  for (int pg = bf; pg < ef; ++pg) cnt.x += ofp[pg] < 0 ? 1 : 0;
+  for (int pg = bq; pg < eq; ++pg) cnt.x += oq[pg] < 0 ? 0x10000 : 0;
+  for (int c = bc; c < ec; ++c) {
+    cnt.y += (q_needs(c) ? 1 : 0) + (fp_needs(c) ? 0x10000 : 0);
+    cnt.z += (cnew[c] == QEVICT_TIER_FULL ? 1 : 0) + (cnew[c] == QEVICT_TIER_QUANT ? 0x10000 : 0);
+  }
+  int3 tot;
+  int3 rk = block_exclusive_scan3(cnt, scratch, &tot);
+  const int n_free_fp = tot.x & 0xFFFF, n_free_q = tot.x >> 16, n_q_need = tot.y & 0xFFFF, n_fp_need = tot.y >> 16;
+  const int n_f = tot.z & 0xFFFF, n_q = tot.z >> 16;
+  int32_t* qlist = flist + n_f;
+  {
+    int r = rk.x & 0xFFFF;
+    for (int pg = bf; pg < ef; ++pg) if (ofp[pg] < 0) free_fp[r++] = pg;
+    r = rk.x >> 16;
+    for (int pg = bq; pg < eq; ++pg) if (oq[pg] < 0) free_q[r++] = pg;
+    int r0 = rk.y & 0xFFFF, r1 = rk.y >> 16, r2 = rk.z & 0xFFFF, r3 = rk.z >> 16;
+    for (int c = bc; c < ec; ++c) {
+      if (q_needs(c)) need_q[r0++] = c;
+      if (fp_needs(c)) need_fp[r1++] = c;
+      if (cnew[c] == QEVICT_TIER_FULL) { if (r2 < g.EMAX) flist[r2] = c; ++r2; }
+      if (cnew[c] == QEVICT_TIER_QUANT) { if (n_f + r3 < g.EMAX) qlist[r3] = c; ++r3; }
+    }
+  }
+  const int qcap = g.PF + g.Kq;
+  const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, g.Kf));
+  const int n_items = nq + (prefill ? 0 : nfp);
+  int* s_base = scratch + 102;
+  if (tid == 0) {
+    if (n_q_need > nq) record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED);
+    if (n_fp_need > nfp) record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED);
+    // this unit's migrations join the call's queue (the order of the units in it does not matter: the
+    // items are independent of one another); the reply is needed only at the very end
+    *s_base = n_items > 0 ? atomicAdd(a.st.mig_count + 2 * (a.unit0 / g.batch), n_items) : 0;
+  }
+  __syncthreads();
+
+  // first demotions take the free quantized pages in ascending order.  reader[p] = index of the
+  // quantization that reads full-precision page p
+  for (int k = tid; k < nq; k += ROUTE_THREADS) {
+    const int c = need_q[k], pg = free_q[k];
+    oq[pg] = cw[c];
+    qrec[k] = make_int4(cw[c], prefill ? -1 : cfp[c], pg, -1);  // {window, source page, destination page, linked promotion}
+    if (!prefill && cfp[c] >= 0) reader[cfp[c]] = k;
+    cq[c] = pg;
+    cled[c] = QEVICT_LEDGER_ACTIVE;
+  }
+  __syncthreads();
+  // windows entering the Full tier take the free full-precision pages in ascending order.  A promotion
+  // that receives a page some quantization of this event still has to read is linked to that quantization
+  // (the migration kernel runs it right after it, in the same warps).
   int4* copy_list = a.st.copy_list + (size_t)u * g.Kf;
-  const int n_fp_need = block_compact(
-      n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_FULL && ctier[c] != QEVICT_TIER_FULL && cfp[c] < 0; },
-      [&](int c, int k) {
-        if (k >= n_free_fp || k >= g.Kf) { record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED); return; }
-        const int pg = free_fp[k];
-        ofp[pg] = cw[c];
-        cfp[c] = pg;
-        if (prefill) {
-          copy_list[k] = make_int4(cw[c], pg, 0, 0);
-        } else {
-          const int rd = reader[pg];
-          promote_list[k] = make_int4(cw[c], cq[c], pg, rd >= 0 ? 1 : 0);
-          if (rd >= 0) quant_list[rd].w = k;
-        }
-      });
+  for (int k = tid; k < nfp; k += ROUTE_THREADS) {
+    const int c = need_fp[k], pg = free_fp[k];
+    ofp[pg] = cw[c];
+    cfp[c] = pg;
+    if (prefill) {
+      copy_list[k] = make_int4(cw[c], pg, 0, 0);
+    } else {
+      const int rd = reader[pg];
+      prec[k] = make_int4(cw[c], cq[c], pg, rd >= 0 ? 1 : 0);  // {window, source quantized page, destination page, linked}
+      if (rd >= 0) qrec[rd].w = k;
+    }
+  }
+  __syncthreads();
 
   // ---- commit: the candidates' rows and the owner tables go back to global memory --------------------
   for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
@@ -388,17 +457,27 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   }
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) fp_owner[i] = ofp[i];
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) q_owner[i] = oq[i];
-  __syncthreads();
+  // the migration records (32 bytes each; format: see the migration kernel)
+  {
+    int4* queue = a.st.mig_queue + ((size_t)a.unit0 * (g.PF + g.Kq + g.Kf) + *s_base) * 2;
+    for (int i = tid; i < n_items; i += ROUTE_THREADS) {
+      if (i < nq) {
+        const int4 it = qrec[i];
+        queue[2 * i] = make_int4(u, 0, it.x, it.y);
+        queue[2 * i + 1] = make_int4(it.z, it.w >= 0 ? prec[it.w].y : -1, 0, 0);
+      } else {
+        const int4 it = prec[i - nq];
+        queue[2 * i] = make_int4(u, it.w ? 2 : 1, it.x, it.y);
+        queue[2 * i + 1] = make_int4(it.z, -1, 0, 0);
+      }
+    }
+  }
+  __syncthreads();  // cfp / cq / cled are final (the evictions above reset theirs)
 
   // ---- decode work list: Full and Quantized windows (each ascending) interleaved in proportion, so that
   // every stretch of the list -- and therefore every warp of the attention kernel at every moment --
   // sees the same mix of 16-bit and low-bit pages; open window last -------------------------------------
   uint2* entries = a.st.entries + (size_t)u * g.EMAX;
-  const int n_f = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_FULL; },
-                                [&](int c, int k) { if (k < g.EMAX) flist[k] = c; });
-  int32_t* qlist = flist + n_f;
-  const int n_q = block_compact(n_cand, scratch, [&](int c) { return cnew[c] == QEVICT_TIER_QUANT; },
-                                [&](int c, int k) { if (n_f + k < g.EMAX) qlist[k] = c; });
   {
     const int n = n_f + n_q;
     for (int k = tid; k < n && k < g.EMAX; k += ROUTE_THREADS) {
@@ -416,14 +495,11 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   if (tid == 0) {
     int n = n_f + n_q;
     if (ow >= 0) {
-      if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)fp_page[ow]);
+      if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)ow_page);
       n += 1;
     }
     if (n > g.EMAX) { record_check(a.st.status, CHECK_ENTRY_OVERFLOW); n = g.EMAX; }
     a.st.n_live[u] = n;
-    const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, g.Kf));
-    a.st.n_quant[u] = nq;
-    a.st.n_promote[u] = prefill ? 0 : nfp;
     a.st.n_copy[u] = prefill ? nfp : 0;
     unsigned long long* c = a.st.counters + (size_t)u * 4;
     c[0] += prefill ? 0ull : (unsigned long long)nfp;
@@ -446,7 +522,8 @@ __global__ void export_mass_kernel(const KernelArgs a, int u, float* __restrict_
 }  // namespace
 
 size_t route_smem_bytes(const Geometry& g, int sort_cap) {
-  return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 40) * 4 + 16;
+  return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(g.PF + g.Kq + (g.Kf > 0 ? g.Kf : 1)) * 16 +
+         (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 128) * 4 + 16;
 }
 
 cudaError_t route_prepare(size_t max_smem) {
