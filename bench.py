@@ -226,8 +226,10 @@ def run_ours(args, rank, world):
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    host_t0 = time.perf_counter()
     for _ in range(K):
         step(t); t += 1
+    host_enqueue_s = time.perf_counter() - host_t0   # host time to enqueue the K steps (no synchronisation)
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -289,6 +291,7 @@ def run_ours(args, rank, world):
             "kernel_share_of_step": k_avg_ms / (ms / K),
             "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
         },
+        "host_enqueue_us_per_step": round(host_enqueue_s * 1e6 / K, 2),
         "kernel_us_per_step": {k: round(v[0] * 1e3 / K, 2) for k, v in ktimes.items()},
         "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_open", "n_evicted", "promotions",
                                              "quantizations", "reactivations", "deletions")},

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
 #pragma unroll
   for (int k = 0; k < NE; ++k) {
     const int e = e0 + wid + 4 * k;
-    rec[k] = (e < e1 && lane < g.Hq) ? __ldg(wrec + (size_t)lane * g.EMAX + e) : make_float2(0.f, 0.f);
+    rec[k] = (e < e1 && lane < g.Hq) ? __ldg(wrec + (size_t)e * g.Hq + lane) : make_float2(0.f, 0.f);
     ewin[k] = (e < e1) ? __ldg(&entries[e].x) : 0u;
   }
 
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
     for (int hb = 0; hb < g.Hq; hb += 32) {
       const int h = hb + lane;
       float2 rr = r;
-      if (hb > 0) rr = (h < g.Hq) ? __ldg(wrec + (size_t)h * g.EMAX + e) : make_float2(0.f, 0.f);
+      if (hb > 0) rr = (h < g.Hq) ? __ldg(wrec + (size_t)e * g.Hq + h) : make_float2(0.f, 0.f);
       if (h < g.Hq) term += rr.x * ex2a(rr.y - s_m[h]) * s_invl[h];
     }
 #pragma unroll

@@ -69,7 +69,7 @@ struct State {
   char* q_pool;         // [PQ] pages
   float* o_part;        // [Hq][MAX_SPLITS][D]
   float* ml;            // [Hq][MAX_SPLITS][2]
-  float2* wrec;         // [Hq][EMAX] {window exp-sum, reference max (log2 domain)}
+  float2* wrec;         // [EMAX][Hq] {window exp-sum, reference max (log2 domain)}
   float* mass_e;        // [EMAX] last step's mass per entry
   int32_t* status;      // [1] (shared by all units)
 };

@@ -40,7 +40,7 @@ struct DecodeParams {
   const char* q_pool;
   float* o_part;          // [n_units][Hq][MAX_SPLITS][D]
   float* ml;              // [n_units][Hq][MAX_SPLITS][2]
-  float2* wrec;           // [n_units][Hq][EMAX]
+  float2* wrec;           // [n_units][EMAX][Hq]
   int32_t* status;
   int unit0, S, Hq, Hkv, G, EMAX, PF, PQ;
   uint32_t fp_page_bytes, q_page_bytes;
@@ -472,7 +472,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
     if (g == 0) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        if (2 * t + h < p.G) p.wrec[((size_t)u * p.Hq + (size_t)hk * p.G + 2 * t + h) * p.EMAX + e] = make_float2(wsum[h], m_run[h]);
+        if (2 * t + h < p.G) p.wrec[((size_t)u * p.EMAX + e) * p.Hq + hk * p.G + 2 * t + h] = make_float2(wsum[h], m_run[h]);
       }
     }
   }

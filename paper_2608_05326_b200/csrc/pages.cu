@@ -284,7 +284,7 @@ __device__ __forceinline__ void promote_value_task(const Geometry& g, int tile, 
 // launch costs the same whether one unit or all of them migrate something, and the tasks are independent
 // (see above), so nothing waits on another warp.  The last CTA to finish empties the queue.
 template <class T>
-__global__ void __launch_bounds__(MIGRATE_THREADS) migrate_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
+__global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
                                                                   const T* __restrict__ v_prompt, int ctx) {
   const Geometry& g = a.geo;
   pdl_prologue();
@@ -423,10 +423,10 @@ static int items_grid(int max_items, const KernelArgs& a) {
 cudaError_t launch_migrate(const KernelArgs& a, const void* k_prompt, const void* v_prompt, int ctx, int max_items,
                            cudaStream_t s) {
   if (max_items <= 0) return cudaSuccess;
-  // warp tasks there can be at most, capped at a few resident waves of CTAs
+  // warp tasks there can be at most, capped at the CTAs that are resident at once (6 per SM)
   const int ks_n = a.geo.D >> 4, n_kt = (a.geo.W / a.geo.group) * ks_n, n_vt = a.geo.tiles * (a.geo.D / a.geo.group) * 2;
   const long long bound = ((long long)max_items * a.n_units * a.geo.Hkv * 2 * (n_kt > n_vt ? n_kt : n_vt) + 3) / 4;
-  dim3 grid((unsigned)(bound < 1184 ? bound : 1184));
+  dim3 grid((unsigned)(bound < 888 ? bound : 888));
   const size_t sm = 0;
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
     return launch_pdl(migrate_kernel<__half>, grid, dim3(MIGRATE_THREADS), sm, s, a, (const __half*)k_prompt, (const __half*)v_prompt, ctx);
