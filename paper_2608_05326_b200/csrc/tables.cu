@@ -8,7 +8,6 @@ namespace qevict {
 namespace {
 
 constexpr int ROUTE_THREADS = 256;
-constexpr unsigned long long KEY_SENTINEL = ~0ull;
 
 // order-preserving map float -> uint32 (ascending); -0 and +0 collapse
 __device__ __forceinline__ uint32_t mono_bits(float f) {
@@ -253,7 +252,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int32_t* reader = free_q + g.PQ;                                           // [PF] quantization that reads a page
   int32_t* flist = reader + g.PF;                                            // [EMAX] Full, then Quantized candidates
   int32_t* scratch = flist + g.EMAX;                                         // [128]
-  uint8_t* ctier = reinterpret_cast<uint8_t*>(scratch + 128);                 // [sort_cap] state before
+  int32_t* rhist = scratch + 128;                                            // [512] radix-selection histograms
+  uint8_t* ctier = reinterpret_cast<uint8_t*>(rhist + 512);                 // [sort_cap] state before
   uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
   uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
   pdl_prologue();
@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
 
   // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
   // Quantized, remainder -> Evicted -----------------------------------------------------------------
-  if (n_cand <= 512) {
+  if (n_cand <= 256) {
     // rank of a key = number of smaller keys (all keys are distinct)
     for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
       const unsigned long long mine = keys[c];
@@ -319,26 +319,63 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
       cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
     }
   } else {
-    int n_sort = 2;
-    while (n_sort < n_cand) n_sort <<= 1;
-    for (int i = n_cand + tid; i < n_sort; i += ROUTE_THREADS) keys[i] = KEY_SENTINEL;
-    __syncthreads();
-    for (int k = 2; k <= n_sort; k <<= 1) {
-      for (int j = k >> 1; j > 0; j >>= 1) {
-        for (int i = tid; i < n_sort; i += ROUTE_THREADS) {
-          const int ixj = i ^ j;
-          if (ixj > i) {
-            const unsigned long long x = keys[i], y = keys[ixj];
-            const bool asc = (i & k) == 0;
-            if ((x > y) == asc) { keys[i] = y; keys[ixj] = x; }
-          }
-        }
-        __syncthreads();
+    // Only the two cuts are needed, not the order: most-significant-digit-first radix selection of the
+    // K_f-th and the (K_f + K_q)-th smallest key, both in the same six passes (four 8-bit digits of the
+    // score, two of the candidate index).  thr[j] = the selected key: a candidate belongs to the first
+    // K_j exactly if its key is <= thr[j].
+    const int kk[2] = {min(g.Kf, n_cand), min(g.Kf + g.Kq, n_cand)};
+    int* hist = rhist;                                   // [2][256]
+    uint32_t* sel = reinterpret_cast<uint32_t*>(scratch + 104);  // [2][2] selected prefixes {low, high word}
+    int* need = scratch + 108;                           // [2] rank still to find inside the current bucket
+    if (tid < 2) { sel[2 * tid] = 0u; sel[2 * tid + 1] = 0u; need[tid] = kk[tid]; }
+    unsigned long long mask = 0ull;
+#pragma unroll 1
+    for (int pass = 0; pass < 6; ++pass) {
+      const int shift = pass < 4 ? 56 - 8 * pass : (pass == 4 ? 8 : 0);
+      for (int i = tid; i < 512; i += ROUTE_THREADS) hist[i] = 0;
+      __syncthreads();
+      const unsigned long long p0 = ((unsigned long long)sel[1] << 32) | sel[0], p1 = ((unsigned long long)sel[3] << 32) | sel[2];
+      for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+        const unsigned long long key = keys[c];
+        const int d = (int)((key >> shift) & 255ull);
+        if ((key & mask) == p0) atomicAdd(&hist[d], 1);
+        if ((key & mask) == p1) atomicAdd(&hist[256 + d], 1);
       }
+      __syncthreads();
+      if (tid < 64) {
+        // warp j finds the digit of cut j: the first digit whose running count reaches need[j]
+        const int j = tid >> 5, lane = tid & 31;
+        const int* hj = hist + 256 * j;
+        int loc[8], sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { loc[i] = hj[lane * 8 + i]; sum += loc[i]; }
+        int inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += v;
+        }
+        const int want = need[j];
+        const unsigned hit = __ballot_sync(0xffffffffu, inc >= want);
+        const int owner = hit ? __ffs(hit) - 1 : 31;  // kk >= 1 and the bucket holds >= want keys, so hit != 0
+        if (lane == owner) {
+          int run = inc - sum, d = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (run + loc[i] < want && i < 7) { run += loc[i]; d = i + 1; }
+            else break;
+          }
+          need[j] = want - run;
+          sel[2 * j + (shift >= 32 ? 1 : 0)] |= (uint32_t)(lane * 8 + d) << (shift & 31);
+        }
+      }
+      mask |= 255ull << shift;
+      __syncthreads();
     }
-    for (int pos = tid; pos < n_cand; pos += ROUTE_THREADS) {
-      const uint32_t c = (uint32_t)keys[pos];
-      cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+    const unsigned long long t0 = ((unsigned long long)sel[1] << 32) | sel[0], t1 = ((unsigned long long)sel[3] << 32) | sel[2];
+    for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+      const unsigned long long key = keys[c];
+      cnew[c] = (kk[0] > 0 && key <= t0) ? QEVICT_TIER_FULL : ((kk[1] > 0 && key <= t1) ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
     }
   }
   __syncthreads();
@@ -523,7 +560,7 @@ __global__ void export_mass_kernel(const KernelArgs a, int u, float* __restrict_
 
 size_t route_smem_bytes(const Geometry& g, int sort_cap) {
   return (size_t)sort_cap * (8 + 12 + 3) + (size_t)(g.PF + g.Kq + (g.Kf > 0 ? g.Kf : 1)) * 16 +
-         (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 128) * 4 + 16;
+         (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 128 + 512) * 4 + 16;
 }
 
 cudaError_t route_prepare(size_t max_smem) {

@@ -104,7 +104,7 @@ class LockstepRun:
     """One workload instance on the GPU (all its units in one cache) and oracles for a subset of units."""
 
     def __init__(self, wl, oracle_units=None, score_mode="observation", rebalance_interval=None, device="cuda",
-                 gen_device="cpu"):
+                 gen_device="cpu", score_levels=None):
         self.wl = wl
         self.R = wl.rebalance_interval if rebalance_interval is None else rebalance_interval
         self.units = list(range(wl.n_units)) if oracle_units is None else list(oracle_units)
@@ -125,6 +125,8 @@ class LockstepRun:
                     s = workloads.synthetic_window_scores(wl, u)
                 s = workloads.place_planted(s, workloads.planted_windows(wl, u), wl.fp_budget_windows,
                                             wl.q_budget_windows)
+                if score_levels:  # few distinct prefill scores: the first routing event is decided by the tie-break
+                    s = torch.round(s / s.max() * score_levels) * (s.max() / score_levels)
                 ks.append(k); vs.append(v); ss.append(s)
                 self.scores[u] = s
                 self.queries[u] = workloads.gen_queries(wl, u, k, s)

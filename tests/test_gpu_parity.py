@@ -76,6 +76,21 @@ def test_shapes_lockstep(kw):
     run.close()
 
 
+def test_many_candidates_and_tied_scores():
+    # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
+    # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides
+    ls = _lockstep()
+    wl = _small("ties", context=16384, n_q_heads=1, n_kv_heads=1, fp_budget_windows=120, q_budget_windows=260, steps=10)
+    run = ls.LockstepRun(wl, rebalance_interval=1, score_levels=7)
+    run.check_state("all", "after prefill")
+    st = run.cache.stats()
+    assert (st["n_full"], st["n_quant"]) == (120, 260)
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    run.close()
+
+
 def test_multiple_units_and_layers():
     ls = _lockstep()
     wl = _small("multi", batch=3, n_layers=2, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, steps=40)
