@@ -5,8 +5,9 @@
 // numerator, from which the combine kernel forms the window mass of Eq. 1.
 //
 // Work decomposition: CTA = (split, KV head, unit), 4 warps.  Warp `wid` of split `s` owns the work
-// list entries s*4+wid, s*4+wid + 4S, ...; the list is ordered Full.., Quantized.., recent.., so a
-// strided walk gives every warp the same mix of 16-bit and low-bit windows (balanced bytes).  Each
+// list entries s*4+wid, s*4+wid + 4S, ...; the routing kernel interleaves Full and Quantized windows
+// in the list in proportion to their numbers (recent windows last), so every warp alternates between
+// bandwidth-heavy 16-bit tiles and arithmetic-heavy low-bit tiles all the way through its walk.  Each
 // warp runs an independent online softmax over its windows; the four warps are merged in shared
 // memory and the CTA writes one partial (m, l, O) per query head of its KV head.
 //
