@@ -104,7 +104,7 @@ class LockstepRun:
     """One workload instance on the GPU (all its units in one cache) and oracles for a subset of units."""
 
     def __init__(self, wl, oracle_units=None, score_mode="observation", rebalance_interval=None, device="cuda",
-                 gen_device="cpu", score_levels=None):
+                 gen_device="cpu", score_levels=None, free_running=False):
         self.wl = wl
         self.R = wl.rebalance_interval if rebalance_interval is None else rebalance_interval
         self.units = list(range(wl.n_units)) if oracle_units is None else list(oracle_units)
@@ -140,6 +140,11 @@ class LockstepRun:
             torch.cuda.synchronize()
             del ks, vs, kd, vd
         self.step_idx = 0
+        # free-running: the oracle keeps its own float64 scores (no overwrite with the GPU's); a routing event
+        # may then differ, but only by windows whose scores sit on a tier cut (see rebalance)
+        self.free_running = free_running
+        self.boundary_flips = 0
+        self.diverged = False
 
     def unit_ls(self, u):
         return u // self.wl.batch, u % self.wl.batch
@@ -174,13 +179,16 @@ class LockstepRun:
                 assert abs(mass.sum() - wl.n_q_heads) < 1e-4 * wl.n_q_heads, what
             imp = tab["importance"].double().numpy()
             assert np.all(np.abs(imp - orc.importance) <= MASS_RTOL * np.abs(orc.importance) + 1e-7), what + " scores"
-            orc.importance[:] = imp  # lockstep: route on the GPU's float32 scores
+            if not self.free_running:
+                orc.importance[:] = imp  # lockstep: route on the GPU's float32 scores
         self.step_idx += 1
         if self.step_idx % self.R == 0:
             self.rebalance()
         return out
 
     def rebalance(self, full_check=False):
+        if self.free_running:
+            return self._rebalance_free()
         before = {u: (o.tier.copy(), o.ledger_flag.copy()) for u, o in self.oracles.items()}
         self.cache.rebalance(-1)
         changed = {}
@@ -190,6 +198,40 @@ class LockstepRun:
             changed[u] = [int(w) for w in np.flatnonzero((t0 != orc.tier) | (l0 != orc.ledger_flag))
                           if orc.tier[w] in (TIER_FULL, TIER_QUANT)]
         self.check_state("all" if full_check else changed, what="after rebalance at step %d" % self.step_idx)
+
+    def _rebalance_free(self):
+        """Both sides route on their own scores.  Equal tiers -> everything must still match bit for bit.
+        Different tiers are admissible only for windows whose oracle score lies within 1e-4 relative of the
+        score at one of the two cuts (the K_f-th or the (K_f+K_q)-th candidate); the run then counts the flip
+        and stops comparing states (pages are handed out differently from there on)."""
+        wl = self.wl
+        cuts = {}
+        for u, orc in self.oracles.items():
+            ranked = orc.ranked_candidates()
+            sc = orc.importance.astype(np.float32)
+            cuts[u] = [float(sc[ranked[k - 1]]) for k in (wl.fp_budget_windows, wl.fp_budget_windows + wl.q_budget_windows)
+                       if 1 <= k <= len(ranked)]
+            cuts[u] += [float(sc[ranked[k]]) for k in (wl.fp_budget_windows, wl.fp_budget_windows + wl.q_budget_windows)
+                        if k < len(ranked)]
+        self.cache.rebalance(-1)
+        for u, orc in self.oracles.items():
+            orc.rebalance()
+            layer, seq = self.unit_ls(u)
+            t = self.cache.export_tables(layer, seq)
+            n = int(t["n_windows"][0])
+            got = t["tier"].numpy()[:n]
+            bad = np.flatnonzero(got != orc.tier[:n])
+            if bad.size == 0:
+                continue
+            for w in bad:
+                s = float(np.float32(orc.importance[w]))
+                assert any(abs(s - c) <= MASS_RTOL * max(abs(c), 1e-30) for c in cuts[u]), \
+                    "unit %d window %d: tiers differ (gpu %d oracle %d) away from a tier cut (score %.9g, cuts %s)" % (
+                        u, w, got[w], orc.tier[w], s, cuts[u])
+            self.boundary_flips += int(bad.size)
+            self.diverged = True
+        if not self.diverged:
+            self.check_state("all", what="free-running, after rebalance at step %d" % self.step_idx)
 
     def close(self):
         self.cache.close()
