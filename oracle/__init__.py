@@ -34,6 +34,7 @@ from .cache import (  # noqa: F401
     TIER_FULL,
     TIER_QUANT,
     TIER_EVICTED,
+    TIER_SINK,
     LEDGER_NONE,
     LEDGER_ACTIVE,
     LEDGER_DORMANT,

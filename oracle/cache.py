@@ -16,9 +16,13 @@ Paper basis:
 Readings taken where the paper is silent (each is listed in the design notes):
   * the window size W and the routing interval are separate parameters; routing
     happens when `rebalance()` is called;
-  * the protected recent region is the open window being filled plus the filled
-    windows waiting for the next routing event ("aged"); both stay in full
-    precision and are attended to; there are no sink windows in this version;
+  * the protected regions are window-granular: the sink prefix is the first
+    `sink_windows` windows of the prompt, the recent region is the open window
+    being filled plus the `recent_windows` most recently filled windows; both stay
+    in full precision, are attended to, are never candidates and do not count
+    against K_f (the budget constraint reserves B_sink and B_local separately);
+    a filled window that is no longer among the `recent_windows` newest has exited
+    the recent region and waits ("aged") for the next routing event;
   * the score is the raw sum over query heads (Eq. 1 without its constant
     1/H_q, which does not change any ranking) and is accumulated at every decode
     step, as the sum over tau in Eq. 1 states;
@@ -45,7 +49,7 @@ from .attention import accessible_attention
 from .numerics import round_to_dtype
 from .quantizer import dequantize_window, quantize_window
 
-TIER_NONE, TIER_OPEN, TIER_AGED, TIER_FULL, TIER_QUANT, TIER_EVICTED = 0, 1, 2, 3, 4, 5
+TIER_NONE, TIER_OPEN, TIER_AGED, TIER_FULL, TIER_QUANT, TIER_EVICTED, TIER_SINK = 0, 1, 2, 3, 4, 5, 6
 LEDGER_NONE, LEDGER_ACTIVE, LEDGER_DORMANT = 0, 1, 2
 
 _ELEM_BYTES = {"fp16": 2, "bf16": 2}
@@ -65,6 +69,8 @@ class OracleConfig:
     max_context: int
     aged_windows: int = 2  # filled windows that may wait for the next routing event
     softmax_scale: float = 0.0  # 0 => 1/sqrt(head_dim)
+    sink_windows: int = 0  # protected sink prefix, in windows
+    recent_windows: int = 0  # filled windows kept in the protected recent region
 
     @property
     def scale(self):
@@ -76,7 +82,7 @@ class OracleConfig:
 
     @property
     def fp_pool_pages(self):
-        return self.fp_budget_windows + self.aged_windows + 1
+        return self.fp_budget_windows + self.sink_windows + self.recent_windows + self.aged_windows + 1
 
     @property
     def q_pool_pages(self):
@@ -147,7 +153,7 @@ class UnitOracle:
         for w in range(n):
             sl = slice(w * cfg.window, (w + 1) * cfg.window)
             self.fp[w] = (np.array(k[:, sl, :], dtype=np.float64), np.array(v[:, sl, :], dtype=np.float64))
-            self.tier[w] = TIER_AGED
+            self.tier[w] = TIER_SINK if w < cfg.sink_windows else TIER_AGED
             self.importance[w] = float(window_scores[w])
         self.n_windows = n
         self.rebalance()
@@ -189,7 +195,7 @@ class UnitOracle:
         acc = []
         for w in range(self.n_windows):
             t = self.tier[w]
-            if t in (TIER_FULL, TIER_AGED):
+            if t in (TIER_FULL, TIER_AGED, TIER_SINK):
                 k, v = self.fp[w]
                 acc.append((w, k, v, cfg.window))
             elif t == TIER_OPEN:
@@ -226,10 +232,19 @@ class UnitOracle:
         return round_to_dtype(out, cfg.dtype), mass
 
     # -------------------------------------------------------------- routing
-    def ranked_candidates(self):
-        """Candidate pool F ∪ Q ∪ aged, ranked by float32 score, higher first, lower index first."""
+    def recent_lo(self):
+        """First window index of the protected recent region: the `recent_windows` newest filled
+        windows (the open window, if any, comes after them)."""
         t = self.tier[: self.n_windows]
-        cand = np.flatnonzero((t == TIER_FULL) | (t == TIER_QUANT) | (t == TIER_AGED))
+        n_filled = self.n_windows - int((t == TIER_OPEN).sum())
+        return n_filled - self.cfg.recent_windows
+
+    def ranked_candidates(self):
+        """Candidate pool F ∪ Q ∪ aged (filled windows that have exited the recent region), ranked by
+        float32 score, higher first, lower index first.  Sink windows are never candidates."""
+        t = self.tier[: self.n_windows]
+        idx = np.arange(self.n_windows)
+        cand = np.flatnonzero((t == TIER_FULL) | (t == TIER_QUANT) | ((t == TIER_AGED) & (idx < self.recent_lo())))
         s32 = self.importance[cand].astype(np.float32)
         order = np.lexsort((cand, -s32.astype(np.float64)))
         return cand[order]
@@ -275,9 +290,14 @@ class UnitOracle:
 
         # allocations, ascending window index, ascending free page id.  A window of the new Full tier
         # that holds no full-precision page needs one: a promotion, or a prompt window at prefill.
-        for w in sorted(int(x) for x in new_f):
+        in_f = set(int(x) for x in new_f)
+        pinned = [w for w in range(self.n_windows)
+                  if self.tier[w] in (TIER_SINK, TIER_AGED) and w not in in_f and self.fp_page[w] < 0 and w in self.fp]
+        for w in sorted(in_f | set(pinned)):
             if self.fp_page[w] < 0:
                 self.fp_page[w] = self._take_lowest_free(self.fp_owner, w)
+            if w not in in_f:
+                continue  # sink or recent window of the prompt: gets its page, keeps its state
             if self.tier[w] == TIER_QUANT:
                 self.fp[w] = promoted_data[w]
                 self.ledger_flag[w] = LEDGER_DORMANT
@@ -299,4 +319,4 @@ class UnitOracle:
         t = self.tier[: self.n_windows]
         return {name: int((t == val).sum()) for name, val in
                 (("open", TIER_OPEN), ("aged", TIER_AGED), ("full", TIER_FULL),
-                 ("quant", TIER_QUANT), ("evicted", TIER_EVICTED))}
+                 ("quant", TIER_QUANT), ("evicted", TIER_EVICTED), ("sink", TIER_SINK))}

@@ -19,6 +19,7 @@ from oracle import (
     TIER_FULL,
     TIER_OPEN,
     TIER_QUANT,
+    TIER_SINK,
     OracleConfig,
     UnitOracle,
     accessible_attention,
@@ -94,6 +95,89 @@ def _prefilled(cfg, rng, ctx_windows=16, scores=None):
     return u, k, v, scores
 
 
+def _protected_cfg(dtype="fp16", k_f=3, k_q=4, sinks=2, recent=3, ctx_windows=16, extra=12):
+    return OracleConfig(4, 2, 64, dtype, 32, 4, 32, k_f, k_q, (ctx_windows + extra) * 32, aged_windows=2,
+                        sink_windows=sinks, recent_windows=recent)
+
+
+# ------------------------------------------------------------- protected sink and recent regions
+def test_sink_and_recent_windows_are_protected_and_outside_the_budget():
+    """Cache partition (sink, recent, Full, Quantized, Evicted): the protected regions stay in full
+    precision and never enter the candidate pool; candidates are the Full and Quantized windows plus the
+    windows that have exited the recent region.  Checked against a model of the regions kept here: the
+    sink prefix is windows 0..n_s-1; after every step the recent region is the n_r newest filled windows."""
+    rng = np.random.default_rng(31)
+    cfg = _protected_cfg()
+    # lowest scores on the sink windows and on the newest prompt windows: unprotected they would be evicted
+    scores = np.linspace(0.1, 1.0, 16).astype(np.float32)
+    scores[:2] = 0.0
+    scores[-3:] = 0.0
+    u, k, v, _ = _prefilled(cfg, rng, scores=scores)
+    c = u.tier_counts()
+    assert c == {"open": 0, "aged": 3, "full": 3, "quant": 4, "evicted": 4, "sink": 2}
+    assert list(np.flatnonzero(u.tier == TIER_SINK)) == [0, 1]
+    assert list(np.flatnonzero(u.tier == TIER_AGED)) == [13, 14, 15]          # recent region of the prompt
+    # the 11 unprotected windows were ranked on their own: 3 best Full, next 4 Quantized, 4 evicted
+    assert list(np.flatnonzero(u.tier == TIER_FULL)) == [10, 11, 12]
+    assert list(np.flatnonzero(u.tier == TIER_QUANT)) == [6, 7, 8, 9]
+    assert list(np.flatnonzero(u.tier == TIER_EVICTED)) == [2, 3, 4, 5]
+    # pages at prefill: ascending window index over everything that stays in full precision
+    assert [int(u.fp_page[w]) for w in (0, 1, 10, 11, 12, 13, 14, 15)] == list(range(8))
+    n_filled = 16
+    for t in range(32 * 6):
+        q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), cfg.dtype)
+        kn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+        vn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+        out, mass = u.decode_attn(q, kn, vn)
+        assert abs(mass.sum() - cfg.n_q_heads) < 1e-9
+        if (t + 1) % 32 == 0:
+            n_filled += 1
+        recent = set(range(n_filled - cfg.recent_windows, n_filled))
+        cand = set(int(w) for w in u.ranked_candidates())
+        assert cand.isdisjoint(recent) and cand.isdisjoint({0, 1})
+        expect_cand = {w for w in range(n_filled) if u.tier[w] in (TIER_FULL, TIER_QUANT)} | \
+                      {w for w in range(2, n_filled) if u.tier[w] == TIER_AGED and w not in recent}
+        assert cand == expect_cand
+        if t % 5 == 4:
+            u.rebalance()
+            c = u.tier_counts()
+            assert c["sink"] == 2 and c["full"] <= cfg.fp_budget_windows and c["quant"] <= cfg.q_budget_windows
+            assert all(u.tier[w] == TIER_AGED for w in recent)               # still protected
+            assert c["aged"] == len(recent)                                   # everything that exited was routed
+            fp_held = u.fp_page[u.fp_page >= 0]
+            assert len(set(fp_held.tolist())) == len(fp_held) <= cfg.fp_pool_pages
+            for w in range(u.n_windows):
+                assert (u.fp_page[w] >= 0) == (u.tier[w] in (TIER_FULL, TIER_AGED, TIER_OPEN, TIER_SINK))
+    assert u.stats["deletions"] > 4
+
+
+def test_protected_regions_with_full_budget_equal_brute_force_attention():
+    rng = np.random.default_rng(32)
+    cfg = _protected_cfg("bf16", k_f=64, k_q=4, sinks=1, recent=2)
+    u, k, v, _ = _prefilled(cfg, rng)
+    assert u.tier_counts()["full"] == 13 and u.tier_counts()["sink"] == 1 and u.tier_counts()["aged"] == 2
+    ks, vs = [k], [v]
+    for t in range(70):
+        q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), "bf16")
+        kn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), "bf16")
+        vn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), "bf16")
+        ks.append(kn[:, None]); vs.append(vn[:, None])
+        out, mass = u.decode_attn(q, kn, vn)
+        ref, p = _full_attention_reference(q, np.concatenate(ks, 1), np.concatenate(vs, 1), cfg.scale)
+        assert np.array_equal(out, round_to_dtype(ref, "bf16"))
+        if t % 7 == 6:
+            u.rebalance()
+            assert u.tier_counts()["evicted"] == 0 and u.tier_counts()["quant"] == 0
+
+
+def test_no_protected_regions_is_the_default():
+    rng = np.random.default_rng(33)
+    a, k, v, s = _prefilled(_small_cfg(), rng)
+    b = UnitOracle(_protected_cfg(k_f=4, k_q=6, sinks=0, recent=0, extra=8))
+    b.prefill_assign(k, v, s)
+    assert np.array_equal(a.tier, b.tier) and np.array_equal(a.fp_page, b.fp_page) and np.array_equal(a.q_page, b.q_page)
+
+
 # ------------------------------------------------- (a) everything in full precision = full attention
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
 def test_full_budget_equals_brute_force_attention(dtype):
@@ -130,7 +214,7 @@ def test_mass_sums_to_heads_times_steps_and_budgets_hold():
     u = UnitOracle(cfg)
     u.prefill_assign(k, v, scores.numpy())
     base = u.importance.sum()
-    assert u.tier_counts() == {"open": 0, "aged": 0, "full": 8, "quant": 16, "evicted": 40}
+    assert u.tier_counts() == {"open": 0, "aged": 0, "full": 8, "quant": 16, "evicted": 40, "sink": 0}
     q_all = wlmod.gen_queries(wl, 0, torch.from_numpy(k), scores).double().numpy()
     kn, vn = wlmod.gen_new_kv(wl, 0)
     evicted_before = set()
