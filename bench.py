@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--bits", type=int, default=None, help="config 4 sweep point")
     ap.add_argument("--fp-frac", type=float, default=None, help="config 4 sweep point")
     ap.add_argument("--rebalance-interval", type=int, default=1)
+    ap.add_argument("--sink-windows", type=int, default=0, help="protected sink prefix, in windows (0 in every BASELINE config)")
+    ap.add_argument("--recent-windows", type=int, default=0, help="filled windows kept in the protected recent region")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -69,7 +71,8 @@ def make_workload(args, total_steps):
     wl = workloads.config(args.config, **kw)
     layers = args.layers if args.layers is not None else (32 if args.config == 1 else (8 if args.config == 3 else wl.n_layers))
     batch = args.batch if args.batch is not None else wl.batch
-    return replace(wl, n_layers=layers, batch=batch, steps=total_steps, rebalance_interval=args.rebalance_interval)
+    return replace(wl, n_layers=layers, batch=batch, steps=total_steps, rebalance_interval=args.rebalance_interval,
+                   sink_windows=args.sink_windows, recent_windows=args.recent_windows)
 
 
 def peak_hbm_gbs():
@@ -167,8 +170,9 @@ def attention_kernel_bytes(wl, stats, n_splits_hint=None):
     windows at 16 bit, Quantized windows as codes + parameters), the queries, the work list, and the
     partial results it writes."""
     m_f, m_q = wl.fp_window_bytes(), wl.q_window_bytes()
-    kv = (stats["n_full"] + stats["n_aged"]) * m_f + stats["n_quant"] * m_q + stats["n_open"] * m_f // 2
-    live = stats["n_full"] + stats["n_aged"] + stats["n_quant"] + stats["n_open"]
+    n_fp = stats["n_full"] + stats["n_aged"] + stats.get("n_sink", 0)
+    kv = n_fp * m_f + stats["n_quant"] * m_q + stats["n_open"] * m_f // 2
+    live = n_fp + stats["n_quant"] + stats["n_open"]
     q_bytes = wl.n_units * wl.n_q_heads * wl.head_dim * 2
     lists = live * 8 + live * wl.n_q_heads * 8  # work list read, per-(head, window) records written
     return kv + q_bytes + lists
@@ -189,7 +193,8 @@ def run_ours(args, rank, world):
     wl = sharding.rank_workload(wl, rank)  # every rank owns its own sequences (weak scaling, no exchange)
     cfg = binding.make_config(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window,
                               wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
-                              rebalance_interval_hint=args.rebalance_interval, device=dev.index)
+                              rebalance_interval_hint=args.rebalance_interval, device=dev.index,
+                              sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
     cache = binding.QEvictCache(cfg)
     if args.splits:
         cache.set_splits(args.splits)
@@ -278,7 +283,8 @@ def run_ours(args, rank, world):
             "workload": "%s x %d layers x batch %d (layer-batched launches)" % (wl.name, wl.n_layers, wl.batch),
             "units_per_step": wl.n_units, "context": wl.context, "window": wl.window, "quant_bits": wl.quant_bits,
             "group_size": wl.group_size, "fp_budget_windows": wl.fp_budget_windows,
-            "q_budget_windows": wl.q_budget_windows, "rebalance_interval": R, "append": append,
+            "q_budget_windows": wl.q_budget_windows, "sink_windows": wl.sink_windows, "recent_windows": wl.recent_windows,
+            "rebalance_interval": R, "append": append,
             "l2": "inputs larger than L2 (KV working set %.0f MB per step)" % (kbytes / 1e6),
         },
         "layer_steps_per_sec": world * K * wl.n_units / (ms * 1e-3),
@@ -293,7 +299,7 @@ def run_ours(args, rank, world):
         },
         "host_enqueue_us_per_step": round(host_enqueue_s * 1e6 / K, 2),
         "kernel_us_per_step": {k: round(v[0] * 1e3 / K, 2) for k, v in ktimes.items()},
-        "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_open", "n_evicted", "promotions",
+        "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_sink", "n_open", "n_evicted", "promotions",
                                              "quantizations", "reactivations", "deletions")},
     }
     if e2e:
@@ -321,7 +327,8 @@ def time_oracle(wl, n_steps, warmup, budget_s):
     from oracle import OracleConfig, UnitOracle
     aged = (wl.rebalance_interval + wl.window - 1) // wl.window + 1
     ocfg = OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
-                        wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged)
+                        wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged,
+                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
     k, v = workloads.gen_prompt_kv(wl, 0)
     s = workloads.place_planted(workloads.synthetic_window_scores(wl, 0), workloads.planted_windows(wl, 0),
                                 wl.fp_budget_windows, wl.q_budget_windows)

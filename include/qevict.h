@@ -65,10 +65,12 @@ enum { QEVICT_DTYPE_FP16 = 0, QEVICT_DTYPE_BF16 = 1 };
 enum {
   QEVICT_TIER_NONE = 0,    /* window index not created yet */
   QEVICT_TIER_OPEN = 1,    /* recent region: the window being filled by appended tokens */
-  QEVICT_TIER_AGED = 2,    /* recent region: filled, waiting for the next routing event */
+  QEVICT_TIER_AGED = 2,    /* filled: inside the protected recent region, or out of it and waiting for the
+                              next routing event */
   QEVICT_TIER_FULL = 3,
   QEVICT_TIER_QUANT = 4,
-  QEVICT_TIER_EVICTED = 5
+  QEVICT_TIER_EVICTED = 5,
+  QEVICT_TIER_SINK = 6     /* protected sink prefix: full precision, never a candidate */
 };
 /* ledger states */
 enum { QEVICT_LEDGER_NONE = 0, QEVICT_LEDGER_ACTIVE = 1, QEVICT_LEDGER_DORMANT = 2 };
@@ -91,6 +93,12 @@ typedef struct {
                                       the full-precision pages that hold aged windows; 0 => W */
   float softmax_scale;       /* 0 => 1/sqrt(d) */
   int32_t device;            /* CUDA device ordinal */
+  int32_t sink_windows;      /* protected sink prefix: the first windows of the prompt stay in full precision,
+                                are never candidates and do not count against K_f [cache partition] */
+  int32_t recent_windows;    /* protected recent region: besides the window being filled, this many of the
+                                most recently filled windows stay in full precision and are not candidates
+                                until newer windows push them out [candidate pool: windows that have exited
+                                the recent region] */
 } qevict_config;
 
 typedef struct {
@@ -100,6 +108,7 @@ typedef struct {
   uint64_t deletions;      /* windows evicted */
   uint64_t n_full, n_quant, n_aged, n_open, n_evicted; /* current window counts */
   uint64_t decode_steps;
+  uint64_t n_sink;         /* protected sink windows */
 } qevict_stats;
 
 /* Bytes of one Full window and one Quantized window (all KV heads, keys and values), and the tier

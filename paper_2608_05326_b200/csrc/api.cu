@@ -71,6 +71,8 @@ const char* validate(const qevict_config* c) {
   if (c->window < 1 || c->max_context < c->window || c->max_context % c->window) return "max_context must be a positive multiple of window";
   if (c->group_size < 1 || c->window % c->group_size || c->head_dim % c->group_size) return "group_size must divide window and head_dim";
   if (c->rebalance_interval_hint < 0) return "rebalance_interval_hint < 0";
+  if (c->sink_windows < 0 || c->recent_windows < 0) return "sink_windows and recent_windows must be >= 0";
+  if (c->sink_windows + c->recent_windows > c->max_context / c->window) return "protected windows exceed max_context";
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return "softmax_scale must be finite and >= 0";
   return nullptr;
 }
@@ -93,9 +95,11 @@ void make_geometry(const qevict_config& c, Geometry& g) {
   g.NW = c.max_context / c.window;
   const int r = c.rebalance_interval_hint > 0 ? c.rebalance_interval_hint : c.window;
   g.aged_cap = (r + g.W - 1) / g.W + 1;
-  g.PF = g.Kf + g.aged_cap + 1;
+  g.n_sink = c.sink_windows; g.n_recent = c.recent_windows;
+  g.Kfp = g.Kf + g.n_sink + g.n_recent;
+  g.PF = g.Kfp + g.aged_cap + 1;
   g.PQ = g.Kq + g.Kf;
-  g.EMAX = g.Kf + g.Kq + g.aged_cap + 1;
+  g.EMAX = g.Kfp + g.Kq + g.aged_cap + 1;
   g.tiles = g.W / 32;
   g.fp_tile_bytes = 32u * g.D * 2u;
   g.fp_head_bytes = g.tiles * 2u * g.fp_tile_bytes;
@@ -136,7 +140,7 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.open_fill = (int32_t*)take(U * 4);
   s.n_live = (int32_t*)take(U * 4);
   s.entries = (uint2*)take(U * g.EMAX * 8);
-  s.copy_list = (int4*)take(U * (size_t)(g.Kf > 0 ? g.Kf : 1) * 16);
+  s.copy_list = (int4*)take(U * (size_t)(g.Kfp > 0 ? g.Kfp : 1) * 16);
   s.n_copy = (int32_t*)take(U * 4);
   s.mig_queue = (int4*)take(U * (size_t)(g.PF + g.Kq + g.Kf) * 32);
   s.mig_count = (int32_t*)take((size_t)g.n_layers * 2 * 4);
@@ -183,7 +187,7 @@ int qevict::choose_splits(const qevict_ctx* h, int n_units) {
     const int f = h->forced_splits < smin ? smin : h->forced_splits;
     return f < MAX_SPLITS ? f : MAX_SPLITS;
   }
-  const int entries = g.Kf + g.Kq + 1;
+  const int entries = g.Kfp + g.Kq + 1;
   const long pairs = (long)n_units * g.Hkv;
   const long slots = (long)h->sm_count * 3;  // resident CTAs
   int best = smin;
@@ -241,7 +245,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   int e_bound = 1;  // upper bound of every unit's work-list length, from the host's mirror of the window counts
   for (int l = l0; l < l1; ++l) {
     const LayerMirror& m = h->layers[l];
-    const int e = g.Kf + g.Kq + m.aged + (m.has_open ? 1 : 0);
+    const int e = g.Kfp + g.Kq + m.aged + (m.has_open ? 1 : 0);
     if (e > e_bound) e_bound = e;
   }
   QE_CUDA(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
@@ -414,9 +418,9 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   const int n_prompt = ctx_tokens / g.W;
   QE_CUDA(h, launch_prefill_init(a, n_prompt, window_scores, s));
   QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
-  QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kf, s));
+  QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kfp, s));
   QE_CUDA(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));
-  h->launches += 2 + (g.Kf > 0) + (g.Kq > 0);
+  h->launches += 2 + (g.Kfp > 0) + (g.Kq > 0);
   for (int l = l0; l < l1; ++l) {
     h->layers[l].prefilled = true;
     h->layers[l].n_windows = n_prompt;
@@ -465,7 +469,7 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   QE_CUDA(h, cudaSetDevice(h->cfg.device));
   cudaStream_t s = (cudaStream_t)stream;
   const KernelArgs a = make_args(h, l0, l1);
-  QE_CUDA(h, timed_launch(h, 3, s, [&] { return launch_route(a, 0, next_pow2(g.Kf + g.Kq + g.aged_cap + 1), s); }));
+  QE_CUDA(h, timed_launch(h, 3, s, [&] { return launch_route(a, 0, next_pow2(g.Kfp + g.Kq + g.aged_cap + 1), s); }));
   // quantizations and promotions of the event in one launch (linked where they share a page)
   const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
   const int max_items = (g.Kq > 0 ? g.PF : 0) + max_promote;
@@ -500,6 +504,7 @@ QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict
       case QEVICT_TIER_AGED: out->n_aged++; break;
       case QEVICT_TIER_OPEN: out->n_open++; break;
       case QEVICT_TIER_EVICTED: out->n_evicted++; break;
+      case QEVICT_TIER_SINK: out->n_sink++; break;
       default: break;
     }
   }

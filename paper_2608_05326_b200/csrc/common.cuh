@@ -37,6 +37,8 @@ struct Geometry {
   int PF, PQ;    // pages per unit in the full-precision / quantized pool
   int EMAX;      // max entries of a unit's work list
   int aged_cap;  // filled windows that may wait for a routing event
+  int n_sink, n_recent;  // protected windows: sink prefix, recent region (besides the open window)
+  int Kfp;       // K_f + n_sink + n_recent: windows that may need a full-precision page in one event
   int tiles;     // W / 32
   // full-precision page: [H_kv][tile]{K tile, V tile}, each tile 32 x D elements, fragment-major
   uint32_t fp_tile_bytes, fp_head_bytes, fp_page_bytes;

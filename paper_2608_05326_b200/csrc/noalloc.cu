@@ -105,7 +105,7 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   int e_bound = 1;
   for (int l = l0; l < l1; ++l) {
     const LayerMirror& m = h->layers[l];
-    const int eb = g.Kf + g.Kq + m.aged + (m.has_open ? 1 : 0);
+    const int eb = g.Kfp + g.Kq + m.aged + (m.has_open ? 1 : 0);
     if (eb > e_bound) e_bound = eb;
   }
   e = launch_combine(a, p.S, e_bound, out, stream);

@@ -345,7 +345,7 @@ __global__ void __launch_bounds__(PAGE_THREADS) copy_prompt_kernel(const KernelA
   const int ul = blockIdx.z, u = a.unit0 + ul, hk = blockIdx.y;
   const int n_items = a.st.n_copy[u];
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-  const int4 it = a.st.copy_list[(size_t)u * g.Kf + item];
+  const int4 it = a.st.copy_list[(size_t)u * g.Kfp + item];
   const int w = it.x, dst = it.y, D = g.D;
   const T* kr = k_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * g.W) * D;
   const T* vr = v_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * g.W) * D;

@@ -220,7 +220,7 @@ __global__ void prefill_init_kernel(const KernelArgs a, int n_prompt, const floa
   const int w = blockIdx.x * blockDim.x + threadIdx.x;
   if (w < n_prompt) {
     const size_t wi = (size_t)u * g.NW + w;
-    a.st.tier[wi] = QEVICT_TIER_AGED;
+    a.st.tier[wi] = w < g.n_sink ? QEVICT_TIER_SINK : QEVICT_TIER_AGED;
     a.st.importance[wi] = scores[(size_t)ul * n_prompt + w];
   }
   if (w == 0) a.st.n_windows[u] = n_prompt;
@@ -231,8 +231,16 @@ __global__ void prefill_init_kernel(const KernelArgs a, int n_prompt, const floa
 // order into shared memory together with the two page-owner tables; ranking, tier assignment, page
 // release and allocation, migration lists and the decode work list all run on those shared copies, and
 // the tables go back to global memory once at the end.  Global memory is waited on three times.
-__device__ __forceinline__ bool is_candidate(uint8_t t) {
-  return t == QEVICT_TIER_FULL || t == QEVICT_TIER_QUANT || t == QEVICT_TIER_AGED;
+// A window is gathered by a routing event if it is a candidate (Full, Quantized, or filled and out of the
+// protected recent region) or pinned (sink prefix, or filled and still inside the recent region: windows
+// recent_lo and above).  Pinned windows keep their state; they are gathered because they are part of the
+// decode work list and, at prefill, need a full-precision page like the Full windows.
+constexpr uint8_t PINNED = 0x80;  // flag in the new-state byte of a gathered window
+__device__ __forceinline__ bool is_candidate(uint8_t t, int w, int recent_lo) {
+  return t == QEVICT_TIER_FULL || t == QEVICT_TIER_QUANT || (t == QEVICT_TIER_AGED && w < recent_lo);
+}
+__device__ __forceinline__ bool is_pinned(uint8_t t, int w, int recent_lo) {
+  return t == QEVICT_TIER_SINK || (t == QEVICT_TIER_AGED && w >= recent_lo);
 }
 
 __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a, int prefill, int sort_cap) {
@@ -275,17 +283,21 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) ofp[i] = fp_owner[i];
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) oq[i] = q_owner[i];
 
-  // ---- gather the candidates in ascending window order ----------------------------------------------
-  auto emit_candidate = [&](int w, int k, uint8_t t) {
+  // ---- gather the candidates and the pinned windows in ascending window order -------------------------
+  const int recent_lo = nw - (ow >= 0 ? 1 : 0) - g.n_recent;
+  auto emit_gathered = [&](int w, int k, uint8_t t) {
     if (k >= sort_cap) return;
+    const bool pin = is_pinned(t, w, recent_lo);
     cw[k] = w;
     ctier[k] = t;
     cled[k] = ledger[w];
     cfp[k] = fp_page[w];
     cq[k] = q_page[w];
-    keys[k] = ((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)k;
+    if (pin) cnew[k] = PINNED | t;
+    // pinned windows get the largest keys: they are never counted among the smaller keys of a candidate
+    keys[k] = pin ? (0xFFFFFFFF00000000ull | (uint32_t)k) : (((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)k);
   };
-  int n_all;
+  int n_all, n_real;
   const int chunk = (nw + ROUTE_THREADS - 1) / ROUTE_THREADS;
   if (chunk <= 16) {
     // every thread reads its (up to 16) window states in one go and keeps them in registers
@@ -293,18 +305,32 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     const int b = tid * chunk;
 #pragma unroll
     for (int k = 0; k < 16; ++k) tc[k] = (k < chunk && b + k < nw) ? tier[b + k] : (uint8_t)QEVICT_TIER_NONE;
-    int cnt = 0;
-#pragma unroll
-    for (int k = 0; k < 16; ++k) cnt += is_candidate(tc[k]) ? 1 : 0;
-    int rank = block_exclusive_scan(cnt, scratch, &n_all);
+    int cnt = 0;  // gathered | candidates << 16
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
-      if (is_candidate(tc[k])) emit_candidate(b + k, rank++, tc[k]);
+      const bool c = is_candidate(tc[k], b + k, recent_lo);
+      cnt += (c || is_pinned(tc[k], b + k, recent_lo) ? 1 : 0) + (c ? 0x10000 : 0);
+    }
+    int tot;
+    int rank = block_exclusive_scan(cnt, scratch, &tot) & 0xFFFF;
+    n_all = tot & 0xFFFF; n_real = tot >> 16;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if (is_candidate(tc[k], b + k, recent_lo) || is_pinned(tc[k], b + k, recent_lo)) emit_gathered(b + k, rank++, tc[k]);
     }
     __syncthreads();
   } else {
-    n_all = block_compact(nw, scratch, [&](int w) { return is_candidate(tier[w]); },
-                          [&](int w, int k) { emit_candidate(w, k, tier[w]); });
+    int* s_real = scratch + 103;
+    if (tid == 0) *s_real = 0;
+    __syncthreads();
+    n_all = block_compact(nw, scratch,
+                          [&](int w) { const uint8_t t = tier[w]; return is_candidate(t, w, recent_lo) || is_pinned(t, w, recent_lo); },
+                          [&](int w, int k) {
+                            const uint8_t t = tier[w];
+                            if (is_candidate(t, w, recent_lo)) atomicAdd(s_real, 1);
+                            emit_gathered(w, k, t);
+                          });
+    n_real = *s_real;
   }
   const int n_cand = min(n_all, sort_cap);
 
@@ -314,6 +340,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     // rank of a key = number of smaller keys (all keys are distinct)
     for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
       const unsigned long long mine = keys[c];
+      if ((uint32_t)(mine >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
       int pos = 0;
       for (int i = 0; i < n_cand; ++i) pos += keys[i] < mine ? 1 : 0;
       cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
@@ -323,7 +350,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     // K_f-th and the (K_f + K_q)-th smallest key, both in the same six passes (four 8-bit digits of the
     // score, two of the candidate index).  thr[j] = the selected key: a candidate belongs to the first
     // K_j exactly if its key is <= thr[j].
-    const int kk[2] = {min(g.Kf, n_cand), min(g.Kf + g.Kq, n_cand)};
+    const int n_rk = min(n_real, n_cand);  // candidates (the pinned windows hold the largest keys)
+    const int kk[2] = {min(g.Kf, n_rk), min(g.Kf + g.Kq, n_rk)};
     int* hist = rhist;                                   // [2][256]
     uint32_t* sel = reinterpret_cast<uint32_t*>(scratch + 104);  // [2][2] selected prefixes {low, high word}
     int* need = scratch + 108;                           // [2] rank still to find inside the current bucket
@@ -375,6 +403,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     const unsigned long long t0 = ((unsigned long long)sel[1] << 32) | sel[0], t1 = ((unsigned long long)sel[3] << 32) | sel[2];
     for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
       const unsigned long long key = keys[c];
+      if ((uint32_t)(key >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
       cnew[c] = (kk[0] > 0 && key <= t0) ? QEVICT_TIER_FULL : ((kk[1] > 0 && key <= t1) ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
     }
   }
@@ -399,7 +428,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   // free quantized pages, first demotions (need a quantized page), windows entering the Full tier without
   // a page (promotions; prompt windows at prefill), and the Full / Quantized members of the work list ----
   auto q_needs = [&](int c) { return cnew[c] == QEVICT_TIER_QUANT && ctier[c] != QEVICT_TIER_QUANT && cled[c] == QEVICT_LEDGER_NONE; };
-  auto fp_needs = [&](int c) { return cnew[c] == QEVICT_TIER_FULL && ctier[c] != QEVICT_TIER_FULL && cfp[c] < 0; };
+  auto fp_needs = [&](int c) {
+    return ((cnew[c] == QEVICT_TIER_FULL && ctier[c] != QEVICT_TIER_FULL) || (cnew[c] & PINNED)) && cfp[c] < 0;
+  };
+  auto lists_as_full = [&](int c) { return cnew[c] == QEVICT_TIER_FULL || (cnew[c] & PINNED); };
   int32_t* need_q = reinterpret_cast<int32_t*>(keys);  // the sort keys are dead from here on
   int32_t* need_fp = need_q + sort_cap;
   const int ch_f = (g.PF + ROUTE_THREADS - 1) / ROUTE_THREADS, ch_q = (g.PQ + ROUTE_THREADS - 1) / ROUTE_THREADS;
@@ -411,7 +443,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   for (int pg = bq; pg < eq; ++pg) cnt.x += oq[pg] < 0 ? 0x10000 : 0;
   for (int c = bc; c < ec; ++c) {
     cnt.y += (q_needs(c) ? 1 : 0) + (fp_needs(c) ? 0x10000 : 0);
-    cnt.z += (cnew[c] == QEVICT_TIER_FULL ? 1 : 0) + (cnew[c] == QEVICT_TIER_QUANT ? 0x10000 : 0);
+    cnt.z += (lists_as_full(c) ? 1 : 0) + (cnew[c] == QEVICT_TIER_QUANT ? 0x10000 : 0);
   }
   int3 tot;
   int3 rk = block_exclusive_scan3(cnt, scratch, &tot);
@@ -427,12 +459,12 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     for (int c = bc; c < ec; ++c) {
       if (q_needs(c)) need_q[r0++] = c;
       if (fp_needs(c)) need_fp[r1++] = c;
-      if (cnew[c] == QEVICT_TIER_FULL) { if (r2 < g.EMAX) flist[r2] = c; ++r2; }
+      if (lists_as_full(c)) { if (r2 < g.EMAX) flist[r2] = c; ++r2; }
       if (cnew[c] == QEVICT_TIER_QUANT) { if (n_f + r3 < g.EMAX) qlist[r3] = c; ++r3; }
     }
   }
   const int qcap = g.PF + g.Kq;
-  const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, g.Kf));
+  const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, prefill ? g.Kfp : g.Kf));
   const int n_items = nq + (prefill ? 0 : nfp);
   int* s_base = scratch + 102;
   if (tid == 0) {
@@ -458,7 +490,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   // windows entering the Full tier take the free full-precision pages in ascending order.  A promotion
   // that receives a page some quantization of this event still has to read is linked to that quantization
   // (the migration kernel runs it right after it, in the same warps).
-  int4* copy_list = a.st.copy_list + (size_t)u * g.Kf;
+  int4* copy_list = a.st.copy_list + (size_t)u * g.Kfp;
   for (int k = tid; k < nfp; k += ROUTE_THREADS) {
     const int c = need_fp[k], pg = free_fp[k];
     ofp[pg] = cw[c];
@@ -477,6 +509,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
     const uint8_t old = ctier[c], nt = cnew[c];
     const int w = cw[c];
+    if (nt & PINNED) {  // state unchanged; at prefill the window has just received its page
+      fp_page[w] = cfp[c];
+      continue;
+    }
     if (nt == QEVICT_TIER_FULL) {
       if (old == QEVICT_TIER_QUANT) cled[c] = QEVICT_LEDGER_DORMANT;  // codes retained for a later demotion
     } else if (nt == QEVICT_TIER_QUANT) {

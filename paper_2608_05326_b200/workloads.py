@@ -42,6 +42,8 @@ class Workload:
     outlier_channels: int = 0
     outlier_scale: float = 1.0
     seed: int = BASE_SEED
+    sink_windows: int = 0    # protected sink prefix (windows)
+    recent_windows: int = 0  # filled windows kept in the protected recent region
 
     @property
     def n_units(self):

@@ -10,7 +10,7 @@ page tables, ledger flags, codes, parameters, promoted page contents -- must mat
 import numpy as np
 import torch
 
-from oracle import (LEDGER_NONE, TIER_AGED, TIER_FULL, TIER_OPEN, TIER_QUANT, OracleConfig, UnitOracle,
+from oracle import (LEDGER_NONE, TIER_AGED, TIER_FULL, TIER_OPEN, TIER_QUANT, TIER_SINK, OracleConfig, UnitOracle,
                     accessible_attention)
 from paper_2608_05326_b200 import binding, workloads
 
@@ -20,7 +20,8 @@ MASS_RTOL = 1e-4                    # window scores / per-step mass
 
 def oracle_config(wl, aged_windows):
     return OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
-                        wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged_windows)
+                        wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged_windows,
+                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
 
 
 def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
@@ -28,7 +29,7 @@ def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
     return binding.make_config(wl.batch if batch is None else batch, wl.n_layers if n_layers is None else n_layers,
                                wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits,
                                wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
-                               rebalance_interval_hint=r)
+                               rebalance_interval_hint=r, sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
 
 
 def aged_capacity(wl, rebalance_interval=None):
@@ -78,7 +79,7 @@ def compare_state(cache, layer, seq, orc, wl, check_pages=None, what=""):
             what, name, bad[:8], got[bad[:8]], ref[:n][bad[:8]])
     windows = range(n) if check_pages is None else check_pages
     for w in windows:
-        if orc.fp_page[w] >= 0 and orc.tier[w] in (TIER_FULL, TIER_AGED, TIER_OPEN):
+        if orc.fp_page[w] >= 0 and orc.tier[w] in (TIER_FULL, TIER_AGED, TIER_OPEN, TIER_SINK):
             k, v = cache.export_fp_page(layer, seq, int(orc.fp_page[w]))
             rk, rv = orc.fp[w]
             if orc.tier[w] == TIER_OPEN:
@@ -196,7 +197,7 @@ class LockstepRun:
             orc.rebalance()
             t0, l0 = before[u]
             changed[u] = [int(w) for w in np.flatnonzero((t0 != orc.tier) | (l0 != orc.ledger_flag))
-                          if orc.tier[w] in (TIER_FULL, TIER_QUANT)]
+                          if orc.tier[w] in (TIER_FULL, TIER_QUANT, TIER_SINK)]
         self.check_state("all" if full_check else changed, what="after rebalance at step %d" % self.step_idx)
 
     def _rebalance_free(self):

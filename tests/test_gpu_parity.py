@@ -92,6 +92,33 @@ def test_free_running_routes_identically_or_flips_only_at_a_cut(cfg):
     run.close()
 
 
+@pytest.mark.parametrize("kw", [
+    dict(sink_windows=2, recent_windows=3),
+    dict(sink_windows=1, recent_windows=0, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, quant_bits=2),
+    dict(sink_windows=0, recent_windows=2, window=64, group_size=64, context=2048, head_dim=128, n_q_heads=8, n_kv_heads=1,
+         dtype="bf16"),
+], ids=lambda kw: "-".join("%s%s" % (k[0], v) for k, v in kw.items()))
+def test_protected_sink_and_recent_windows(kw):
+    # the sink prefix and the recent region stay in full precision outside K_f and never become candidates;
+    # filled windows turn into candidates only when newer windows have pushed them out of the recent region
+    ls = _lockstep()
+    w = kw.get("window", 32)
+    wl = _small("protected", steps=4 * w + 7, **kw)
+    for interval in (1, 5):
+        run = ls.LockstepRun(wl, rebalance_interval=interval)
+        run.check_state("all", "after prefill")
+        st = run.cache.stats()
+        assert st["n_sink"] == wl.sink_windows and st["n_aged"] == wl.recent_windows
+        assert (st["n_full"], st["n_quant"]) == (wl.fp_budget_windows, wl.q_budget_windows)
+        for _ in range(wl.steps):
+            run.step(append=True)
+        run.rebalance(full_check=True)
+        st = run.cache.stats()
+        assert st["n_sink"] == wl.sink_windows and st["n_aged"] == wl.recent_windows
+        assert st["deletions"] == run.oracles[0].stats["deletions"] > 0
+        run.close()
+
+
 def test_many_candidates_and_tied_scores():
     # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
     # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides
