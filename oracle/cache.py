@@ -9,6 +9,8 @@ Paper basis:
   * write-once ledger (quantize on the first demotion only, dormant on
     promotion, reactivated on a later demotion, deleted on eviction):
     "Migration-Stable Quantization" and Algorithm 1;
+  * alternative ranking functions (exponentially decayed attention, attention
+    p-norm): the ranking-function appendix, Eqs. for u_t(w), S_decay and S_p;
   * capacities K_f, K_q from a byte budget: the tier-capacity equation of
     "Byte-Constrained Tier Allocation"; per-window byte costs: the memory
     accounting appendix.
@@ -34,6 +36,16 @@ Readings taken where the paper is silent (each is listed in the design notes):
     routing event, windows that need a page take the free page ids in ascending
     order, in ascending window index; a newly opened window takes the lowest
     free full-precision page.
+
+Ranking variants (rank_mode 1, 2): the mass a window receives is collected in an
+event accumulator u (raw sum over heads, like the score) and folded into the score at
+every routing event after prefill, for every window that is still stored:
+    decayed:  S <- RN32(RN32(lambda * S) + u)
+    p-norm:   P <- RN32(P + u^p), u^p by p-1 float32 multiplications; windows are ranked
+              by P, which orders them as S_p = P^(1/p) does
+in float32 with every operation rounded separately, so that the ranking -- an integer
+decision taken on floating point -- is taken on the same numbers by any implementation.
+The prefill scores initialise S (or P) directly.
 
 Parity unpinned: the page-id assignment order above is this build's own rule (the
 paper never speaks of pages), so nothing outside this file fixes it; and the
@@ -70,6 +82,8 @@ class OracleConfig:
     aged_windows: int = 2  # filled windows that may wait for the next routing event
     softmax_scale: float = 0.0  # 0 => 1/sqrt(head_dim)
     sink_windows: int = 0  # protected sink prefix, in windows
+    rank_mode: int = 0  # 0 cumulative attention (Eq. 1), 1 exponentially decayed, 2 attention p-norm
+    rank_param: float = 0.0  # lambda of the decayed score, p of the p-norm (integer >= 2)
     recent_windows: int = 0  # filled windows kept in the protected recent region
 
     @property
@@ -125,6 +139,7 @@ class UnitOracle:
         self.fp_page = np.full(n, -1, dtype=np.int32)
         self.q_page = np.full(n, -1, dtype=np.int32)
         self.importance = np.zeros(n, dtype=np.float64)
+        self.event_mass = np.zeros(n, dtype=np.float64)  # u: mass since the last routing event (rank_mode 1, 2)
         self.fp = {}  # window -> (k, v) [H_kv, W, d] float64 in the execution datatype
         self.ledger = {}  # window -> dict of codes and params
         self.fp_owner = np.full(cfg.fp_pool_pages, -1, dtype=np.int32)
@@ -156,7 +171,7 @@ class UnitOracle:
             self.tier[w] = TIER_SINK if w < cfg.sink_windows else TIER_AGED
             self.importance[w] = float(window_scores[w])
         self.n_windows = n
-        self.rebalance()
+        self.rebalance(prefill=True)
 
     # --------------------------------------------------------------- append
     def _append(self, k_new, v_new):
@@ -227,7 +242,10 @@ class UnitOracle:
         for w, _, _, n in acc:
             mass[w] = probs[:, pos : pos + n].sum()
             pos += n
-        self.importance += mass
+        if cfg.rank_mode == 0:
+            self.importance += mass
+        else:
+            self.event_mass += mass
         self.stats["steps"] += 1
         return round_to_dtype(out, cfg.dtype), mass
 
@@ -249,9 +267,29 @@ class UnitOracle:
         order = np.lexsort((cand, -s32.astype(np.float64)))
         return cand[order]
 
-    def rebalance(self):
+    def fold_event_mass(self):
+        """Ranking-function appendix: S_decay <- lambda S_decay + u and S_p^p <- S_p^p + u^p at a routing
+        event, for every stored window; float32, each operation rounded on its own."""
+        cfg = self.cfg
+        t = self.tier[: self.n_windows]
+        live = np.flatnonzero((t != TIER_NONE) & (t != TIER_EVICTED))
+        s = self.importance[live].astype(np.float32)
+        u = self.event_mass[live].astype(np.float32)
+        if cfg.rank_mode == 1:
+            s = np.float32(cfg.rank_param) * s + u  # numpy rounds the product, then the sum, to float32
+        else:
+            v = u.copy()
+            for _ in range(int(cfg.rank_param) - 1):
+                v = v * u
+            s = s + v
+        self.importance[live] = s.astype(np.float64)
+        self.event_mass[live] = 0.0
+
+    def rebalance(self, prefill=False):
         """Algorithm 1: TopK partition of the candidates, then promote / demote / evict with the ledger."""
         cfg = self.cfg
+        if cfg.rank_mode != 0 and not prefill:
+            self.fold_event_mass()
         ranked = self.ranked_candidates()
         k_f, k_q = cfg.fp_budget_windows, cfg.q_budget_windows
         new_f = ranked[:k_f]

@@ -170,6 +170,70 @@ def test_protected_regions_with_full_budget_equal_brute_force_attention():
             assert u.tier_counts()["evicted"] == 0 and u.tier_counts()["quant"] == 0
 
 
+# ------------------------------------------------------------------- alternative ranking functions
+def _rank_cfg(mode, param, k_f=3, k_q=4):
+    return OracleConfig(4, 2, 64, "fp16", 32, 4, 32, k_f, k_q, 28 * 32, aged_windows=2, rank_mode=mode, rank_param=param)
+
+
+@pytest.mark.parametrize("mode,param", [(1, 0.9), (2, 3.0)])
+def test_ranking_variants_follow_their_recurrences(mode, param):
+    """S_decay(t) = lambda S_decay(t - Omega) + u_t and S_p = (sum_r u_r^p)^(1/p): the oracle's scores are
+    recomputed here in float64 from the per-step masses it returned, event by event."""
+    rng = np.random.default_rng(41)
+    cfg = _rank_cfg(mode, param, k_f=32, k_q=4)  # nothing is evicted: every window keeps a full history
+    scores = rng.random(16).astype(np.float32)
+    u, k, v, _ = _prefilled(cfg, rng, scores=scores)
+    ref = np.zeros(cfg.max_windows)
+    ref[:16] = scores
+    acc = np.zeros(cfg.max_windows)
+    for t in range(45):
+        q = _rand_T(rng, (cfg.n_q_heads, cfg.head_dim), cfg.dtype)
+        kn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+        vn = _rand_T(rng, (cfg.n_kv_heads, cfg.head_dim), cfg.dtype)
+        _, mass = u.decode_attn(q, kn, vn)
+        acc += mass
+        if t % 4 == 3:  # a routing event every 4 steps: u_t sums 4 steps
+            u.rebalance()
+            live = np.arange(u.n_windows)
+            if mode == 1:
+                ref[live] = param * ref[live] + acc[live]
+            else:
+                ref[live] = ref[live] + acc[live] ** param
+            acc[:] = 0.0
+            assert np.allclose(u.importance[: u.n_windows], ref[: u.n_windows], rtol=2e-6, atol=1e-12)
+            assert np.all(u.event_mass == 0.0)
+    if mode == 2:  # the stored quantity is S_p^p; S_p itself is its p-th root
+        s_p = u.importance[: u.n_windows] ** (1.0 / param)
+        assert np.allclose(s_p, ref[: u.n_windows] ** (1.0 / param), rtol=1e-6)
+
+
+def test_decay_forgets_and_pnorm_prefers_peaks():
+    """What distinguishes the variants: with equal total mass, the decayed score ranks the window attended
+    recently above the one attended long ago, and the p-norm ranks a window attended in one burst above one
+    attended evenly; the cumulative score cannot separate either pair."""
+    for mode, param in ((0, 0.0), (1, 0.5), (2, 3.0)):
+        cfg = _rank_cfg(mode, param, k_f=32, k_q=4)
+        u = UnitOracle(cfg)
+        u.n_windows = 4
+        u.tier[:4] = TIER_FULL
+        # per-event masses of windows 0..3 over 4 events: early, late, burst, even (total 4 each)
+        events = np.array([[4, 0, 0, 0], [0, 0, 0, 4], [0, 4, 0, 0], [1, 1, 1, 1]], dtype=np.float64).T
+        for e in events:
+            if mode == 0:
+                u.importance[:4] += e
+            else:
+                u.event_mass[:4] = e
+                u.fold_event_mass()
+        s = u.importance[:4]
+        if mode == 0:
+            assert s[0] == s[1] == s[2] == s[3] == 4.0
+        elif mode == 1:
+            assert s[1] > s[3] > s[0]            # late > even > early
+            assert s[1] == 4.0 and s[0] == 4.0 * 0.5 ** 3
+        else:
+            assert s[0] == s[1] == s[2] == 64.0 and s[3] == 4.0   # one burst: 4^3; even: 4 x 1^3
+
+
 def test_no_protected_regions_is_the_default():
     rng = np.random.default_rng(33)
     a, k, v, s = _prefilled(_small_cfg(), rng)
