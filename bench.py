@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--rebalance-interval", type=int, default=1)
     ap.add_argument("--sink-windows", type=int, default=0, help="protected sink prefix, in windows (0 in every BASELINE config)")
     ap.add_argument("--recent-windows", type=int, default=0, help="filled windows kept in the protected recent region")
+    ap.add_argument("--rank-mode", type=int, default=0, help="0 cumulative attention (Eq. 1), 1 decayed, 2 p-norm")
+    ap.add_argument("--rank-param", type=float, default=0.0, help="lambda of the decayed score / p of the p-norm")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -72,7 +74,8 @@ def make_workload(args, total_steps):
     layers = args.layers if args.layers is not None else (32 if args.config == 1 else (8 if args.config == 3 else wl.n_layers))
     batch = args.batch if args.batch is not None else wl.batch
     return replace(wl, n_layers=layers, batch=batch, steps=total_steps, rebalance_interval=args.rebalance_interval,
-                   sink_windows=args.sink_windows, recent_windows=args.recent_windows)
+                   sink_windows=args.sink_windows, recent_windows=args.recent_windows, rank_mode=args.rank_mode,
+                   rank_param=args.rank_param)
 
 
 def peak_hbm_gbs():
@@ -194,7 +197,8 @@ def run_ours(args, rank, world):
     cfg = binding.make_config(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window,
                               wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
                               rebalance_interval_hint=args.rebalance_interval, device=dev.index,
-                              sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
+                              sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
+                              rank_param=wl.rank_param)
     cache = binding.QEvictCache(cfg)
     if args.splits:
         cache.set_splits(args.splits)
@@ -328,7 +332,8 @@ def time_oracle(wl, n_steps, warmup, budget_s):
     aged = (wl.rebalance_interval + wl.window - 1) // wl.window + 1
     ocfg = OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
                         wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged,
-                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
+                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
+                        rank_param=wl.rank_param)
     k, v = workloads.gen_prompt_kv(wl, 0)
     s = workloads.place_planted(workloads.synthetic_window_scores(wl, 0), workloads.planted_windows(wl, 0),
                                 wl.fp_budget_windows, wl.q_budget_windows)

@@ -72,6 +72,12 @@ enum {
   QEVICT_TIER_EVICTED = 5,
   QEVICT_TIER_SINK = 6     /* protected sink prefix: full precision, never a candidate */
 };
+/* ranking functions.  CUMULATIVE is Eq. 1 (mass added to the score at every step).  With the other two
+ * the mass is collected in an event accumulator u and folded into the score by every routing event after
+ * prefill, for every stored window, in float32 with each operation rounded on its own:
+ *   DECAYED  S <- lambda * S + u;   PNORM  P <- P + u^p (p - 1 multiplications); windows are ranked by
+ *   P, which orders them as S_p = P^(1/p) does.  The prefill scores initialise S (or P) directly. */
+enum { QEVICT_RANK_CUMULATIVE = 0, QEVICT_RANK_DECAYED = 1, QEVICT_RANK_PNORM = 2 };
 /* ledger states */
 enum { QEVICT_LEDGER_NONE = 0, QEVICT_LEDGER_ACTIVE = 1, QEVICT_LEDGER_DORMANT = 2 };
 
@@ -99,6 +105,8 @@ typedef struct {
                                 most recently filled windows stay in full precision and are not candidates
                                 until newer windows push them out [candidate pool: windows that have exited
                                 the recent region] */
+  int32_t rank_mode;         /* QEVICT_RANK_*: which score orders the candidates [ranking-function appendix] */
+  float rank_param;          /* lambda of the decayed score (0 < lambda <= 1); p of the p-norm (integer 2..8) */
 } qevict_config;
 
 typedef struct {
@@ -217,6 +225,11 @@ QEVICT_API qevict_status qevict_export_fp_page(qevict_handle h, int32_t layer, i
 QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, int32_t seq, int32_t q_page,
                                    uint8_t* k_codes, void* k_params, uint8_t* v_codes, void* v_params,
                                    void* stream);
+
+/* The event accumulator u of a unit (rank_mode DECAYED or PNORM): float32 [max_context / W], DEVICE
+ * buffer; all zeros right after a routing event. */
+QEVICT_API qevict_status qevict_export_event_mass(qevict_handle h, int32_t layer, int32_t seq, float* event_mass,
+                                                  void* stream);
 
 /* Tuning: force the number of KV splits per (unit, KV head) of the decode kernel (1..64); 0 restores
  * the built-in choice, which fills the GPU in whole waves.  Results do not depend on it beyond

@@ -30,6 +30,7 @@ class qevict_config(C.Structure):
         ("quant_bits", C.c_int32), ("group_size", C.c_int32), ("fp_budget_windows", C.c_int32),
         ("q_budget_windows", C.c_int32), ("max_context", C.c_int32), ("rebalance_interval_hint", C.c_int32),
         ("softmax_scale", C.c_float), ("device", C.c_int32), ("sink_windows", C.c_int32), ("recent_windows", C.c_int32),
+        ("rank_mode", C.c_int32), ("rank_param", C.c_float),
     ]
 
 
@@ -52,6 +53,7 @@ _SIGNATURES = {
     "qevict_create": (C.c_int, [C.POINTER(qevict_config), C.c_void_p, C.c_uint64, C.POINTER(C.c_void_p)]),
     "qevict_destroy": (C.c_int, [C.c_void_p]),
     "qevict_set_splits": (C.c_int, [C.c_void_p, C.c_int32]),
+    "qevict_export_event_mass": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32]),
     "qevict_kernel_time": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
     "qevict_kernel_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
@@ -92,11 +94,12 @@ def _check(status, handle=None):
 
 def make_config(batch, n_layers, n_q_heads, n_kv_heads, head_dim, dtype, window, quant_bits, group_size,
                 fp_budget_windows, q_budget_windows, max_context, rebalance_interval_hint=0, softmax_scale=0.0,
-                device=0, sink_windows=0, recent_windows=0):
+                device=0, sink_windows=0, recent_windows=0, rank_mode=0, rank_param=0.0):
     dt = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, torch.float16: DTYPE_FP16, torch.bfloat16: DTYPE_BF16}[dtype]
     return qevict_config(C.sizeof(qevict_config), batch, n_layers, n_q_heads, n_kv_heads, head_dim, dt, window,
                          quant_bits, group_size, fp_budget_windows, q_budget_windows, max_context,
-                         rebalance_interval_hint, softmax_scale, device, sink_windows, recent_windows)
+                         rebalance_interval_hint, softmax_scale, device, sink_windows, recent_windows, rank_mode,
+                         rank_param)
 
 
 # --- plain function wrappers, same names as the C entry points -----------------------------------------
@@ -280,6 +283,11 @@ class QEvictCache:
     def export_last_mass(self, layer, seq):
         m = torch.zeros(self.max_windows, dtype=torch.float32, device=self.device)
         _check(lib().qevict_export_last_mass(self.handle, layer, seq, _ptr(m), _stream(None)), self.handle)
+        return m.cpu()
+
+    def export_event_mass(self, layer, seq):
+        m = torch.zeros(self.max_windows, dtype=torch.float32, device=self.device)
+        _check(lib().qevict_export_event_mass(self.handle, layer, seq, _ptr(m), _stream(None)), self.handle)
         return m.cpu()
 
     def export_fp_page(self, layer, seq, page):

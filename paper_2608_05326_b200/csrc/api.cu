@@ -71,6 +71,10 @@ const char* validate(const qevict_config* c) {
   if (c->window < 1 || c->max_context < c->window || c->max_context % c->window) return "max_context must be a positive multiple of window";
   if (c->group_size < 1 || c->window % c->group_size || c->head_dim % c->group_size) return "group_size must divide window and head_dim";
   if (c->rebalance_interval_hint < 0) return "rebalance_interval_hint < 0";
+  if (c->rank_mode < QEVICT_RANK_CUMULATIVE || c->rank_mode > QEVICT_RANK_PNORM) return "rank_mode must be a QEVICT_RANK_* value";
+  if (c->rank_mode == QEVICT_RANK_DECAYED && !(c->rank_param > 0.f && c->rank_param <= 1.f)) return "decayed ranking needs 0 < rank_param <= 1";
+  if (c->rank_mode == QEVICT_RANK_PNORM && !(c->rank_param >= 2.f && c->rank_param <= 8.f && c->rank_param == floorf(c->rank_param)))
+    return "p-norm ranking needs an integer rank_param in 2..8";
   if (c->sink_windows < 0 || c->recent_windows < 0) return "sink_windows and recent_windows must be >= 0";
   if (c->sink_windows + c->recent_windows > c->max_context / c->window) return "protected windows exceed max_context";
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return "softmax_scale must be finite and >= 0";
@@ -96,6 +100,7 @@ void make_geometry(const qevict_config& c, Geometry& g) {
   const int r = c.rebalance_interval_hint > 0 ? c.rebalance_interval_hint : c.window;
   g.aged_cap = (r + g.W - 1) / g.W + 1;
   g.n_sink = c.sink_windows; g.n_recent = c.recent_windows;
+  g.rank_mode = c.rank_mode; g.rank_param = c.rank_param;
   g.Kfp = g.Kf + g.n_sink + g.n_recent;
   g.PF = g.Kfp + g.aged_cap + 1;
   g.PQ = g.Kq + g.Kf;
@@ -133,6 +138,7 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.fp_page = (int32_t*)take(U * g.NW * 4);
   s.q_page = (int32_t*)take(U * g.NW * 4);
   s.importance = (float*)take(U * g.NW * 4);
+  s.event_mass = (float*)take(U * g.NW * 4);
   s.fp_owner = (int32_t*)take(U * g.PF * 4);
   s.q_owner = (int32_t*)take(U * g.PQ * 4);
   s.n_windows = (int32_t*)take(U * 4);
@@ -334,6 +340,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
     if (e == cudaSuccess) e = cudaMemset(h->st.fp_page, 0xFF, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.q_page, 0xFF, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.importance, 0, U * g.NW * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.event_mass, 0, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.fp_owner, 0xFF, U * g.PF * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.q_owner, 0xFF, U * g.PQ * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.n_windows, 0, U * 4);
@@ -538,6 +545,16 @@ QEVICT_API qevict_status qevict_export_tables(qevict_handle h, int32_t layer, in
   if (fp_page) QE_CUDA(h, cudaMemcpyAsync(fp_page, h->st.fp_page + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
   if (q_page) QE_CUDA(h, cudaMemcpyAsync(q_page, h->st.q_page + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
   if (importance) QE_CUDA(h, cudaMemcpyAsync(importance, h->st.importance + o, (size_t)g.NW * 4, cudaMemcpyDeviceToDevice, s));
+  return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_export_event_mass(qevict_handle h, int32_t layer, int32_t seq, float* event_mass, void* stream) {
+  if (!h || !event_mass) return QEVICT_ERR_INVALID_ARG;
+  int u;
+  if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_CUDA(h, cudaMemcpyAsync(event_mass, h->st.event_mass + (size_t)u * h->geo.NW, (size_t)h->geo.NW * 4,
+                             cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return QEVICT_OK;
 }
 

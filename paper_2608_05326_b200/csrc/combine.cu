@@ -94,12 +94,14 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
     s_m[h] = mx;
     s_invl[h] = invl;
   }
-  // old scores of this warp's windows (needs only the entries), requested before the barrier
+  // old scores of this warp's windows (needs only the entries), requested before the barrier; with Eq. 1 the
+  // mass goes straight into the score, with the other ranking functions into the event accumulator
+  float* score = g.rank_mode == QEVICT_RANK_CUMULATIVE ? a.st.importance : a.st.event_mass;
   float old[NE];
 #pragma unroll
   for (int k = 0; k < NE; ++k) {
     const int e = e0 + wid + 4 * k;
-    old[k] = (e < e1 && e < n && lane == 0) ? a.st.importance[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] : 0.f;
+    old[k] = (e < e1 && e < n && lane == 0) ? score[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] : 0.f;
   }
   __syncthreads();
 
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
     const bool live = e < e1 && e < n;
     const float mass = live ? head_sum(rec[k], e) : 0.f;
     if (live && lane == 0) {
-      a.st.importance[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] = old[k] + mass;
+      score[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] = old[k] + mass;
       a.st.mass_e[(size_t)u * g.EMAX + e] = mass;
     }
   }

@@ -38,6 +38,8 @@ struct Geometry {
   int EMAX;      // max entries of a unit's work list
   int aged_cap;  // filled windows that may wait for a routing event
   int n_sink, n_recent;  // protected windows: sink prefix, recent region (besides the open window)
+  int rank_mode;     // QEVICT_RANK_*
+  float rank_param;  // lambda or p
   int Kfp;       // K_f + n_sink + n_recent: windows that may need a full-precision page in one event
   int tiles;     // W / 32
   // full-precision page: [H_kv][tile]{K tile, V tile}, each tile 32 x D elements, fragment-major
@@ -54,6 +56,7 @@ struct State {
   int32_t* fp_page;     // [NW]
   int32_t* q_page;      // [NW]
   float* importance;    // [NW]
+  float* event_mass;    // [NW] mass since the last routing event (ranking functions other than Eq. 1)
   int32_t* fp_owner;    // [PF] window holding the page, -1 free
   int32_t* q_owner;     // [PQ]
   int32_t* n_windows;   // [1]

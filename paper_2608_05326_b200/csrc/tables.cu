@@ -283,6 +283,30 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) ofp[i] = fp_owner[i];
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) oq[i] = q_owner[i];
 
+  // ---- ranking functions other than Eq. 1: fold the event accumulator into the score of every stored
+  // window (each operation rounded on its own, so that the ranking is taken on reproducible numbers) ----
+  if (g.rank_mode != QEVICT_RANK_CUMULATIVE && !prefill) {
+    float* score = a.st.importance + (size_t)u * g.NW;
+    float* ev = a.st.event_mass + (size_t)u * g.NW;
+    const int p = (int)g.rank_param;
+    for (int w = tid; w < nw; w += ROUTE_THREADS) {
+      const uint8_t t = tier[w];
+      if (t == QEVICT_TIER_NONE || t == QEVICT_TIER_EVICTED) continue;
+      const float uw = ev[w], s0 = score[w];
+      float s1;
+      if (g.rank_mode == QEVICT_RANK_DECAYED) {
+        s1 = __fadd_rn(__fmul_rn(g.rank_param, s0), uw);
+      } else {
+        float v = uw;
+        for (int i = 1; i < p; ++i) v = __fmul_rn(v, uw);
+        s1 = __fadd_rn(s0, v);
+      }
+      score[w] = s1;
+      ev[w] = 0.f;
+    }
+    __syncthreads();
+  }
+
   // ---- gather the candidates and the pinned windows in ascending window order -------------------------
   const int recent_lo = nw - (ow >= 0 ? 1 : 0) - g.n_recent;
   auto emit_gathered = [&](int w, int k, uint8_t t) {

@@ -44,6 +44,8 @@ class Workload:
     seed: int = BASE_SEED
     sink_windows: int = 0    # protected sink prefix (windows)
     recent_windows: int = 0  # filled windows kept in the protected recent region
+    rank_mode: int = 0       # 0 cumulative attention, 1 exponentially decayed, 2 attention p-norm
+    rank_param: float = 0.0  # lambda or p
 
     @property
     def n_units(self):

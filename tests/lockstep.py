@@ -21,7 +21,8 @@ MASS_RTOL = 1e-4                    # window scores / per-step mass
 def oracle_config(wl, aged_windows):
     return OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
                         wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged_windows,
-                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
+                        sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
+                        rank_param=wl.rank_param)
 
 
 def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
@@ -29,7 +30,8 @@ def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
     return binding.make_config(wl.batch if batch is None else batch, wl.n_layers if n_layers is None else n_layers,
                                wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits,
                                wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
-                               rebalance_interval_hint=r, sink_windows=wl.sink_windows, recent_windows=wl.recent_windows)
+                               rebalance_interval_hint=r, sink_windows=wl.sink_windows, recent_windows=wl.recent_windows,
+                               rank_mode=wl.rank_mode, rank_param=wl.rank_param)
 
 
 def aged_capacity(wl, rebalance_interval=None):
@@ -180,6 +182,11 @@ class LockstepRun:
                 assert abs(mass.sum() - wl.n_q_heads) < 1e-4 * wl.n_q_heads, what
             imp = tab["importance"].double().numpy()
             assert np.all(np.abs(imp - orc.importance) <= MASS_RTOL * np.abs(orc.importance) + 1e-7), what + " scores"
+            if wl.rank_mode != 0:  # the mass went to the event accumulator, the scores move at routing events only
+                ev = self.cache.export_event_mass(layer, seq).double().numpy()
+                assert np.all(np.abs(ev - orc.event_mass) <= MASS_RTOL * np.abs(orc.event_mass) + 1e-7), what + " event mass"
+                if not self.free_running:
+                    orc.event_mass[:] = ev
             if not self.free_running:
                 orc.importance[:] = imp  # lockstep: route on the GPU's float32 scores
         self.step_idx += 1

@@ -119,6 +119,23 @@ def test_protected_sink_and_recent_windows(kw):
         run.close()
 
 
+@pytest.mark.parametrize("mode,param", [(1, 0.9), (1, 0.5), (2, 3.0), (2, 2.0)])
+def test_ranking_function_variants(mode, param):
+    # decayed attention and attention p-norm: the mass is collected per routing event and folded into the score
+    # in float32 by the routing kernel; tiers, pages and codes must still match bit for bit
+    ls = _lockstep()
+    wl = _small("rank", steps=72, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, rank_mode=mode, rank_param=param)
+    run = ls.LockstepRun(wl, rebalance_interval=3)
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    o = run.oracles[0]
+    st = run.cache.stats()
+    assert st["promotions"] == o.stats["promotions"] and st["deletions"] == o.stats["deletions"] > 0
+    run.close()
+
+
 def test_many_candidates_and_tied_scores():
     # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
     # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides
