@@ -105,10 +105,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+// Pages are read once per step and a step reads several times the L2's capacity, so the copies carry an
+// evict-first policy: the stream of pages then leaves the small tables, the partials and the code of the
+// step's other kernels in L2 instead of flushing them every step.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -378,6 +387,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   const char* pr_base = nullptr;  // page of the producer's current entry (this KV head), set on its first piece
   const char* const fp_unit = p.fp_pool + (size_t)u * p.PF * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES;
   const char* const q_unit = p.q_pool + (size_t)u * p.PQ * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
+  const uint64_t l2pol = l2_evict_first_policy();
   auto issue_next = [&]() {  // warp-collective
     if (issued >= n_pieces || dead) return;
     if (pr_tile == 0 && pr_part == 0) {
@@ -390,11 +400,11 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
       const uint32_t dst = ring + slot * TT::SLOT_BYTES, bar = bars + slot * 8;
       if (!pr_isq) {
         mbar_expect_tx(bar, TT::FP_TILE_BYTES);
-        bulk_g2s(dst, pr_base + (size_t)(pr_tile * 2 + pr_part) * TT::FP_TILE_BYTES, TT::FP_TILE_BYTES, bar);
+        bulk_g2s(dst, pr_base + (size_t)(pr_tile * 2 + pr_part) * TT::FP_TILE_BYTES, TT::FP_TILE_BYTES, bar, l2pol);
       } else {
         mbar_expect_tx(bar, TT::Q_TILE_STRIDE + TT::KP_BYTES);
-        bulk_g2s(dst, pr_base + (size_t)pr_tile * TT::Q_TILE_STRIDE, TT::Q_TILE_STRIDE, bar);
-        bulk_g2s(dst + TT::Q_TILE_STRIDE, pr_base + TT::KP_OFF + (size_t)((pr_tile * 32) / GROUP) * TT::KP_BYTES, TT::KP_BYTES, bar);
+        bulk_g2s(dst, pr_base + (size_t)pr_tile * TT::Q_TILE_STRIDE, TT::Q_TILE_STRIDE, bar, l2pol);
+        bulk_g2s(dst + TT::Q_TILE_STRIDE, pr_base + TT::KP_OFF + (size_t)((pr_tile * 32) / GROUP) * TT::KP_BYTES, TT::KP_BYTES, bar, l2pol);
       }
     }
     ++issued;
