@@ -136,6 +136,23 @@ def test_ranking_function_variants(mode, param):
     run.close()
 
 
+def test_more_than_4096_windows():
+    # the routing kernel reads window states 16 per thread up to 4096 windows and falls back to a block-wide
+    # compaction above that; this prompt has 4200 windows
+    ls = _lockstep()
+    wl = _small("long", context=4200 * 32, n_q_heads=1, n_kv_heads=1, fp_budget_windows=6, q_budget_windows=10, steps=40,
+                sink_windows=1, recent_windows=1)
+    run = ls.LockstepRun(wl, rebalance_interval=1, score_mode="synthetic")
+    run.check_state("all", "after prefill")
+    st = run.cache.stats()
+    assert (st["n_full"], st["n_quant"], st["n_sink"], st["n_aged"]) == (6, 10, 1, 1)
+    assert st["n_evicted"] == 4200 - 18
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    run.close()
+
+
 def test_many_candidates_and_tied_scores():
     # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
     # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides
