@@ -167,6 +167,14 @@ QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer,
                                       const void* k_new_host, const void* v_new_host, void* out_host,
                                       void* stream);
 
+/* The same without the final synchronisation: the copies and the step are only enqueued.  `out_host` holds
+ * the result once the caller has synchronised `stream`; the host buffers must stay valid and unchanged until
+ * then (pinned memory, or the copies are not asynchronous).  Lets the caller enqueue more work -- the
+ * step's routing event, for one -- before it waits for the result. */
+QEVICT_API qevict_status qevict_decode_attn_host_async(qevict_handle h, int32_t layer, const void* q_host,
+                                                       const void* k_new_host, const void* v_new_host,
+                                                       void* out_host, void* stream);
+
 /* The same decode step for callers that must not allocate device memory (the paper has no counterpart:
  * this is a deployment variant of qevict_decode_attn, not a step of the method).
  *

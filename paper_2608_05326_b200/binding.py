@@ -60,6 +60,7 @@ _SIGNATURES = {
     "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_decode_attn_host_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_rebalance": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "qevict_get_stats": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(qevict_stats)]),
@@ -153,6 +154,11 @@ def qevict_decode_attn_host(h, layer, q, k_new, v_new, out, stream=None):
     _check(lib().qevict_decode_attn_host(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
 
 
+def qevict_decode_attn_host_async(h, layer, q, k_new, v_new, out, stream=None):
+    """Host tensors (pinned); the caller synchronises the stream before reading `out`."""
+    _check(lib().qevict_decode_attn_host_async(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
+
+
 def qevict_decode_attn_noalloc(h, layer, q, k_new, v_new, out, stream=None):
     """qevict_decode_attn with the attention scratch in the library's built-in device array: for callers
     that must not allocate device memory.  Raises QEvictError(NO_MEMORY) if the call's scratch does not fit."""
@@ -239,6 +245,9 @@ class QEvictCache:
     def decode_attn_host(self, layer, q, k_new, v_new, out, stream=None):
         qevict_decode_attn_host(self.handle, layer, q, k_new, v_new, out, stream)
         return out
+
+    def decode_attn_host_async(self, layer, q, k_new, v_new, out, stream=None):
+        qevict_decode_attn_host_async(self.handle, layer, q, k_new, v_new, out, stream)
 
     def rebalance(self, layer, stream=None):
         qevict_rebalance(self.handle, layer, stream)

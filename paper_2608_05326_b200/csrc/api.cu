@@ -441,8 +441,8 @@ QEVICT_API qevict_status qevict_decode_attn(qevict_handle h, int32_t layer, cons
   return decode_impl(h, layer, q, k_new, v_new, out, (cudaStream_t)stream);
 }
 
-QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer, const void* q_host, const void* k_new_host,
-                                      const void* v_new_host, void* out_host, void* stream) {
+static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void* q_host, const void* k_new_host,
+                                      const void* v_new_host, void* out_host, void* stream, bool sync) {
   if (!h) return QEVICT_ERR_INVALID_ARG;
   int l0, l1;
   if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
@@ -462,8 +462,19 @@ QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer,
                                        k_new_host ? h->stage_v : nullptr, h->stage_out, s);
   if (st != QEVICT_OK) return st;
   QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
-  QE_CUDA(h, cudaStreamSynchronize(s));
+  if (sync) QE_CUDA(h, cudaStreamSynchronize(s));
   return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer, const void* q_host, const void* k_new_host,
+                                      const void* v_new_host, void* out_host, void* stream) {
+  return decode_host_impl(h, layer, q_host, k_new_host, v_new_host, out_host, stream, true);
+}
+
+QEVICT_API qevict_status qevict_decode_attn_host_async(qevict_handle h, int32_t layer, const void* q_host,
+                                                       const void* k_new_host, const void* v_new_host, void* out_host,
+                                                       void* stream) {
+  return decode_host_impl(h, layer, q_host, k_new_host, v_new_host, out_host, stream, false);
 }
 
 QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* stream) {

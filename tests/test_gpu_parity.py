@@ -273,8 +273,13 @@ def test_host_buffer_entry_point_matches_device_call():
         kn = torch.stack([b.new_kv[u][0][t] for u in range(2)]).contiguous().pin_memory()
         vn = torch.stack([b.new_kv[u][1][t] for u in range(2)]).contiguous().pin_memory()
         out = torch.empty_like(q).pin_memory()
-        b.cache.decode_attn_host(-1, q, kn, vn, out)
-        b.cache.rebalance(-1)
+        if t % 2 == 0:
+            b.cache.decode_attn_host(-1, q, kn, vn, out)
+            b.cache.rebalance(-1)
+        else:  # the variant that only enqueues: the routing event goes in before the host waits for the result
+            b.cache.decode_attn_host_async(-1, q, kn, vn, out)
+            b.cache.rebalance(-1)
+            torch.cuda.current_stream().synchronize()
         assert torch.equal(out, oa)
     a.close(); b.close()
 
