@@ -323,7 +323,52 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   };
   int n_all, n_real;
   const int chunk = (nw + ROUTE_THREADS - 1) / ROUTE_THREADS;
-  if (chunk <= 16) {
+  constexpr int PRE = 10;
+  const int cs = (g.NW + ROUTE_THREADS - 1) / ROUTE_THREADS;  // rows of the table per thread (not of the windows in use)
+  if (cs <= PRE && (g.rank_mode == QEVICT_RANK_CUMULATIVE || prefill)) {
+    // Small tables: every thread requests all five columns of its rows at once, before it knows how many
+    // windows exist or which of them are candidates (rows past the last window hold state NONE), so the
+    // whole gather costs one global round trip.
+    const int b = tid * cs;
+    uint8_t tc[PRE], lc[PRE];
+    int32_t fc[PRE], qc[PRE];
+    float ic[PRE];
+#pragma unroll
+    for (int k = 0; k < PRE; ++k) {
+      const bool ok = k < cs && b + k < g.NW;
+      tc[k] = ok ? tier[b + k] : (uint8_t)QEVICT_TIER_NONE;
+      lc[k] = ok ? ledger[b + k] : (uint8_t)0;
+      fc[k] = ok ? fp_page[b + k] : -1;
+      qc[k] = ok ? q_page[b + k] : -1;
+      ic[k] = ok ? imp[b + k] : 0.f;
+    }
+    int cnt = 0;  // gathered | candidates << 16
+#pragma unroll
+    for (int k = 0; k < PRE; ++k) {
+      const bool c = is_candidate(tc[k], b + k, recent_lo);
+      cnt += (c || is_pinned(tc[k], b + k, recent_lo) ? 1 : 0) + (c ? 0x10000 : 0);
+    }
+    int tot;
+    int rank = block_exclusive_scan(cnt, scratch, &tot) & 0xFFFF;
+    n_all = tot & 0xFFFF; n_real = tot >> 16;
+#pragma unroll
+    for (int k = 0; k < PRE; ++k) {
+      const int w = b + k;
+      const bool pin = is_pinned(tc[k], w, recent_lo);
+      if ((is_candidate(tc[k], w, recent_lo) || pin) && rank < sort_cap) {
+        cw[rank] = w;
+        ctier[rank] = tc[k];
+        cled[rank] = lc[k];
+        cfp[rank] = fc[k];
+        cq[rank] = qc[k];
+        if (pin) cnew[rank] = PINNED | tc[k];
+        keys[rank] = pin ? (0xFFFFFFFF00000000ull | (uint32_t)rank)
+                         : (((unsigned long long)(~mono_bits(ic[k])) << 32) | (uint32_t)rank);
+        ++rank;
+      }
+    }
+    __syncthreads();
+  } else if (chunk <= 16) {
     // every thread reads its (up to 16) window states in one go and keeps them in registers
     uint8_t tc[16];
     const int b = tid * chunk;
@@ -490,13 +535,13 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   const int qcap = g.PF + g.Kq;
   const int nq = min(n_q_need, min(n_free_q, qcap)), nfp = min(n_fp_need, min(n_free_fp, prefill ? g.Kfp : g.Kf));
   const int n_items = nq + (prefill ? 0 : nfp);
-  int* s_base = scratch + 102;
+  int qbase = 0;  // thread 0: where this unit's records start in the call's queue (waited for only at the end)
   if (tid == 0) {
     if (n_q_need > nq) record_check(a.st.status, CHECK_Q_POOL_EXHAUSTED);
     if (n_fp_need > nfp) record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED);
     // this unit's migrations join the call's queue (the order of the units in it does not matter: the
     // items are independent of one another); the reply is needed only at the very end
-    *s_base = n_items > 0 ? atomicAdd(a.st.mig_count + 2 * (a.unit0 / g.batch), n_items) : 0;
+    if (n_items > 0) qbase = atomicAdd(a.st.mig_count + 2 * (a.unit0 / g.batch), n_items);
   }
   __syncthreads();
 
@@ -554,10 +599,12 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   }
   for (int i = tid; i < g.PF; i += ROUTE_THREADS) fp_owner[i] = ofp[i];
   for (int i = tid; i < g.PQ; i += ROUTE_THREADS) q_owner[i] = oq[i];
-  // the migration records (32 bytes each; format: see the migration kernel)
-  {
-    int4* queue = a.st.mig_queue + ((size_t)a.unit0 * (g.PF + g.Kq + g.Kf) + *s_base) * 2;
-    for (int i = tid; i < n_items; i += ROUTE_THREADS) {
+  // the migration records (32 bytes each; format: see the migration kernel), written by the first warp: the
+  // reply of the queue reservation reaches the other lanes by shuffle
+  if (tid < 32) {
+    const int base = __shfl_sync(0xffffffffu, qbase, 0);
+    int4* queue = a.st.mig_queue + ((size_t)a.unit0 * (g.PF + g.Kq + g.Kf) + base) * 2;
+    for (int i = tid; i < n_items; i += 32) {
       if (i < nq) {
         const int4 it = qrec[i];
         queue[2 * i] = make_int4(u, 0, it.x, it.y);
