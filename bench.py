@@ -35,7 +35,7 @@ HBM_FALLBACK_GBS = 6650.0
 # summarised under profiles/ (bytes per launch, keyed by workload name); None = not captured.
 NCU_TRAFFIC_BYTES = {
     # profiles/decode_attn_c1x32.md: 440.83 MB read + 6.50 MB written per launch
-    "c1-llama3-8b-32k": 447_670_000,
+    "c1-llama3-8b-32k": 446_080_000,
 }
 
 
