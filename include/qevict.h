@@ -149,6 +149,25 @@ QEVICT_API qevict_status qevict_destroy(qevict_handle h);
 QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, const void* k, const void* v,
                                     int32_t ctx_tokens, const float* window_scores, void* stream);
 
+/* Prefill window scores computed on the GPU [Methodology: prompt attention initialises the window scores;
+ * Eq. 1's form].  For every sequence of one layer, n_obs observation queries per query head -- queries that
+ * stand after the prompt, e.g. its last n_obs positions' queries -- attend over the whole prompt in full
+ * precision, and
+ *     window_scores[seq][w] = sum over observation queries and query heads of the softmax mass of window w
+ * (raw sum, the input qevict_prefill_assign expects).  Which queries observe is the caller's choice: the paper
+ * does not fix it.
+ *   k             device, [batch][H_kv][ctx_tokens][d] in the execution datatype (one layer)
+ *   q_obs         device, [batch][n_obs][H_q][d], n_obs in 1..64
+ *   window_scores device, float32 [batch][ctx_tokens / W] (output)
+ *   scratch       device, at least qevict_prefill_score_scratch_bytes(...) bytes, 8-byte aligned; contents
+ *                 are overwritten
+ * Deterministic (fixed summation order). */
+QEVICT_API qevict_status qevict_prefill_score_scratch_bytes(qevict_handle h, int32_t n_obs, int32_t ctx_tokens,
+                                                            uint64_t* bytes);
+QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, const void* q_obs, int32_t n_obs,
+                                              int32_t ctx_tokens, float* window_scores, void* scratch,
+                                              uint64_t scratch_bytes, void* stream);
+
 /* One decode step [attention equation; Eq. 1].  If k_new != NULL the new token's key and value
  * first enter the recent region (the open window); then every query head attends over all accessible
  * tokens (open, aged, Full and Quantized windows, the latter dequantized in registers) and each

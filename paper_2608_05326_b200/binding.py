@@ -53,6 +53,9 @@ _SIGNATURES = {
     "qevict_create": (C.c_int, [C.POINTER(qevict_config), C.c_void_p, C.c_uint64, C.POINTER(C.c_void_p)]),
     "qevict_destroy": (C.c_int, [C.c_void_p]),
     "qevict_set_splits": (C.c_int, [C.c_void_p, C.c_int32]),
+    "qevict_prefill_score_scratch_bytes": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_uint64)]),
+    "qevict_prefill_score": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                      C.c_uint64, C.c_void_p]),
     "qevict_export_event_mass": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32]),
     "qevict_kernel_time": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
@@ -234,6 +237,17 @@ class QEvictCache:
         assert k.is_cuda and k.is_contiguous() and v.is_contiguous() and k.dtype == self.torch_dtype
         assert window_scores.dtype == torch.float32 and window_scores.is_contiguous()
         qevict_prefill_assign(self.handle, layer, k, v, k.shape[-2], window_scores, stream)
+
+    def prefill_score(self, k, q_obs, stream=None):
+        """k [batch, H_kv, ctx, d], q_obs [batch, n_obs, H_q, d] (device) -> window scores [batch, ctx / W] float32."""
+        n_obs, ctx = q_obs.shape[1], k.shape[-2]
+        need = C.c_uint64()
+        _check(lib().qevict_prefill_score_scratch_bytes(self.handle, n_obs, ctx, C.byref(need)), self.handle)
+        scratch = torch.empty(need.value, dtype=torch.uint8, device=self.device)
+        scores = torch.empty((k.shape[0], ctx // self.cfg.window), dtype=torch.float32, device=self.device)
+        _check(lib().qevict_prefill_score(self.handle, _ptr(k), _ptr(q_obs), n_obs, ctx, _ptr(scores), _ptr(scratch),
+                                          need.value, _stream(stream)), self.handle)
+        return scores
 
     def decode_attn(self, layer, q, k_new=None, v_new=None, out=None, stream=None):
         assert q.is_cuda and q.is_contiguous() and q.dtype == self.torch_dtype

@@ -325,3 +325,45 @@ def test_config1_llama_shape_lockstep():
     run.rebalance(full_check=True)
     assert run.cache.stats()["promotions"] == run.oracles[0].stats["promotions"]
     run.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, batch=2, context=2048),
+    dict(dtype="fp16", head_dim=64, n_q_heads=3, n_kv_heads=1, window=64, group_size=32, context=1024),
+], ids=["bf16-d128-g4", "fp16-d64-w64"])
+def test_prefill_scores_on_the_gpu_match_the_oracle(kw):
+    """Window scores of the prompt from observation queries: the GPU routine against the oracle's attention
+    (raw mass per window summed over observers and heads), and a prefill_assign fed with them against the
+    oracle fed with its own."""
+    from oracle import accessible_attention
+    ls = _lockstep()
+    wl = _small("pscore", steps=4, **kw)
+    cache = binding.QEvictCache(ls.gpu_config(wl))
+    n_obs = 6
+    orcs = []
+    ks, vs, qs = [], [], []
+    for u in range(wl.n_units):
+        k, v = workloads.gen_prompt_kv(wl, u)
+        g = torch.Generator().manual_seed(991 + u)
+        q = torch.randn((n_obs, wl.n_q_heads, wl.head_dim), generator=g).to(wl.torch_dtype)
+        ks.append(k); vs.append(v); qs.append(q)
+    kd, vd, qd = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+    got = cache.prefill_score(kd, qd)
+    torch.cuda.synchronize()
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    for u in range(wl.n_units):
+        k64 = ks[u].double().numpy()
+        ref = np.zeros(wl.n_prompt_windows)
+        for o in range(n_obs):
+            _, p = accessible_attention(qs[u][o].double().numpy(), k64, np.zeros_like(k64[:, :, :1]), scale)
+            ref += p.sum(0).reshape(wl.n_prompt_windows, wl.window).sum(1)
+        g_u = got[u].cpu().double().numpy()
+        assert abs(g_u.sum() - n_obs * wl.n_q_heads) < 1e-3
+        assert np.all(np.abs(g_u - ref) <= ls.MASS_RTOL * np.abs(ref) + 1e-7), np.abs(g_u - ref).max()
+    # the scores drive the first tier assignment: same tiers as the oracle routed on the same float32 scores
+    cache.prefill_assign(0, kd, vd, got)
+    for u in range(wl.n_units):
+        orc = ls.UnitOracle(ls.oracle_config(wl, ls.aged_capacity(wl)))
+        orc.prefill_assign(ks[u].double().numpy(), vs[u].double().numpy(), got[u].cpu().numpy())
+        ls.compare_state(cache, 0, u, orc, wl, what="prefill from GPU scores, unit %d" % u)
+    cache.close()
