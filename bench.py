@@ -261,13 +261,15 @@ def run_ours(args, rank, world):
         barrier()
         t0 = time.perf_counter()
         # every step: inputs leave pinned host memory, the step and its routing event are enqueued, and the host
-        # waits until the result is in host memory before it sends the next step's inputs
-        cur = torch.cuda.current_stream()
+        # waits until the result is in host memory before it sends the next step's inputs (the final barrier
+        # waits for the last routing event)
+        got = torch.cuda.Event()
         for i in range(K):
             cache.decode_attn_host_async(-1, qh[i], knh[i] if append else None, vnh[i] if append else None, outh)
+            got.record()          # the result is in host memory once this event has passed
             if (t + i + 1) % R == 0:
                 cache.rebalance(-1)
-            cur.synchronize()
+            got.synchronize()     # the routing event keeps running while the host turns around
         barrier()
         e2e_s = time.perf_counter() - t0
         h2d = qh[0].numel() * 2 + (2 * knh[0].numel() * 2 if append else 0)
