@@ -24,11 +24,11 @@ __device__ __forceinline__ float ex2a(float x) {
 template <class T>
 __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelArgs a, int S, int e_bound, T* __restrict__ out) {
   const Geometry& g = a.geo;
-  // every CTA owns 4 * NE consecutive work-list entries for the mass update and a slice of the
+  // every CTA owns 4 * NE (= 16) consecutive work-list entries for the mass update and a slice of the
   // (head, 4-channel) tasks of the output merge; all its global loads are issued before anything waits
   const int ul = blockIdx.y, u = a.unit0 + ul, tid = threadIdx.x;
   const int lane = tid & 31, wid = tid >> 5;
-  constexpr int NE = 8;  // work-list entries a warp keeps in registers at a time
+  constexpr int NE = 4;  // work-list entries a warp keeps in registers at a time
   extern __shared__ __align__(16) unsigned char csm[];
   float* s_m = reinterpret_cast<float*>(csm);  // [Hq] global maximum
   float* s_invl = s_m + g.Hq;                  // [Hq] 1 / denominator
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
 }  // namespace
 
 cudaError_t launch_combine(const KernelArgs& a, int n_splits, int e_bound, void* out, cudaStream_t s) {
-  const int chunks = (e_bound + 31) / 32;  // 4 warps x 8 entries per CTA
+  const int chunks = (e_bound + 15) / 16;  // 4 warps x 4 entries per CTA
   dim3 grid(chunks > a.geo.Hkv ? chunks : a.geo.Hkv, a.n_units);
   const size_t sm = (size_t)a.geo.Hq * 8 + (size_t)a.geo.Hq * n_splits * 4;
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
