@@ -367,3 +367,53 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw):
         orc.prefill_assign(ks[u].double().numpy(), vs[u].double().numpy(), got[u].cpu().numpy())
         ls.compare_state(cache, 0, u, orc, wl, what="prefill from GPU scores, unit %d" % u)
     cache.close()
+
+
+def _random_workloads(n, seed=20260805):
+    """Seeded draws over the supported configuration space (shapes, tiers, protected regions, ranking
+    functions, routing intervals)."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        window = int(rng.choice([32, 64]))
+        group = int(rng.choice([32, 64])) if window == 64 else 32
+        head_dim = int(rng.choice([64, 128]))
+        if head_dim % group:
+            group = 32
+        n_kv = int(rng.choice([1, 2, 3]))
+        gq = int(rng.choice([1, 2, 3, 4, 5, 7, 8]))
+        n_win = int(rng.integers(10, 28))
+        k_f = int(rng.integers(0, 6))
+        k_q = int(rng.integers(0 if k_f else 1, 9))
+        mode = int(rng.choice([0, 0, 1, 2]))
+        param = {0: 0.0, 1: float(rng.choice([0.5, 0.9, 0.99])), 2: float(rng.choice([2, 3]))}[mode]
+        interval = int(rng.choice([1, 2, 7, window, window + 5]))
+        wl = _small("fuzz%d" % i, dtype=str(rng.choice(["fp16", "bf16"])), head_dim=head_dim, n_q_heads=gq * n_kv,
+                    n_kv_heads=n_kv, window=window, group_size=group, quant_bits=int(rng.choice([2, 4])),
+                    context=n_win * window, fp_budget_windows=k_f, q_budget_windows=k_q,
+                    sink_windows=int(rng.integers(0, 3)), recent_windows=int(rng.integers(0, 3)),
+                    rank_mode=mode, rank_param=param, steps=2 * window + int(rng.integers(3, 20)),
+                    batch=int(rng.choice([1, 2])), rebalance_interval=interval)
+        out.append(wl)
+    return out
+
+
+@pytest.mark.parametrize("wl", _random_workloads(24), ids=lambda wl: "%s-%s-d%d-h%d/%d-w%d-g%d-b%d-f%d-q%d-s%d-r%d-m%d-R%d" % (
+    wl.name, wl.dtype, wl.head_dim, wl.n_q_heads, wl.n_kv_heads, wl.window, wl.group_size, wl.quant_bits,
+    wl.fp_budget_windows, wl.q_budget_windows, wl.sink_windows, wl.recent_windows, wl.rank_mode, wl.rebalance_interval))
+def test_random_configurations_lockstep(wl):
+    ls = _lockstep()
+    run = ls.LockstepRun(wl, rebalance_interval=wl.rebalance_interval, score_mode="synthetic")
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    for u, orc in run.oracles.items():
+        layer, seq = run.unit_ls(u)
+        st = run.cache.stats(layer)
+        assert st["n_sink"] >= 0
+    o = run.oracles[0]
+    st = run.cache.stats()
+    assert st["deletions"] == sum(x.stats["deletions"] for x in run.oracles.values())
+    assert st["promotions"] == sum(x.stats["promotions"] for x in run.oracles.values())
+    run.close()
