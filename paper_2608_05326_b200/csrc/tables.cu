@@ -7,7 +7,7 @@ namespace qevict {
 
 namespace {
 
-constexpr int ROUTE_THREADS = 256;
+constexpr int ROUTE_MAX_THREADS = 512;
 
 // order-preserving map float -> uint32 (ascending); -0 and +0 collapse
 __device__ __forceinline__ uint32_t mono_bits(float f) {
@@ -243,7 +243,8 @@ __device__ __forceinline__ bool is_pinned(uint8_t t, int w, int recent_lo) {
   return t == QEVICT_TIER_SINK || (t == QEVICT_TIER_AGED && w >= recent_lo);
 }
 
-__global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a, int prefill, int sort_cap) {
+template <int NT>  // threads per CTA
+__global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefill, int sort_cap) {
   const Geometry& g = a.geo;
   const int u = a.unit0 + blockIdx.x, tid = threadIdx.x;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -280,8 +281,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   int* s_react = scratch + 100;
   int* s_del = scratch + 101;
   if (tid == 0) { *s_react = 0; *s_del = 0; }
-  for (int i = tid; i < g.PF; i += ROUTE_THREADS) ofp[i] = fp_owner[i];
-  for (int i = tid; i < g.PQ; i += ROUTE_THREADS) oq[i] = q_owner[i];
+  for (int i = tid; i < g.PF; i += NT) ofp[i] = fp_owner[i];
+  for (int i = tid; i < g.PQ; i += NT) oq[i] = q_owner[i];
 
   // ---- ranking functions other than Eq. 1: fold the event accumulator into the score of every stored
   // window (each operation rounded on its own, so that the ranking is taken on reproducible numbers) ----
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     float* score = a.st.importance + (size_t)u * g.NW;
     float* ev = a.st.event_mass + (size_t)u * g.NW;
     const int p = (int)g.rank_param;
-    for (int w = tid; w < nw; w += ROUTE_THREADS) {
+    for (int w = tid; w < nw; w += NT) {
       const uint8_t t = tier[w];
       if (t == QEVICT_TIER_NONE || t == QEVICT_TIER_EVICTED) continue;
       const float uw = ev[w], s0 = score[w];
@@ -322,9 +323,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     keys[k] = pin ? (0xFFFFFFFF00000000ull | (uint32_t)k) : (((unsigned long long)(~mono_bits(imp[w])) << 32) | (uint32_t)k);
   };
   int n_all, n_real;
-  const int chunk = (nw + ROUTE_THREADS - 1) / ROUTE_THREADS;
+  const int chunk = (nw + NT - 1) / NT;
   constexpr int PRE = 10;
-  const int cs = (g.NW + ROUTE_THREADS - 1) / ROUTE_THREADS;  // rows of the table per thread (not of the windows in use)
+  const int cs = (g.NW + NT - 1) / NT;  // rows of the table per thread (not of the windows in use)
   if (cs <= PRE && (g.rank_mode == QEVICT_RANK_CUMULATIVE || prefill)) {
     // Small tables: every thread requests all five columns of its rows at once, before it knows how many
     // windows exist or which of them are candidates (rows past the last window hold state NONE), so the
@@ -406,13 +407,18 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
   // Quantized, remainder -> Evicted -----------------------------------------------------------------
   if (n_cand <= 256) {
-    // rank of a key = number of smaller keys (all keys are distinct)
-    for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
-      const unsigned long long mine = keys[c];
-      if ((uint32_t)(mine >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
+    // rank of a key = number of smaller keys (all keys are distinct); two adjacent lanes share a key and
+    // count over one half of the keys each
+    const int half = tid & 1, i0 = half ? n_cand / 2 : 0, i1 = half ? n_cand : n_cand / 2;
+    for (int cb = 0; cb < n_cand; cb += NT / 2) {  // same trip count for the whole block
+      const int c = cb + (tid >> 1);
+      const unsigned long long mine = c < n_cand ? keys[c] : ~0ull;
       int pos = 0;
-      for (int i = 0; i < n_cand; ++i) pos += keys[i] < mine ? 1 : 0;
-      cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
+      if (c < n_cand)
+        for (int i = i0; i < i1; ++i) pos += keys[i] < mine ? 1 : 0;
+      pos += __shfl_xor_sync(0xffffffffu, pos, 1);
+      if (c < n_cand && !half && (uint32_t)(mine >> 32) != 0xFFFFFFFFu)  // pinned windows keep the state set above
+        cnew[c] = pos < g.Kf ? QEVICT_TIER_FULL : (pos < g.Kf + g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
     }
   } else {
     // Only the two cuts are needed, not the order: most-significant-digit-first radix selection of the
@@ -429,10 +435,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
 #pragma unroll 1
     for (int pass = 0; pass < 6; ++pass) {
       const int shift = pass < 4 ? 56 - 8 * pass : (pass == 4 ? 8 : 0);
-      for (int i = tid; i < 512; i += ROUTE_THREADS) hist[i] = 0;
+      for (int i = tid; i < 512; i += NT) hist[i] = 0;
       __syncthreads();
       const unsigned long long p0 = ((unsigned long long)sel[1] << 32) | sel[0], p1 = ((unsigned long long)sel[3] << 32) | sel[2];
-      for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+      for (int c = tid; c < n_cand; c += NT) {
         const unsigned long long key = keys[c];
         const int d = (int)((key >> shift) & 255ull);
         if ((key & mask) == p0) atomicAdd(&hist[d], 1);
@@ -470,7 +476,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
       __syncthreads();
     }
     const unsigned long long t0 = ((unsigned long long)sel[1] << 32) | sel[0], t1 = ((unsigned long long)sel[3] << 32) | sel[2];
-    for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+    for (int c = tid; c < n_cand; c += NT) {
       const unsigned long long key = keys[c];
       if ((uint32_t)(key >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
       cnew[c] = (kk[0] > 0 && key <= t0) ? QEVICT_TIER_FULL : ((kk[1] > 0 && key <= t1) ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED);
@@ -479,7 +485,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   __syncthreads();
 
   // ---- releases (owner tables only; the candidates' page ids stay readable until the lists are built) --
-  for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+  for (int c = tid; c < n_cand; c += NT) {
     const uint8_t old = ctier[c], nt = cnew[c];
     if ((nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT) || nt == QEVICT_TIER_EVICTED) {
       if (cfp[c] >= 0) ofp[cfp[c]] = -1;
@@ -490,7 +496,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
       atomicAdd(s_react, 1);
     }
   }
-  for (int i = tid; i < g.PF; i += ROUTE_THREADS) reader[i] = -1;
+  for (int i = tid; i < g.PF; i += NT) reader[i] = -1;
   __syncthreads();
 
   // ---- one packed scan yields six stable compactions at once (all ascending): free full-precision pages,
@@ -503,8 +509,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   auto lists_as_full = [&](int c) { return cnew[c] == QEVICT_TIER_FULL || (cnew[c] & PINNED); };
   int32_t* need_q = reinterpret_cast<int32_t*>(keys);  // the sort keys are dead from here on
   int32_t* need_fp = need_q + sort_cap;
-  const int ch_f = (g.PF + ROUTE_THREADS - 1) / ROUTE_THREADS, ch_q = (g.PQ + ROUTE_THREADS - 1) / ROUTE_THREADS;
-  const int ch_c = (n_cand + ROUTE_THREADS - 1) / ROUTE_THREADS;
+  const int ch_f = (g.PF + NT - 1) / NT, ch_q = (g.PQ + NT - 1) / NT;
+  const int ch_c = (n_cand + NT - 1) / NT;
   const int bf = min(g.PF, tid * ch_f), ef = min(g.PF, bf + ch_f), bq = min(g.PQ, tid * ch_q), eq = min(g.PQ, bq + ch_q);
   const int bc = min(n_cand, tid * ch_c), ec = min(n_cand, bc + ch_c);
   int3 cnt = make_int3(0, 0, 0);  // {free fp | free q << 16, need q | need fp << 16, Full | Quantized << 16}
@@ -547,7 +553,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
 
   // first demotions take the free quantized pages in ascending order.  reader[p] = index of the
   // quantization that reads full-precision page p
-  for (int k = tid; k < nq; k += ROUTE_THREADS) {
+  for (int k = tid; k < nq; k += NT) {
     const int c = need_q[k], pg = free_q[k];
     oq[pg] = cw[c];
     qrec[k] = make_int4(cw[c], prefill ? -1 : cfp[c], pg, -1);  // {window, source page, destination page, linked promotion}
@@ -560,7 +566,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   // that receives a page some quantization of this event still has to read is linked to that quantization
   // (the migration kernel runs it right after it, in the same warps).
   int4* copy_list = a.st.copy_list + (size_t)u * g.Kfp;
-  for (int k = tid; k < nfp; k += ROUTE_THREADS) {
+  for (int k = tid; k < nfp; k += NT) {
     const int c = need_fp[k], pg = free_fp[k];
     ofp[pg] = cw[c];
     cfp[c] = pg;
@@ -575,7 +581,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   __syncthreads();
 
   // ---- commit: the candidates' rows and the owner tables go back to global memory --------------------
-  for (int c = tid; c < n_cand; c += ROUTE_THREADS) {
+  for (int c = tid; c < n_cand; c += NT) {
     const uint8_t old = ctier[c], nt = cnew[c];
     const int w = cw[c];
     if (nt & PINNED) {  // state unchanged; at prefill the window has just received its page
@@ -597,8 +603,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
     fp_page[w] = cfp[c];
     q_page[w] = cq[c];
   }
-  for (int i = tid; i < g.PF; i += ROUTE_THREADS) fp_owner[i] = ofp[i];
-  for (int i = tid; i < g.PQ; i += ROUTE_THREADS) q_owner[i] = oq[i];
+  for (int i = tid; i < g.PF; i += NT) fp_owner[i] = ofp[i];
+  for (int i = tid; i < g.PQ; i += NT) q_owner[i] = oq[i];
   // the migration records (32 bytes each; format: see the migration kernel), written by the first warp: the
   // reply of the queue reservation reaches the other lanes by shuffle
   if (tid < 32) {
@@ -624,7 +630,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_kernel(const KernelArgs a
   uint2* entries = a.st.entries + (size_t)u * g.EMAX;
   {
     const int n = n_f + n_q;
-    for (int k = tid; k < n && k < g.EMAX; k += ROUTE_THREADS) {
+    for (int k = tid; k < n && k < g.EMAX; k += NT) {
       const int cf = (int)(((long long)k * n_f) / n);                       // Full windows before position k
       const bool is_f = (int)(((long long)(k + 1) * n_f) / n) > cf;
       if (is_f) {
@@ -672,7 +678,9 @@ size_t route_smem_bytes(const Geometry& g, int sort_cap) {
 
 cudaError_t route_prepare(size_t max_smem) {
   if (max_smem <= 48 * 1024) return cudaSuccess;
-  return cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  cudaError_t e = cudaFuncSetAttribute(route_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(route_kernel<ROUTE_MAX_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
 }
 
 cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s) {
@@ -689,7 +697,11 @@ cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt, const float* 
 }
 
 cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_cap, cudaStream_t s) {
-  return launch_pdl(route_kernel, dim3(a.n_units), dim3(ROUTE_THREADS), route_smem_bytes(a.geo, sort_cap), s, a, prefill, sort_cap);
+  // more threads only pay when there are many candidates (every phase is a loop over them)
+  if (sort_cap > 512)
+    return launch_pdl(route_kernel<ROUTE_MAX_THREADS>, dim3(a.n_units), dim3(ROUTE_MAX_THREADS), route_smem_bytes(a.geo, sort_cap), s, a,
+                      prefill, sort_cap);
+  return launch_pdl(route_kernel<256>, dim3(a.n_units), dim3(256), route_smem_bytes(a.geo, sort_cap), s, a, prefill, sort_cap);
 }
 
 cudaError_t launch_export_mass(const KernelArgs& a, int unit, float* mass, cudaStream_t s) {
