@@ -59,3 +59,19 @@ def test_config3_long_context_window64_sampled_unit():
 def test_config4_qwen_gqa7_sampled_unit(bits, fp_frac):
     wl = workloads.config(4, bits=bits, fp_frac=fp_frac)
     _run(wl, oracle_units=[3], steps=34, rebalance_interval=2)
+
+
+def test_config1_all_256_steps_two_units():
+    # the whole run of the configuration (256 decode steps, routing event after every step), two units followed
+    # step by step, every page, code and table compared at the end
+    import lockstep
+    wl = replace(workloads.config(1, n_layers=32), steps=256)
+    run = lockstep.LockstepRun(wl, oracle_units=[0, 17], score_mode="synthetic", rebalance_interval=1, gen_device="cuda")
+    for _ in range(256):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    st = run.cache.stats()
+    assert st["decode_steps"] == 256 and st["n_full"] == 32 * 64 and st["n_quant"] == 32 * 128
+    for u, o in run.oracles.items():
+        assert o.stats["promotions"] > 50 and o.stats["deletions"] > 832
+    run.close()
