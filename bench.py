@@ -55,6 +55,9 @@ def parse_args():
     ap.add_argument("--recent-windows", type=int, default=0, help="filled windows kept in the protected recent region")
     ap.add_argument("--rank-mode", type=int, default=0, help="0 cumulative attention (Eq. 1), 1 decayed, 2 p-norm")
     ap.add_argument("--rank-param", type=float, default=0.0, help="lambda of the decayed score / p of the p-norm")
+    ap.add_argument("--prefill-score", type=int, default=0, metavar="N_OBS",
+                    help="instead of the decode loop: time qevict_prefill_score (window scores of one layer's prompt from "
+                         "N_OBS observation queries per head) and print its own JSON line")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -384,10 +387,47 @@ def run_reference(args, rank):
     }
 
 
+def run_prefill_score(args):
+    """Prefill-side step of the path (not part of the decode metric): window scores of the prompt on the GPU."""
+    from paper_2608_05326_b200 import binding, build
+    build.build()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    wl = replace(workloads.config(args.config), n_layers=1)
+    cfg = binding.make_config(wl.batch, 1, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits,
+                              wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, device=dev.index)
+    cache = binding.QEvictCache(cfg)
+    k = torch.stack([workloads.gen_prompt_kv(wl, u, device=dev)[0] for u in range(wl.batch)])
+    g = torch.Generator(device=dev).manual_seed(wl.seed)
+    q = torch.randn((wl.batch, args.prefill_score, wl.n_q_heads, wl.head_dim), generator=g, device=dev).to(wl.torch_dtype)
+    for _ in range(max(3, args.warmup)):
+        s = cache.prefill_score(k, q)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = max(1, min(args.steps, 50))
+    e0.record()
+    for _ in range(n):
+        s = cache.prefill_score(k, q)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    line = {"metric": "prefill_score_ms", "value": ms, "unit": "ms", "higher_is_better": False, "n_gpus": 1, "steps": n,
+            "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": "%s, one layer, %d observation queries per head" % (wl.name, args.prefill_score),
+                       "key_bytes": k.numel() * 2},
+            "mass_sum": float(s.sum()), "expected_mass_sum": float(wl.batch * args.prefill_score * wl.n_q_heads)}
+    cache.close()
+    return line
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.prefill_score > 0:
+        if rank == 0:
+            print(json.dumps(run_prefill_score(args)))
+        return
     if args.impl == "reference":
         line = run_reference(args, rank)
         if line is not None:

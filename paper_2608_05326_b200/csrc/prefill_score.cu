@@ -67,6 +67,138 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_tiles_kernel(const T* __r
   }
 }
 
+// ---- the same tile records on the 5th-generation tensor cores ---------------------------------------------
+// logits[128 tokens][NP queries] = K[128][D] . Q^T[D][NP] is a dense contraction: one tcgen05.mma chain per CTA
+// (M = 128, N = NP, D / 16 steps of K = 16), operands in shared memory in the canonical K-major layout without
+// swizzle -- 8-row x 16-byte core matrices, 128 bytes each, SBO between 8-row groups, LBO between the two
+// 16-byte halves of a K = 16 step -- written with plain stores, accumulator in tensor memory (128 lanes x NP
+// fp32 columns), read back with tcgen05.ld so that lane = token, exactly as the shuffle reductions want it.
+// Every wait is bounded; a wait that runs out records CHECK_COPY_TIMEOUT and the CTA frees its tensor memory
+// and leaves.
+__device__ __forceinline__ uint32_t sm_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // start address, leading and stride byte offsets in 16-byte units; version 1; no swizzle
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+template <class T>
+__global__ void __launch_bounds__(128) score_tiles_tc_kernel(const T* __restrict__ k, const T* __restrict__ q_obs,
+                                                             float2* __restrict__ rec, int32_t* __restrict__ status, int n_obs,
+                                                             int ctx, int Hq, int Hkv, int D, int NP, float scale_log2) {
+  extern __shared__ __align__(128) unsigned char tsm[];
+  unsigned char* sA = tsm;                        // [D/8] column blocks of 16 core matrices (the 128-token block)
+  constexpr uint32_t LBO_A = 16 * 128 + 16;       // bytes between the column blocks of the key operand
+  unsigned char* sB = tsm + (D / 8) * LBO_A;      // [D/8][NP/8] core matrices of the queries
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(sB + (size_t)NP * D * 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 1);
+  const int hk = blockIdx.y, b = blockIdx.z, G = Hq / Hkv, nqh = n_obs * G, NQ = n_obs * Hq;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int tok0 = blockIdx.x * 128, n_tiles = ctx / 32;
+
+  if (wid == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sm_u32(tmem_slot)), "r"((uint32_t)NP) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(mbar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // keys: consecutive threads take consecutive 16-byte pieces of the rows (coalesced); piece c8 of row r goes
+  // to core matrix (c8, r / 8), row r % 8.  The column blocks are LBO_A apart: one extra 16 bytes per block
+  // spreads a warp's stores over all banks.
+  {
+    const int ppr = D / 8;  // pieces per row
+    const T* kb = k + (((size_t)b * Hkv + hk) * ctx + tok0) * D;
+    for (int idx = tid; idx < 128 * ppr; idx += 128) {
+      const int r = idx / ppr, c8 = idx - r * ppr;
+      const uint4 v = tok0 + r < ctx ? __ldg(reinterpret_cast<const uint4*>(kb) + idx) : make_uint4(0u, 0u, 0u, 0u);
+      *reinterpret_cast<uint4*>(sA + ((size_t)c8 * LBO_A + (size_t)(r >> 3) * 128 + (r & 7) * 16)) = v;
+    }
+  }
+  // queries (rows past the last one are zero)
+  for (int i = tid; i < NP * (D / 8); i += 128) {
+    const int qi = i / (D / 8), c8 = i - qi * (D / 8);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (qi < nqh) {
+      const int o = qi / G, hl = qi - o * G;
+      v = __ldg(reinterpret_cast<const uint4*>(q_obs + (((size_t)b * n_obs + o) * Hq + hk * G + hl) * D) + c8);
+    }
+    *reinterpret_cast<uint4*>(sB + ((size_t)(c8 * (NP / 8) + (qi >> 3)) * 128 + (qi & 7) * 16)) = v;
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // plain stores -> operands of the tensor core
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *tmem_slot;
+
+  if (tid == 0) {
+    // instruction descriptor: fp32 accumulator, 16-bit inputs of type T, both operands K-major, N = NP, M = 128
+    const uint32_t fmt = Tr<T>::MAGIC == 0x64006400u ? 0u : 1u;  // 0 = fp16, 1 = bf16
+    const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(NP >> 3) << 17) | ((128u >> 4) << 24);
+    const uint32_t a0 = sm_u32(sA), b0 = sm_u32(sB);
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint64_t da = umma_desc(a0 + (uint32_t)(2 * ks) * LBO_A, LBO_A, 128u);
+      const uint64_t db = umma_desc(b0 + (uint32_t)(2 * ks * (NP / 8)) * 128u, (uint32_t)(NP / 8) * 128u, 128u);
+      const uint32_t acc = ks > 0 ? 1u : 0u;
+      asm volatile(
+          "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+          "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n" ::"r"(tmem),
+          "l"(da), "l"(db), "r"(idesc), "r"(acc), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+          : "memory");
+    }
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(sm_u32(mbar)) : "memory");
+  }
+  // bounded wait for the products
+  bool ok = false;
+  for (uint32_t it = 0; it < (1u << 18) && !ok; ++it) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(done) : "r"(sm_u32(mbar)), "r"(0u) : "memory");
+    ok = done != 0;
+  }
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (!ok && tid == 0) record_check(status, CHECK_COPY_TIMEOUT);
+  const int tile = blockIdx.x * 4 + wid;
+  if (ok && tile < n_tiles) {
+    for (int c0 = 0; c0 < NP && c0 < nqh; c0 += 32) {
+      uint32_t v[32];
+      const uint32_t taddr = tmem + ((uint32_t)(wid * 32) << 16) + (uint32_t)c0;
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+          "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+            "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+            "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+            "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+          : "r"(taddr)
+          : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const int qi = c0 + j;
+        if (qi < nqh) {  // uniform across the warp
+          const float x = __uint_as_float(v[j]) * scale_log2;
+          float m = x;
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o2));
+          float l = exp2f(x - m);
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o2);
+          if (lane == 0) {
+            const int o = qi / G, hl = qi - o * G;
+            rec[((size_t)b * n_tiles + tile) * NQ + (size_t)o * Hq + hk * G + hl] = make_float2(m, l);
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (wid == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)NP) : "memory");
+}
+
 // Global maximum and 1 / denominator of every (observer, head): one warp per query, lanes stride over the
 // tiles, fixed shuffle trees.
 __global__ void __launch_bounds__(SCORE_THREADS) score_stats_kernel(const float2* __restrict__ rec, float2* __restrict__ stats,
@@ -141,17 +273,36 @@ QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, co
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSetDevice(h->cfg.device);
   float2* rec = static_cast<float2*>(scratch);
-  dim3 grid((n_tiles + SCORE_THREADS / 32 - 1) / (SCORE_THREADS / 32), g.Hkv, g.batch);
-  if (e == cudaSuccess && g.dtype == QEVICT_DTYPE_FP16) {
-    if (sm_a > 48 * 1024) e = cudaFuncSetAttribute(score_tiles_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_a);
-    if (e == cudaSuccess)
-      score_tiles_kernel<__half><<<grid, SCORE_THREADS, sm_a, s>>>((const __half*)k, (const __half*)q_obs, rec, n_obs, ctx_tokens,
-                                                                   g.Hq, g.Hkv, g.D, g.scale_log2);
-  } else if (e == cudaSuccess) {
-    if (sm_a > 48 * 1024) e = cudaFuncSetAttribute(score_tiles_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_a);
-    if (e == cudaSuccess)
-      score_tiles_kernel<__nv_bfloat16><<<grid, SCORE_THREADS, sm_a, s>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)q_obs, rec,
-                                                                          n_obs, ctx_tokens, g.Hq, g.Hkv, g.D, g.scale_log2);
+  if (nqh <= 128 && ctx_tokens % 128 == 0) {
+    // tensor-core path: NP = queries padded to a power of two (tensor-memory columns)
+    const int NP = nqh <= 32 ? 32 : (nqh <= 64 ? 64 : 128);
+    const size_t sm_t = (size_t)(g.D / 8) * (16 * 128 + 16) + (size_t)NP * g.D * 2 + 16;
+    dim3 tgrid(ctx_tokens / 128, g.Hkv, g.batch);
+    if (e == cudaSuccess && g.dtype == QEVICT_DTYPE_FP16) {
+      e = cudaFuncSetAttribute(score_tiles_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_t);
+      if (e == cudaSuccess)
+        score_tiles_tc_kernel<__half><<<tgrid, 128, sm_t, s>>>((const __half*)k, (const __half*)q_obs, rec, h->st.status, n_obs,
+                                                                ctx_tokens, g.Hq, g.Hkv, g.D, NP, g.scale_log2);
+    } else if (e == cudaSuccess) {
+      e = cudaFuncSetAttribute(score_tiles_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_t);
+      if (e == cudaSuccess)
+        score_tiles_tc_kernel<__nv_bfloat16><<<tgrid, 128, sm_t, s>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)q_obs, rec,
+                                                                       h->st.status, n_obs, ctx_tokens, g.Hq, g.Hkv, g.D, NP,
+                                                                       g.scale_log2);
+    }
+  } else {
+    dim3 grid((n_tiles + SCORE_THREADS / 32 - 1) / (SCORE_THREADS / 32), g.Hkv, g.batch);
+    if (e == cudaSuccess && g.dtype == QEVICT_DTYPE_FP16) {
+      if (sm_a > 48 * 1024) e = cudaFuncSetAttribute(score_tiles_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_a);
+      if (e == cudaSuccess)
+        score_tiles_kernel<__half><<<grid, SCORE_THREADS, sm_a, s>>>((const __half*)k, (const __half*)q_obs, rec, n_obs, ctx_tokens,
+                                                                     g.Hq, g.Hkv, g.D, g.scale_log2);
+    } else if (e == cudaSuccess) {
+      if (sm_a > 48 * 1024) e = cudaFuncSetAttribute(score_tiles_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_a);
+      if (e == cudaSuccess)
+        score_tiles_kernel<__nv_bfloat16><<<grid, SCORE_THREADS, sm_a, s>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)q_obs, rec,
+                                                                            n_obs, ctx_tokens, g.Hq, g.Hkv, g.D, g.scale_log2);
+    }
   }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) {

@@ -327,11 +327,14 @@ def test_config1_llama_shape_lockstep():
     run.close()
 
 
-@pytest.mark.parametrize("kw", [
-    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, batch=2, context=2048),
-    dict(dtype="fp16", head_dim=64, n_q_heads=3, n_kv_heads=1, window=64, group_size=32, context=1024),
-], ids=["bf16-d128-g4", "fp16-d64-w64"])
-def test_prefill_scores_on_the_gpu_match_the_oracle(kw):
+@pytest.mark.parametrize("kw,n_obs", [
+    (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, batch=2, context=2048), 6),     # tensor-core path, N = 32
+    (dict(dtype="fp16", head_dim=64, n_q_heads=3, n_kv_heads=1, window=64, group_size=32, context=1024), 6),
+    (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1, context=1024), 12),              # 96 queries: N = 128
+    (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, context=1056), 5),               # not a multiple of 128: CUDA cores
+    (dict(dtype="fp16", head_dim=128, n_q_heads=8, n_kv_heads=1, context=1024), 20),              # 160 queries: CUDA cores
+], ids=["bf16-d128-g4", "fp16-d64-w64", "bf16-96q", "bf16-ctx1056", "fp16-160q"])
+def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
     """Window scores of the prompt from observation queries: the GPU routine against the oracle's attention
     (raw mass per window summed over observers and heads), and a prefill_assign fed with them against the
     oracle fed with its own."""
@@ -339,7 +342,6 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw):
     ls = _lockstep()
     wl = _small("pscore", steps=4, **kw)
     cache = binding.QEvictCache(ls.gpu_config(wl))
-    n_obs = 6
     orcs = []
     ks, vs, qs = [], [], []
     for u in range(wl.n_units):
