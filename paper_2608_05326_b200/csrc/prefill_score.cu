@@ -175,22 +175,37 @@ __global__ void __launch_bounds__(128) score_tiles_tc_kernel(const T* __restrict
           : "r"(taddr)
           : "memory");
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // Lane = token, v[j] = logit of query c0 + j.  Both reductions run over the lanes for all 32 queries at
+      // once: a butterfly in which every step halves the values a lane still carries (31 shuffles instead of
+      // 160) and leaves lane L with the result of query c0 + L.
+      float x[32], r[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int qi = c0 + j;
-        if (qi < nqh) {  // uniform across the warp
-          const float x = __uint_as_float(v[j]) * scale_log2;
-          float m = x;
+      for (int j = 0; j < 32; ++j) { x[j] = __uint_as_float(v[j]) * scale_log2; r[j] = x[j]; }
 #pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o2));
-          float l = exp2f(x - m);
+      for (int st = 16; st >= 1; st >>= 1) {
+        const bool upper = (lane & st) != 0;
 #pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o2);
-          if (lane == 0) {
-            const int o = qi / G, hl = qi - o * G;
-            rec[((size_t)b * n_tiles + tile) * NQ + (size_t)o * Hq + hk * G + hl] = make_float2(m, l);
-          }
+        for (int j = 0; j < st; ++j) {
+          const float keep = upper ? r[j + st] : r[j], send = upper ? r[j] : r[j + st];
+          r[j] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, st));
         }
+      }
+      const float m_mine = r[0];  // maximum of query c0 + lane over the tile
+#pragma unroll
+      for (int j = 0; j < 32; ++j) r[j] = exp2f(x[j] - __shfl_sync(0xffffffffu, m_mine, j));
+#pragma unroll
+      for (int st = 16; st >= 1; st >>= 1) {
+        const bool upper = (lane & st) != 0;
+#pragma unroll
+        for (int j = 0; j < st; ++j) {
+          const float keep = upper ? r[j + st] : r[j], send = upper ? r[j] : r[j + st];
+          r[j] = keep + __shfl_xor_sync(0xffffffffu, send, st);
+        }
+      }
+      const int qi = c0 + lane;
+      if (qi < nqh) {
+        const int o = qi / G, hl = qi - o * G;
+        rec[((size_t)b * n_tiles + tile) * NQ + (size_t)o * Hq + hk * G + hl] = make_float2(m_mine, r[0]);
       }
     }
   }
