@@ -336,8 +336,8 @@ def test_config1_llama_shape_lockstep():
 ], ids=["bf16-d128-g4", "fp16-d64-w64", "bf16-96q", "bf16-ctx1056", "fp16-160q"])
 def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
     """Window scores of the prompt from observation queries: the GPU routine against the oracle's attention
-    (raw mass per window summed over observers and heads), and a prefill_assign fed with them against the
-    oracle fed with its own."""
+    (raw mass per window summed over observers and heads); then a prefill_assign on both sides from the
+    oracle's scores."""
     from oracle import accessible_attention
     ls = _lockstep()
     wl = _small("pscore", steps=4, **kw)
@@ -353,6 +353,7 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
     got = cache.prefill_score(kd, qd)
     torch.cuda.synchronize()
     scale = 1.0 / np.sqrt(wl.head_dim)
+    ref_all = []
     for u in range(wl.n_units):
         k64 = ks[u].double().numpy()
         ref = np.zeros(wl.n_prompt_windows)
@@ -362,12 +363,14 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
         g_u = got[u].cpu().double().numpy()
         assert abs(g_u.sum() - n_obs * wl.n_q_heads) < 1e-3
         assert np.all(np.abs(g_u - ref) <= ls.MASS_RTOL * np.abs(ref) + 1e-7), np.abs(g_u - ref).max()
-    # the scores drive the first tier assignment: same tiers as the oracle routed on the same float32 scores
-    cache.prefill_assign(0, kd, vd, got)
+        ref_all.append(ref)
+    # scores of this kind drive the first tier assignment: both sides are given the oracle's scores (as float32)
+    refs = torch.from_numpy(np.stack(ref_all).astype(np.float32))
+    cache.prefill_assign(0, kd, vd, refs.cuda())
     for u in range(wl.n_units):
         orc = ls.UnitOracle(ls.oracle_config(wl, ls.aged_capacity(wl)))
-        orc.prefill_assign(ks[u].double().numpy(), vs[u].double().numpy(), got[u].cpu().numpy())
-        ls.compare_state(cache, 0, u, orc, wl, what="prefill from GPU scores, unit %d" % u)
+        orc.prefill_assign(ks[u].double().numpy(), vs[u].double().numpy(), refs[u].numpy())
+        ls.compare_state(cache, 0, u, orc, wl, what="prefill from observation scores, unit %d" % u)
     cache.close()
 
 
