@@ -242,18 +242,19 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
       if (++m.open_fill == g.W) { m.has_open = false; m.open_fill = 0; m.aged++; }
     }
   }
-  DecodeParams p;
-  p.q = q; p.entries = h->st.entries; p.n_live = h->st.n_live; p.open_fill = h->st.open_fill;
-  p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
-  p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
-  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
-  QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
   int e_bound = 1;  // upper bound of every unit's work-list length, from the host's mirror of the window counts
   for (int l = l0; l < l1; ++l) {
     const LayerMirror& m = h->layers[l];
     const int e = g.Kfp + g.Kq + m.aged + (m.has_open ? 1 : 0);
     if (e > e_bound) e_bound = e;
   }
+  DecodeParams p;
+  p.e_bound = e_bound < g.EMAX ? e_bound : g.EMAX;
+  p.q = q; p.entries = h->st.entries; p.n_live = h->st.n_live; p.open_fill = h->st.open_fill;
+  p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
+  p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
+  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
+  QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
   QE_CUDA(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
   h->decode_steps++;
   return QEVICT_OK;

@@ -4,10 +4,10 @@
 // equation of the Methodology] and records, per (query head, window), the window's softmax
 // numerator, from which the combine kernel forms the window mass of Eq. 1.
 //
-// Work decomposition: CTA = (split, KV head, unit), 4 warps.  Warp `wid` of split `s` owns the work
-// list entries s*4+wid, s*4+wid + 4S, ...; the routing kernel interleaves Full and Quantized windows
-// in the list in proportion to their numbers (recent windows last), so every warp alternates between
-// bandwidth-heavy 16-bit tiles and arithmetic-heavy low-bit tiles all the way through its walk.  Each
+// Work decomposition: CTA = (split, KV head, unit), 4 warps.  Warp `wid` of split `s` owns one contiguous
+// run of the work list; the routing kernel interleaves Full and Quantized windows in the list in
+// proportion to their numbers (recent windows last), so every warp alternates between bandwidth-heavy
+// 16-bit tiles and arithmetic-heavy low-bit tiles all the way through its walk.  Each
 // warp runs an independent online softmax over its windows; the four warps are merged in shared
 // memory and the CTA writes one partial (m, l, O) per query head of its KV head.
 //
@@ -44,6 +44,7 @@ struct DecodeParams {
   float2* wrec;           // [n_units][EMAX][Hq]
   int32_t* status;
   int unit0, S, Hq, Hkv, G, EMAX, PF, PQ;
+  int e_bound;            // upper bound of every unit's work-list length (host's mirror of the window counts)
   uint32_t fp_page_bytes, q_page_bytes;
   float scale_log2;
 };
@@ -361,16 +362,19 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
 #pragma unroll
   for (int i = 0; i < MT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
 
-  // The work-list entries are fetched without waiting for the list length (the slots exist up to EMAX;
-  // what lies past the end is masked afterwards), so start-up costs one global round trip, not two.
-  const int stride = p.S * DECODE_WARPS;
-  const int first = s * DECODE_WARPS + wid;
+  // Every warp of the (unit, KV head) takes one contiguous run of the work list: the list interleaves Full and
+  // Quantized windows in proportion, so any run holds the same mix of 16-bit and low-bit pages (a strided walk
+  // would alias with the interleaving period for some split counts).  The runs are cut from the host's upper
+  // bound of the list length, so the entries are fetched without waiting for the length itself (the slots
+  // exist up to EMAX; what lies past the end is masked afterwards): start-up costs one global round trip.
+  const int n_warps = p.S * DECODE_WARPS, gw = s * DECODE_WARPS + wid;
+  const int run = p.e_bound / n_warps, extra = p.e_bound - run * n_warps;
+  const int first = gw * run + min(gw, extra), my_cap = run + (gw < extra ? 1 : 0);  // <= 32: the host picks S so
   uint2 my_ent = make_uint2(0u, 0u);
-  if (first + lane * stride < p.EMAX) my_ent = p.entries[(size_t)u * p.EMAX + first + (size_t)lane * stride];
+  if (lane < my_cap && first + lane < p.EMAX) my_ent = p.entries[(size_t)u * p.EMAX + first + lane];
   const int n_live = p.n_live[u];
   const int fill = p.open_fill[u];
-  // this warp's entries, one per lane (the host picks S so that a warp never owns more than 32)
-  const int my_n = first < n_live ? min(32, (n_live - first + stride - 1) / stride) : 0;
+  const int my_n = max(0, min(my_cap, n_live - first));
   if (lane >= my_n) my_ent = make_uint2(0u, 0u);
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
@@ -450,7 +454,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   for (int ci = 0; ci < my_n; ++ci) {
     const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, ci);
     const uint32_t kind = ex >> ENTRY_KIND_SHIFT;
-    const int e = first + ci * stride;
+    const int e = first + ci;
     const int valid = (kind == KIND_OPEN) ? fill : TT::W;
     float wsum[2] = {0.f, 0.f};
 #pragma unroll 1

@@ -93,7 +93,14 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
       if (++m.open_fill == g.W) { m.has_open = false; m.open_fill = 0; m.aged++; }
     }
   }
+  int e_bound = 1;
+  for (int l = l0; l < l1; ++l) {
+    const LayerMirror& m = h->layers[l];
+    const int eb = g.Kfp + g.Kq + m.aged + (m.has_open ? 1 : 0);
+    if (eb > e_bound) e_bound = eb;
+  }
   DecodeParams p;
+  p.e_bound = e_bound < g.EMAX ? e_bound : g.EMAX;
   p.q = q; p.entries = a.st.entries; p.n_live = a.st.n_live; p.open_fill = a.st.open_fill;
   p.fp_pool = a.st.fp_pool; p.q_pool = a.st.q_pool; p.o_part = a.st.o_part; p.ml = a.st.ml; p.wrec = a.st.wrec;
   p.status = a.st.status;
@@ -102,12 +109,6 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   e = h->decode_fn(p, a.n_units, stream);
   if (e != cudaSuccess) { h->last_error = std::string("attention: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
   h->launches++;
-  int e_bound = 1;
-  for (int l = l0; l < l1; ++l) {
-    const LayerMirror& m = h->layers[l];
-    const int eb = g.Kfp + g.Kq + m.aged + (m.has_open ? 1 : 0);
-    if (eb > e_bound) e_bound = eb;
-  }
   e = launch_combine(a, p.S, e_bound, out, stream);
   if (e != cudaSuccess) { h->last_error = std::string("combine: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
   h->launches++;
