@@ -379,13 +379,6 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
   // pieces per tile: full precision = 2 (key tile, value tile), quantized = 1 (the whole tile)
-  int n_pieces;
-  {
-    int mine = lane < my_n ? (((my_ent.x >> ENTRY_KIND_SHIFT) == KIND_Q) ? 1 : 2) * TILES : 0;
-#pragma unroll
-    for (int o2 = 16; o2 > 0; o2 >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o2);
-    n_pieces = mine;
-  }
   int pr_ci = 0, pr_tile = 0, pr_part = 0, issued = 0, consumed = 0;
   bool dead = false, pr_isq = false;
   const char* pr_base = nullptr;  // page of the producer's current entry (this KV head), set on its first piece
@@ -393,7 +386,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   const char* const q_unit = p.q_pool + (size_t)u * p.PQ * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
   const uint64_t l2pol = l2_evict_first_policy();
   auto issue_next = [&]() {  // warp-collective
-    if (issued >= n_pieces || dead) return;
+    if (pr_ci >= my_n || dead) return;  // every piece of every entry of this warp has been issued
     if (pr_tile == 0 && pr_part == 0) {
       const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, pr_ci), ey = __shfl_sync(0xffffffffu, my_ent.y, pr_ci);
       pr_isq = (ex >> ENTRY_KIND_SHIFT) == KIND_Q;
