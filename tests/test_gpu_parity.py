@@ -153,6 +153,35 @@ def test_more_than_4096_windows():
     run.close()
 
 
+def test_routing_diagnostics_match_the_oracle():
+    # tier-mass share and selection churn of the observation appendix, from the exported tables
+    from oracle import retained_windows, selection_churn, tier_mass_share
+    from paper_2608_05326_b200 import diagnostics
+    ls = _lockstep()
+    wl = _small("diag", steps=100, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, sink_windows=1)
+    run = ls.LockstepRun(wl, rebalance_interval=4)
+    prev_g = prev_o = None
+    churns = []
+    for t in range(wl.steps):
+        run.step(append=True)
+        if run.step_idx % 4 == 0:  # a routing event has just run
+            tab = run.cache.export_tables(0, 0)
+            orc = run.oracles[0]
+            mu_g, mu_o = diagnostics.tier_mass_share(tab), tier_mass_share(orc)
+            for k in mu_o:
+                assert abs(mu_g[k] - mu_o[k]) <= 1e-4 * max(mu_o[k], 1e-6) + 1e-9, (k, mu_g[k], mu_o[k])
+            assert abs(sum(mu_g.values()) - 1.0) < 1e-9
+            rg, ro = diagnostics.retained_windows(tab), retained_windows(orc)
+            assert rg == ro
+            if prev_g is not None:
+                cg, co = diagnostics.selection_churn(prev_g, rg), selection_churn(prev_o, ro)
+                assert cg == co
+                churns.append(cg)
+            prev_g, prev_o = rg, ro
+    assert len(churns) == wl.steps // 4 - 1 and all(0.0 <= c <= 1.0 for c in churns)
+    run.close()
+
+
 def test_many_candidates_and_tied_scores():
     # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
     # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides

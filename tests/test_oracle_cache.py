@@ -234,6 +234,28 @@ def test_decay_forgets_and_pnorm_prefers_peaks():
             assert s[0] == s[1] == s[2] == 64.0 and s[3] == 4.0   # one burst: 4^3; even: 4 x 1^3
 
 
+# ------------------------------------------------------------------------------------ diagnostics
+def test_tier_mass_share_and_selection_churn_on_a_hand_made_state():
+    """Tier-mass equation and selection-churn equation of the observation appendix on a state small enough to
+    do by hand: scores 1..8 on eight windows in tiers S F F Q Q E A(recent) O(pen)."""
+    from oracle import retained_windows, selection_churn, tier_mass_share
+    u = UnitOracle(_protected_cfg())
+    u.n_windows = 8
+    u.tier[:8] = [TIER_SINK, TIER_FULL, TIER_FULL, TIER_QUANT, TIER_QUANT, TIER_EVICTED, TIER_AGED, TIER_OPEN]
+    u.importance[:8] = [1, 2, 3, 4, 5, 6, 7, 8]
+    mu = tier_mass_share(u)
+    assert mu == {"full": 5 / 36, "quant": 9 / 36, "evicted": 6 / 36, "local": 16 / 36}
+    assert abs(sum(mu.values()) - 1.0) < 1e-15
+    before = retained_windows(u)
+    assert before == {1, 2, 3, 4}
+    u.tier[:8] = [TIER_SINK, TIER_FULL, TIER_QUANT, TIER_EVICTED, TIER_QUANT, TIER_EVICTED, TIER_FULL, TIER_OPEN]
+    after = retained_windows(u)
+    assert after == {1, 2, 4, 6}
+    assert selection_churn(before, after) == 1.0 - 3 / 5      # intersection {1,2,4}, union {1,2,3,4,6}
+    assert selection_churn(before, before) == 0.0 and selection_churn(set(), set()) == 0.0
+    assert selection_churn({1}, {2}) == 1.0
+
+
 def test_no_protected_regions_is_the_default():
     rng = np.random.default_rng(33)
     a, k, v, s = _prefilled(_small_cfg(), rng)
