@@ -47,6 +47,12 @@ in float32 with every operation rounded separately, so that the ranking -- an in
 decision taken on floating point -- is taken on the same numbers by any implementation.
 The prefill scores initialise S (or P) directly.
 
+Key-norm ranking (rank_mode 3; ranking-function appendix, key-norm equation): the score of a window is
+minus the mean L2 norm of its cached keys -- attention-free and fixed once the window is complete.  With several
+KV heads the norm is taken per head and averaged over heads and tokens (the paper writes one key vector per
+token and layer and does not say how heads combine).  Prefill scores are ignored; attention mass is still
+collected in the event accumulator but never enters the score.
+
 Parity unpinned: the page-id assignment order above is this build's own rule (the
 paper never speaks of pages), so nothing outside this file fixes it; and the
 prefill window scores are an input here (the paper only says that prompt attention
@@ -82,7 +88,7 @@ class OracleConfig:
     aged_windows: int = 2  # filled windows that may wait for the next routing event
     softmax_scale: float = 0.0  # 0 => 1/sqrt(head_dim)
     sink_windows: int = 0  # protected sink prefix, in windows
-    rank_mode: int = 0  # 0 cumulative attention (Eq. 1), 1 exponentially decayed, 2 attention p-norm
+    rank_mode: int = 0  # 0 cumulative attention (Eq. 1), 1 exponentially decayed, 2 attention p-norm, 3 key norm
     rank_param: float = 0.0  # lambda of the decayed score, p of the p-norm (integer >= 2)
     recent_windows: int = 0  # filled windows kept in the protected recent region
 
@@ -169,9 +175,14 @@ class UnitOracle:
             sl = slice(w * cfg.window, (w + 1) * cfg.window)
             self.fp[w] = (np.array(k[:, sl, :], dtype=np.float64), np.array(v[:, sl, :], dtype=np.float64))
             self.tier[w] = TIER_SINK if w < cfg.sink_windows else TIER_AGED
-            self.importance[w] = float(window_scores[w])
+            self.importance[w] = self.key_norm_score(self.fp[w][0]) if cfg.rank_mode == 3 else float(window_scores[w])
         self.n_windows = n
         self.rebalance(prefill=True)
+
+    @staticmethod
+    def key_norm_score(k):
+        """Key-norm equation: minus the mean over tokens (and KV heads) of the L2 norm of the keys; k [H_kv, W, d]."""
+        return -float(np.sqrt((k * k).sum(axis=-1)).mean())
 
     # --------------------------------------------------------------- append
     def _append(self, k_new, v_new):
@@ -197,6 +208,8 @@ class UnitOracle:
         if self.open_fill == cfg.window:
             self.tier[w] = TIER_AGED
             self.open_fill = 0
+            if cfg.rank_mode == 3:
+                self.importance[w] = self.key_norm_score(self.fp[w][0])
 
     # --------------------------------------------------------------- decode
     def accessible(self):
@@ -288,7 +301,7 @@ class UnitOracle:
     def rebalance(self, prefill=False):
         """Algorithm 1: TopK partition of the candidates, then promote / demote / evict with the ledger."""
         cfg = self.cfg
-        if cfg.rank_mode != 0 and not prefill:
+        if cfg.rank_mode in (1, 2) and not prefill:
             self.fold_event_mass()
         ranked = self.ranked_candidates()
         k_f, k_q = cfg.fp_budget_windows, cfg.q_budget_windows

@@ -234,6 +234,36 @@ def test_decay_forgets_and_pnorm_prefers_peaks():
             assert s[0] == s[1] == s[2] == 64.0 and s[3] == 4.0   # one burst: 4^3; even: 4 x 1^3
 
 
+def test_key_norm_ranking_keeps_the_windows_with_the_smallest_key_norms():
+    """Key-norm equation: score = minus the mean L2 norm of the window's keys; lower norms are retained first.
+    Checked against numpy.linalg.norm on the prompt and on the windows that fill during decoding."""
+    rng = np.random.default_rng(43)
+    cfg = _rank_cfg(3, 0.0, k_f=3, k_q=4)
+    ctx = 16 * 32
+    scale = np.repeat(np.linspace(0.5, 2.0, 16)[rng.permutation(16)], 32)  # every window its own key magnitude
+    k = round_to_dtype(rng.standard_normal((2, ctx, 64)) * scale[None, :, None], "fp16")
+    v = _rand_T(rng, (2, ctx, 64), "fp16")
+    u = UnitOracle(cfg)
+    u.prefill_assign(k, v, np.zeros(16, dtype=np.float32))            # the given scores are ignored
+    norms = np.linalg.norm(k.reshape(2, 16, 32, 64), axis=-1).mean(axis=(0, 2))
+    assert np.allclose(u.importance[:16], -norms, rtol=1e-12)
+    order = np.argsort(norms, kind="stable")
+    assert set(np.flatnonzero(u.tier[:16] == TIER_FULL)) == set(order[:3])
+    assert set(np.flatnonzero(u.tier[:16] == TIER_QUANT)) == set(order[3:7])
+    assert set(np.flatnonzero(u.tier[:16] == TIER_EVICTED)) == set(order[7:])
+    new_k = []
+    for t in range(64):
+        kn = round_to_dtype(rng.standard_normal((2, 64)) * (0.1 if t < 32 else 5.0), "fp16")
+        new_k.append(kn)
+        u.decode_attn(_rand_T(rng, (4, 64), "fp16"), kn, _rand_T(rng, (2, 64), "fp16"))
+    nk = np.stack(new_k, axis=1)                                       # [2, 64, 64]
+    n16, n17 = (np.linalg.norm(nk[:, a:a + 32], axis=-1).mean() for a in (0, 32))
+    assert np.isclose(u.importance[16], -n16, rtol=1e-12) and np.isclose(u.importance[17], -n17, rtol=1e-12)
+    u.rebalance()
+    assert u.tier[16] == TIER_FULL and u.tier[17] == TIER_EVICTED      # tiny keys are kept, huge keys go first
+    assert np.isclose(u.importance[16], -n16, rtol=1e-12)             # attention mass never entered the score
+
+
 # ------------------------------------------------------------------------------------ diagnostics
 def test_tier_mass_share_and_selection_churn_on_a_hand_made_state():
     """Tier-mass equation and selection-churn equation of the observation appendix on a state small enough to
