@@ -76,8 +76,11 @@ enum {
  * the mass is collected in an event accumulator u and folded into the score by every routing event after
  * prefill, for every stored window, in float32 with each operation rounded on its own:
  *   DECAYED  S <- lambda * S + u;   PNORM  P <- P + u^p (p - 1 multiplications); windows are ranked by
- *   P, which orders them as S_p = P^(1/p) does.  The prefill scores initialise S (or P) directly. */
-enum { QEVICT_RANK_CUMULATIVE = 0, QEVICT_RANK_DECAYED = 1, QEVICT_RANK_PNORM = 2 };
+ *   P, which orders them as S_p = P^(1/p) does.  The prefill scores initialise S (or P) directly.
+ * KEYNORM is attention-free: the score of a window is minus the mean L2 norm of its keys (per KV head, averaged
+ * over heads and tokens), fixed when the window is complete; window_scores of qevict_prefill_assign is
+ * ignored and may be NULL; the attention mass is still collected in u but never enters the score. */
+enum { QEVICT_RANK_CUMULATIVE = 0, QEVICT_RANK_DECAYED = 1, QEVICT_RANK_PNORM = 2, QEVICT_RANK_KEYNORM = 3 };
 /* ledger states */
 enum { QEVICT_LEDGER_NONE = 0, QEVICT_LEDGER_ACTIVE = 1, QEVICT_LEDGER_DORMANT = 2 };
 

@@ -14,7 +14,7 @@ QEVICT_OK = 0
 DTYPE_FP16, DTYPE_BF16 = 0, 1
 (QEVICT_TIER_NONE, QEVICT_TIER_OPEN, QEVICT_TIER_AGED, QEVICT_TIER_FULL, QEVICT_TIER_QUANT, QEVICT_TIER_EVICTED,
  QEVICT_TIER_SINK) = range(7)
-QEVICT_RANK_CUMULATIVE, QEVICT_RANK_DECAYED, QEVICT_RANK_PNORM = range(3)
+QEVICT_RANK_CUMULATIVE, QEVICT_RANK_DECAYED, QEVICT_RANK_PNORM, QEVICT_RANK_KEYNORM = range(4)
 TIER_NONE, TIER_OPEN, TIER_AGED, TIER_FULL, TIER_QUANT, TIER_EVICTED = range(6)
 LEDGER_NONE, LEDGER_ACTIVE, LEDGER_DORMANT = range(3)
 STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "NO_MEMORY", "UNSUPPORTED", "CUDA", "DEVICE_CHECK"]

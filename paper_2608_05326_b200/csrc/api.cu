@@ -71,7 +71,7 @@ const char* validate(const qevict_config* c) {
   if (c->window < 1 || c->max_context < c->window || c->max_context % c->window) return "max_context must be a positive multiple of window";
   if (c->group_size < 1 || c->window % c->group_size || c->head_dim % c->group_size) return "group_size must divide window and head_dim";
   if (c->rebalance_interval_hint < 0) return "rebalance_interval_hint < 0";
-  if (c->rank_mode < QEVICT_RANK_CUMULATIVE || c->rank_mode > QEVICT_RANK_PNORM) return "rank_mode must be a QEVICT_RANK_* value";
+  if (c->rank_mode < QEVICT_RANK_CUMULATIVE || c->rank_mode > QEVICT_RANK_KEYNORM) return "rank_mode must be a QEVICT_RANK_* value";
   if (c->rank_mode == QEVICT_RANK_DECAYED && !(c->rank_param > 0.f && c->rank_param <= 1.f)) return "decayed ranking needs 0 < rank_param <= 1";
   if (c->rank_mode == QEVICT_RANK_PNORM && !(c->rank_param >= 2.f && c->rank_param <= 8.f && c->rank_param == floorf(c->rank_param)))
     return "p-norm ranking needs an integer rank_param in 2..8";
@@ -139,6 +139,7 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.q_page = (int32_t*)take(U * g.NW * 4);
   s.importance = (float*)take(U * g.NW * 4);
   s.event_mass = (float*)take(U * g.NW * 4);
+  s.knorm_acc = (float*)take(U * 4);
   s.fp_owner = (int32_t*)take(U * g.PF * 4);
   s.q_owner = (int32_t*)take(U * g.PQ * 4);
   s.n_windows = (int32_t*)take(U * 4);
@@ -342,6 +343,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
     if (e == cudaSuccess) e = cudaMemset(h->st.q_page, 0xFF, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.importance, 0, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.event_mass, 0, U * g.NW * 4);
+    if (e == cudaSuccess) e = cudaMemset(h->st.knorm_acc, 0, U * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.fp_owner, 0xFF, U * g.PF * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.q_owner, 0xFF, U * g.PQ * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.n_windows, 0, U * 4);
@@ -414,7 +416,8 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   if (!h) return QEVICT_ERR_INVALID_ARG;
   int l0, l1;
   if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
-  if (!k || !v || !window_scores) return fail(h, QEVICT_ERR_INVALID_ARG, "k, v and window_scores must not be NULL");
+  if (!k || !v || (!window_scores && h->cfg.rank_mode != QEVICT_RANK_KEYNORM))
+    return fail(h, QEVICT_ERR_INVALID_ARG, "k, v and window_scores must not be NULL");
   const Geometry& g = h->geo;
   if (ctx_tokens < g.W || ctx_tokens % g.W) return fail(h, QEVICT_ERR_UNSUPPORTED, "ctx_tokens must be a positive multiple of window");
   if (ctx_tokens > h->cfg.max_context) return fail(h, QEVICT_ERR_INVALID_ARG, "ctx_tokens exceeds max_context");
@@ -425,6 +428,10 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   const KernelArgs a = make_args(h, l0, l1);
   const int n_prompt = ctx_tokens / g.W;
   QE_CUDA(h, launch_prefill_init(a, n_prompt, window_scores, s));
+  if (g.rank_mode == QEVICT_RANK_KEYNORM) {
+    QE_CUDA(h, launch_key_norm_scores(a, k, ctx_tokens, n_prompt, s));
+    h->launches++;
+  }
   QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
   QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kfp, s));
   QE_CUDA(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));

@@ -57,6 +57,7 @@ struct State {
   int32_t* q_page;      // [NW]
   float* importance;    // [NW]
   float* event_mass;    // [NW] mass since the last routing event (ranking functions other than Eq. 1)
+  float* knorm_acc;     // [1] sum of the key norms of the open window's tokens (key-norm ranking)
   int32_t* fp_owner;    // [PF] window holding the page, -1 free
   int32_t* q_owner;     // [PQ]
   int32_t* n_windows;   // [1]

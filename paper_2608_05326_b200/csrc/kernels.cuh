@@ -21,6 +21,8 @@ cudaError_t launch_combine(const KernelArgs& a, int n_splits, int e_bound, void*
 // routing event ---------------------------------------------------------------------------------------
 // P0 (first half): every prompt window becomes an aged candidate with the given score.
 cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt_windows, const float* scores, cudaStream_t s);
+// key-norm ranking: scores of the prompt windows = minus the mean key norm (k: [units][H_kv][ctx][d])
+cudaError_t launch_key_norm_scores(const KernelArgs& a, const void* k_prompt, int ctx, int n_prompt_windows, cudaStream_t s);
 // A3 + A4 + A7: rank, assign tiers, release / allocate pages, build migration lists and the work list.
 cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_capacity, cudaStream_t s);
 // A5 + A6: quantize the windows of the quantization list (source: their full-precision page, or the

@@ -192,6 +192,34 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
       vt[fpv_off(tk, ch0 + e)] = ve[e];
     }
   }
+  // key-norm ranking: the token's key norms (one per KV head) join the open window's sum; a window that is
+  // complete gets its score, minus the mean norm.  Fixed summation order.
+  float knorm_new = 0.f;
+  if (g.rank_mode == QEVICT_RANK_KEYNORM) {
+    __shared__ float s_sq[128 * MAXV];
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int v = tid + i * 128;
+      float ss = 0.f;
+      if (v < nvec) {
+        const T* ke = reinterpret_cast<const T*>(&kx[i]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { const float x = Tr<T>::to_float(ke[e]); ss = fmaf(x, x, ss); }
+      }
+      s_sq[v] = ss;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const int per_head = g.D / 8;
+      float tok = 0.f;
+      for (int h = 0; h < g.Hkv && h * per_head < 128 * MAXV; ++h) {
+        float ss = 0.f;
+        for (int j = 0; j < per_head; ++j) ss += s_sq[h * per_head + j];
+        tok += sqrtf(ss);
+      }
+      knorm_new = (is_new ? 0.f : a.st.knorm_acc[u]) + tok;
+    }
+  }
   if (tid == 0) {
     const size_t wi = (size_t)u * g.NW + window;
     const int e_idx = is_new ? n_live0 : n_live0 - 1;  // the open window is always the last entry
@@ -202,6 +230,7 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
       a.st.q_page[wi] = -1;
       a.st.ledger[wi] = QEVICT_LEDGER_NONE;
       a.st.importance[wi] = 0.f;
+      a.st.event_mass[wi] = 0.f;
       a.st.n_windows[u] = window + 1;
       a.st.n_live[u] = n_live0 + 1;
     }
@@ -210,6 +239,10 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
         make_uint2((uint32_t)window | ((full ? KIND_FP : KIND_OPEN) << ENTRY_KIND_SHIFT), (uint32_t)page);
     a.st.open_window[u] = full ? -1 : window;
     a.st.open_fill[u] = full ? 0 : slot + 1;
+    if (g.rank_mode == QEVICT_RANK_KEYNORM) {
+      a.st.knorm_acc[u] = knorm_new;
+      if (full) a.st.importance[wi] = -knorm_new / (float)(g.W * g.Hkv);
+    }
   }
 }
 
@@ -221,9 +254,38 @@ __global__ void prefill_init_kernel(const KernelArgs a, int n_prompt, const floa
   if (w < n_prompt) {
     const size_t wi = (size_t)u * g.NW + w;
     a.st.tier[wi] = w < g.n_sink ? QEVICT_TIER_SINK : QEVICT_TIER_AGED;
-    a.st.importance[wi] = scores[(size_t)ul * n_prompt + w];
+    a.st.importance[wi] = scores ? scores[(size_t)ul * n_prompt + w] : 0.f;
   }
   if (w == 0) a.st.n_windows[u] = n_prompt;
+}
+
+// ------------------------------------------------------------------------------- key-norm scores (prefill)
+// One CTA per (prompt window, unit): score = minus the mean over tokens and KV heads of the L2 norm of the keys.
+template <class T>
+__global__ void __launch_bounds__(128) key_norm_kernel(const KernelArgs a, const T* __restrict__ k_prompt, int ctx) {
+  const Geometry& g = a.geo;
+  const int w = blockIdx.x, ul = blockIdx.y, u = a.unit0 + ul, tid = threadIdx.x;
+  __shared__ float s_part[128];
+  float acc = 0.f;
+  for (int pair = tid; pair < g.W * g.Hkv; pair += 128) {  // (head, token of the window)
+    const int h = pair / g.W, tk = pair - h * g.W;
+    const uint4* row = reinterpret_cast<const uint4*>(k_prompt + (((size_t)ul * g.Hkv + h) * ctx + (size_t)w * g.W + tk) * g.D);
+    float ss = 0.f;
+    for (int v = 0; v < g.D / 8; ++v) {
+      const uint4 x = __ldg(row + v);
+      const T* e = reinterpret_cast<const T*>(&x);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { const float f = Tr<T>::to_float(e[j]); ss = fmaf(f, f, ss); }
+    }
+    acc += sqrtf(ss);
+  }
+  s_part[tid] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    float sum = 0.f;
+    for (int i = 0; i < 128; ++i) sum += s_part[i];
+    a.st.importance[(size_t)u * g.NW + w] = -sum / (float)(g.W * g.Hkv);
+  }
 }
 
 // ------------------------------------------------------------------------------------------- route
@@ -286,7 +348,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
 
   // ---- ranking functions other than Eq. 1: fold the event accumulator into the score of every stored
   // window (each operation rounded on its own, so that the ranking is taken on reproducible numbers) ----
-  if (g.rank_mode != QEVICT_RANK_CUMULATIVE && !prefill) {
+  if ((g.rank_mode == QEVICT_RANK_DECAYED || g.rank_mode == QEVICT_RANK_PNORM) && !prefill) {
     float* score = a.st.importance + (size_t)u * g.NW;
     float* ev = a.st.event_mass + (size_t)u * g.NW;
     const int p = (int)g.rank_param;
@@ -326,7 +388,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   const int chunk = (nw + NT - 1) / NT;
   constexpr int PRE = 10;
   const int cs = (g.NW + NT - 1) / NT;  // rows of the table per thread (not of the windows in use)
-  if (cs <= PRE && (g.rank_mode == QEVICT_RANK_CUMULATIVE || prefill)) {
+  if (cs <= PRE && (g.rank_mode == QEVICT_RANK_CUMULATIVE || g.rank_mode == QEVICT_RANK_KEYNORM || prefill)) {
     // Small tables: every thread requests all five columns of its rows at once, before it knows how many
     // windows exist or which of them are candidates (rows past the last window hold state NONE), so the
     // whole gather costs one global round trip.
@@ -688,6 +750,13 @@ cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_
     return launch_pdl(append_kernel<__half>, dim3(a.n_units), dim3(128), 0, s, a, (const __half*)k_new, (const __half*)v_new);
   return launch_pdl(append_kernel<__nv_bfloat16>, dim3(a.n_units), dim3(128), 0, s, a, (const __nv_bfloat16*)k_new,
                     (const __nv_bfloat16*)v_new);
+}
+
+cudaError_t launch_key_norm_scores(const KernelArgs& a, const void* k_prompt, int ctx, int n_prompt, cudaStream_t s) {
+  dim3 grid(n_prompt, a.n_units);
+  if (a.geo.dtype == QEVICT_DTYPE_FP16) key_norm_kernel<__half><<<grid, 128, 0, s>>>(a, (const __half*)k_prompt, ctx);
+  else key_norm_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(a, (const __nv_bfloat16*)k_prompt, ctx);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_init(const KernelArgs& a, int n_prompt, const float* scores, cudaStream_t s) {

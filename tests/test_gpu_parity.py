@@ -119,10 +119,11 @@ def test_protected_sink_and_recent_windows(kw):
         run.close()
 
 
-@pytest.mark.parametrize("mode,param", [(1, 0.9), (1, 0.5), (2, 3.0), (2, 2.0)])
+@pytest.mark.parametrize("mode,param", [(1, 0.9), (1, 0.5), (2, 3.0), (2, 2.0), (3, 0.0)])
 def test_ranking_function_variants(mode, param):
     # decayed attention and attention p-norm: the mass is collected per routing event and folded into the score
-    # in float32 by the routing kernel; tiers, pages and codes must still match bit for bit
+    # in float32 by the routing kernel; key norm (mode 3): the score is minus the mean key norm of a complete
+    # window; tiers, pages and codes must still match bit for bit
     ls = _lockstep()
     wl = _small("rank", steps=72, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, rank_mode=mode, rank_param=param)
     run = ls.LockstepRun(wl, rebalance_interval=3)
@@ -419,8 +420,8 @@ def _random_workloads(n, seed=20260805):
         n_win = int(rng.integers(10, 28))
         k_f = int(rng.integers(0, 6))
         k_q = int(rng.integers(0 if k_f else 1, 9))
-        mode = int(rng.choice([0, 0, 1, 2]))
-        param = {0: 0.0, 1: float(rng.choice([0.5, 0.9, 0.99])), 2: float(rng.choice([2, 3]))}[mode]
+        mode = int(rng.choice([0, 0, 1, 2, 3]))
+        param = {0: 0.0, 1: float(rng.choice([0.5, 0.9, 0.99])), 2: float(rng.choice([2, 3])), 3: 0.0}[mode]
         interval = int(rng.choice([1, 2, 7, window, window + 5]))
         wl = _small("fuzz%d" % i, dtype=str(rng.choice(["fp16", "bf16"])), head_dim=head_dim, n_q_heads=gq * n_kv,
                     n_kv_heads=n_kv, window=window, group_size=group, quant_bits=int(rng.choice([2, 4])),
