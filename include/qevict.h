@@ -125,7 +125,9 @@ typedef struct {
 /* Bytes of one Full window and one Quantized window (all KV heads, keys and values), and the tier
  * capacities K_f = floor((1-q_frac) * hist_bytes / M_f), K_q = floor(q_frac * hist_bytes / M_q)
  * [tier-capacity equation].  M_q counts packed codes plus one (scale, zero) pair of the execution
- * datatype per group [memory accounting appendix].  Host arithmetic only; any output pointer may be
+ * datatype per group [memory accounting appendix].  hist_bytes is the historical budget: what is left of the
+ * total after the protected regions, (sink_windows + recent_windows + 1) * M_f, have been set aside [budget
+ * constraint: B_sink + B_local + the tiers <= B_total].  Host arithmetic only; any output pointer may be
  * NULL.  Only the shape fields of `cfg` are read. */
 QEVICT_API qevict_status qevict_budget_from_bytes(const qevict_config* cfg, uint64_t hist_bytes, double q_frac,
                                        int32_t* k_f, int32_t* k_q, uint64_t* m_f, uint64_t* m_q);
