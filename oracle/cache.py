@@ -53,6 +53,12 @@ KV heads the norm is taken per head and averaged over heads and tokens (the pape
 token and layer and does not say how heads combine).  Prefill scores are ignored; attention mass is still
 collected in the event accumulator but never enters the score.
 
+One-way policy (promotion ablation appendix: Full -> Quantized -> Evicted, "quantized windows may subsequently
+be evicted but cannot return to the full tier", same capacities and ranking): the paper gives no algorithm for
+it; the reading taken is Algorithm 1 with the Full tier drawn from the candidates that are not Quantized --
+F' = TopK_{K_f} of the ranked candidates whose state is not Quantized, Q' = TopK_{K_q} of the ranked remainder,
+E' = the rest.
+
 Parity unpinned: the page-id assignment order above is this build's own rule (the
 paper never speaks of pages), so nothing outside this file fixes it; and the
 prefill window scores are an input here (the paper only says that prompt attention
@@ -90,6 +96,7 @@ class OracleConfig:
     sink_windows: int = 0  # protected sink prefix, in windows
     rank_mode: int = 0  # 0 cumulative attention (Eq. 1), 1 exponentially decayed, 2 attention p-norm, 3 key norm
     rank_param: float = 0.0  # lambda of the decayed score, p of the p-norm (integer >= 2)
+    one_way: bool = False  # no promotion: a Quantized window never returns to the Full tier
     recent_windows: int = 0  # filled windows kept in the protected recent region
 
     @property
@@ -305,9 +312,15 @@ class UnitOracle:
             self.fold_event_mass()
         ranked = self.ranked_candidates()
         k_f, k_q = cfg.fp_budget_windows, cfg.q_budget_windows
-        new_f = ranked[:k_f]
-        new_q = ranked[k_f : k_f + k_q]
-        new_e = ranked[k_f + k_q :]
+        if cfg.one_way:
+            new_f = np.array([w for w in ranked if self.tier[w] != TIER_QUANT][:k_f], dtype=ranked.dtype)
+            in_f = set(int(w) for w in new_f)
+            rest = np.array([w for w in ranked if int(w) not in in_f], dtype=ranked.dtype)
+            new_q, new_e = rest[:k_q], rest[k_q:]
+        else:
+            new_f = ranked[:k_f]
+            new_q = ranked[k_f : k_f + k_q]
+            new_e = ranked[k_f + k_q :]
 
         promotions = sorted(int(w) for w in new_f if self.tier[w] == TIER_QUANT)
         demotions = sorted(int(w) for w in new_q if self.tier[w] != TIER_QUANT)

@@ -264,6 +264,42 @@ def test_key_norm_ranking_keeps_the_windows_with_the_smallest_key_norms():
     assert np.isclose(u.importance[16], -n16, rtol=1e-12)             # attention mass never entered the score
 
 
+def test_one_way_policy_never_promotes():
+    """Promotion ablation: Full -> Quantized -> Evicted only.  Against a brute-force statement of the reading
+    (Full tier = best K_f candidates that are not Quantized; Quantized tier = best K_q of the rest) on random
+    scores, and against the bidirectional policy on the same scores."""
+    rng = np.random.default_rng(44)
+    cfg1 = OracleConfig(4, 2, 64, "fp16", 32, 4, 32, 3, 5, 40 * 32, aged_windows=2, one_way=True)
+    cfg2 = OracleConfig(4, 2, 64, "fp16", 32, 4, 32, 3, 5, 40 * 32, aged_windows=2)
+    a, k, v, s0 = _prefilled(cfg1, rng, ctx_windows=20)
+    b = UnitOracle(cfg2)
+    b.prefill_assign(k, v, s0)
+    assert np.array_equal(a.tier, b.tier)                       # nothing is Quantized before the first event
+    differed = False
+    for it in range(30):
+        scores = rng.random(a.n_windows)
+        a.importance[: a.n_windows] = scores
+        b.importance[: b.n_windows] = scores
+        t0 = a.tier[: a.n_windows].copy()
+        cand = [w for w in range(a.n_windows) if t0[w] in (TIER_FULL, TIER_QUANT, TIER_AGED)]
+        order = sorted(cand, key=lambda w: (-np.float32(scores[w]), w))
+        exp_f = [w for w in order if t0[w] != TIER_QUANT][:3]
+        rest = [w for w in order if w not in exp_f]
+        exp_q, exp_e = rest[:5], rest[5:]
+        a.rebalance()
+        b.rebalance()
+        assert set(np.flatnonzero(a.tier[: a.n_windows] == TIER_FULL)) == set(exp_f)
+        assert set(np.flatnonzero(a.tier[: a.n_windows] == TIER_QUANT)) == set(exp_q)
+        assert all(a.tier[w] == TIER_EVICTED for w in exp_e)
+        assert all(t0[w] != TIER_QUANT for w in exp_f)          # no window came back from the Quantized tier
+        differed = differed or not np.array_equal(a.tier[: a.n_windows], b.tier[: b.n_windows])
+        if not np.array_equal(a.tier[: a.n_windows], b.tier[: b.n_windows]):
+            b.tier[:] = a.tier; b.ledger_flag[:] = a.ledger_flag      # keep the two comparable (states only)
+            break
+    assert a.stats["promotions"] == 0
+    assert differed                                              # the bidirectional policy does promote here
+
+
 # ------------------------------------------------------------------------------------ diagnostics
 def test_tier_mass_share_and_selection_churn_on_a_hand_made_state():
     """Tier-mass equation and selection-churn equation of the observation appendix on a state small enough to
