@@ -110,6 +110,9 @@ typedef struct {
                                 the recent region] */
   int32_t rank_mode;         /* QEVICT_RANK_*: which score orders the candidates [ranking-function appendix] */
   float rank_param;          /* lambda of the decayed score (0 < lambda <= 1); p of the p-norm (integer 2..8) */
+  int32_t one_way;           /* 1: no promotion [promotion ablation: Full -> Quantized -> Evicted].  The paper gives
+                                only the transition diagram; reading: the Full tier is the best K_f candidates that
+                                are not Quantized, the Quantized tier the best K_q of all the others.  0: Algorithm 1 */
 } qevict_config;
 
 typedef struct {

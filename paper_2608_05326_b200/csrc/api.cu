@@ -75,6 +75,7 @@ const char* validate(const qevict_config* c) {
   if (c->rank_mode == QEVICT_RANK_DECAYED && !(c->rank_param > 0.f && c->rank_param <= 1.f)) return "decayed ranking needs 0 < rank_param <= 1";
   if (c->rank_mode == QEVICT_RANK_PNORM && !(c->rank_param >= 2.f && c->rank_param <= 8.f && c->rank_param == floorf(c->rank_param)))
     return "p-norm ranking needs an integer rank_param in 2..8";
+  if (c->one_way != 0 && c->one_way != 1) return "one_way must be 0 or 1";
   if (c->sink_windows < 0 || c->recent_windows < 0) return "sink_windows and recent_windows must be >= 0";
   if (c->sink_windows + c->recent_windows > c->max_context / c->window) return "protected windows exceed max_context";
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return "softmax_scale must be finite and >= 0";
@@ -100,7 +101,7 @@ void make_geometry(const qevict_config& c, Geometry& g) {
   const int r = c.rebalance_interval_hint > 0 ? c.rebalance_interval_hint : c.window;
   g.aged_cap = (r + g.W - 1) / g.W + 1;
   g.n_sink = c.sink_windows; g.n_recent = c.recent_windows;
-  g.rank_mode = c.rank_mode; g.rank_param = c.rank_param;
+  g.rank_mode = c.rank_mode; g.rank_param = c.rank_param; g.one_way = c.one_way != 0;
   g.Kfp = g.Kf + g.n_sink + g.n_recent;
   g.PF = g.Kfp + g.aged_cap + 1;
   g.PQ = g.Kq + g.Kf;

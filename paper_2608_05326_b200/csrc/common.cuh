@@ -39,6 +39,7 @@ struct Geometry {
   int aged_cap;  // filled windows that may wait for a routing event
   int n_sink, n_recent;  // protected windows: sink prefix, recent region (besides the open window)
   int rank_mode;     // QEVICT_RANK_*
+  int one_way;       // 1: a Quantized window never returns to the Full tier
   float rank_param;  // lambda or p
   int Kfp;       // K_f + n_sink + n_recent: windows that may need a full-precision page in one event
   int tiles;     // W / 32

@@ -468,7 +468,31 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
 
   // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
   // Quantized, remainder -> Evicted -----------------------------------------------------------------
-  if (n_cand <= 256) {
+  if (g.one_way) {
+    // One-way policy (no promotion): the Full tier is drawn from the candidates that are not Quantized, the
+    // Quantized tier from everything else.  Two counting ranks (this is a diagnostic policy: no selection path).
+    constexpr uint8_t UNDECIDED = 0x7F;
+    for (int c = tid; c < n_cand; c += NT) {
+      const unsigned long long mine = keys[c];
+      if ((uint32_t)(mine >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
+      uint8_t nt = UNDECIDED;
+      if (ctier[c] != QEVICT_TIER_QUANT) {
+        int pos = 0;
+        for (int i = 0; i < n_cand; ++i) pos += (ctier[i] != QEVICT_TIER_QUANT && keys[i] < mine) ? 1 : 0;
+        if (pos < g.Kf) nt = QEVICT_TIER_FULL;
+      }
+      cnew[c] = nt;
+    }
+    __syncthreads();
+    for (int c = tid; c < n_cand; c += NT) {
+      if (cnew[c] != UNDECIDED) continue;
+      const unsigned long long mine = keys[c];
+      int pos = 0;  // smaller keys among the candidates outside the new Full tier (pinned windows hold the largest keys)
+      for (int i = 0; i < n_cand; ++i) pos += (cnew[i] != QEVICT_TIER_FULL && !(cnew[i] & PINNED) && keys[i] < mine) ? 1 : 0;
+      // written only after the count: other threads test this entry for "not Full", which holds before and after
+      cnew[c] = pos < g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED;
+    }
+  } else if (n_cand <= 256) {
     // rank of a key = number of smaller keys (all keys are distinct); two adjacent lanes share a key and
     // count over one half of the keys each
     const int half = tid & 1, i0 = half ? n_cand / 2 : 0, i1 = half ? n_cand : n_cand / 2;

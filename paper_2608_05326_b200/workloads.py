@@ -46,6 +46,7 @@ class Workload:
     recent_windows: int = 0  # filled windows kept in the protected recent region
     rank_mode: int = 0       # 0 cumulative attention, 1 exponentially decayed, 2 attention p-norm
     rank_param: float = 0.0  # lambda or p
+    one_way: bool = False    # no promotion (promotion ablation)
 
     @property
     def n_units(self):

@@ -183,6 +183,23 @@ def test_routing_diagnostics_match_the_oracle():
     run.close()
 
 
+@pytest.mark.parametrize("kw", [dict(), dict(context=16384, n_q_heads=1, n_kv_heads=1, fp_budget_windows=120, q_budget_windows=260, steps=8)],
+                         ids=["small", "380-candidates"])
+def test_one_way_policy(kw):
+    # no promotion: Quantized windows leave their tier only by eviction; tiers, pages and codes bit for bit
+    ls = _lockstep()
+    wl = _small("oneway", **{**dict(steps=72, dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, one_way=True), **kw})
+    run = ls.LockstepRun(wl, rebalance_interval=1, score_mode="synthetic")
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    st = run.cache.stats()
+    assert st["promotions"] == 0 == run.oracles[0].stats["promotions"]
+    assert st["deletions"] == run.oracles[0].stats["deletions"] and st["quantizations"] == run.oracles[0].stats["quantizations"]
+    run.close()
+
+
 def test_many_candidates_and_tied_scores():
     # more candidates than the counting rank handles (radix selection of the two cuts), with prefill scores
     # on 7 levels, so that both cuts fall inside large groups of equal scores and the window index decides
