@@ -375,6 +375,8 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   const int n_live = p.n_live[u];
   const int fill = p.open_fill[u];
   const int my_n = max(0, min(my_cap, n_live - first));
+  // the runs cover the host's bound of the list length: a longer list would be attended to only in part
+  if (n_live > p.e_bound && s == 0 && threadIdx.x == 0) record_check(p.status, CHECK_ENTRY_OVERFLOW);
   if (lane >= my_n) my_ent = make_uint2(0u, 0u);
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
