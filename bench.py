@@ -58,6 +58,10 @@ def parse_args():
     ap.add_argument("--prefill-score", type=int, default=0, metavar="N_OBS",
                     help="instead of the decode loop: time qevict_prefill_score (window scores of one layer's prompt from "
                          "N_OBS observation queries per head) and print its own JSON line")
+    ap.add_argument("--timeline", action="store_true",
+                    help="instead of the throughput run: load the tracing build of the library and print, per kernel, the "
+                         "median start-to-end interval inside the pipelined step and the median gap to the kernel before "
+                         "(device timer stamps; not a bench value)")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -185,9 +189,11 @@ def attention_kernel_bytes(wl, stats, n_splits_hint=None):
 
 
 def run_ours(args, rank, world):
+    if args.timeline:
+        os.environ["QEVICT_TRACE_LIB"] = "1"  # read when the binding is first imported
     from paper_2608_05326_b200 import binding, build
     if rank == 0:
-        build.build()  # no-op when the in-tree library is newer than its sources
+        build.build(trace=args.timeline)  # no-op when the in-tree library is newer than its sources
     if world > 1:
         torch.distributed.barrier()
     dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
@@ -231,6 +237,13 @@ def run_ours(args, rank, world):
     t = 0
     for _ in range(W):
         step(t); t += 1
+    if args.timeline:
+        cache.kernel_timeline()  # restart the record after the warm-up
+        for _ in range(min(K, 250)):  # the library records 512 calls (two per step)
+            step(t); t += 1
+        line = timeline_summary(cache.kernel_timeline(), wl)
+        cache.close()
+        return line, wl
     # ---- timed region: device-resident inputs ----
     launches0 = cache.launch_count()
     sampler = ClockSampler(dev.index)
@@ -323,6 +336,29 @@ def run_ours(args, rank, world):
 
 
 # ------------------------------------------------------------------------------------- CPU oracle
+def timeline_summary(records, wl):
+    """Per kernel: median duration and median gap since the end of the launch before it, over the launches the
+    tracing library recorded."""
+    import statistics
+    dur, gap, period = {}, {}, []
+    last_append = None
+    for i, (name, t0, t1) in enumerate(records):
+        dur.setdefault(name, []).append(t1 - t0)
+        if i:
+            gap.setdefault(name, []).append(t0 - records[i - 1][2])
+        if name == "append":
+            if last_append is not None:
+                period.append(t0 - last_append)
+            last_append = t0
+    med = statistics.median
+    return {"metric": "kernel_timeline", "unit": "us", "data": "synthetic", "launches": len(records),
+            "config": {"workload": wl.name},
+            "median_us": {k: round(med(v), 2) for k, v in dur.items()},
+            "median_gap_before_us": {k: round(med(v), 2) for k, v in gap.items()},
+            "median_step_period_us": round(med(period), 2) if period else None,
+            "last_step": [(n, round(a, 2), round(b, 2)) for n, a, b in records[-5:]]}
+
+
 def oracle_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -438,7 +474,7 @@ def main():
     res = run_ours(args, rank, world)
     if rank == 0:
         line, wl = res
-        if not args.no_cpu_baseline and world >= 1:
+        if not args.timeline and not args.no_cpu_baseline and world >= 1:
             small = replace(wl, steps=256, seed=wl.seed)
             value, sample, _, _ = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds)
             line["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample}

@@ -281,6 +281,18 @@ QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enabl
 QEVICT_API qevict_status qevict_kernel_time(qevict_handle h, double* total_ms, uint64_t* n_launches);
 QEVICT_API qevict_status qevict_kernel_times(qevict_handle h, double* total_ms, uint64_t* n_launches);
 
+/* Kernel timeline (tracing build of the library only: the same sources compiled with -DQEVICT_TRACE, in which
+ * every warp of the five step kernels stamps the GPU's nanosecond timer when it starts and when it ends).
+ * Synchronises the device and returns the launches made since the previous call of this function (those of the
+ * first 512 API calls; later ones are not recorded), oldest first, the most recent max_records of them:
+ * kernel[i] (0 append, 1 attention, 2 combine, 3 route, 4 migrate), start_us[i] = earliest warp start and
+ * end_us[i] = latest warp end, in microseconds from the first returned start (host arrays of max_records);
+ * *n_records = how many were written.  Then clears the record.  Unlike CUDA events around a launch, this sees
+ * the kernels inside the running pipeline, where the next kernel's launch overlaps the current one.
+ * QEVICT_ERR_UNSUPPORTED (and *n_records = 0) in the normal build. */
+QEVICT_API qevict_status qevict_kernel_timeline(qevict_handle h, int32_t max_records, int32_t* kernel, double* start_us,
+                                                double* end_us, int32_t* n_records);
+
 /* Number of kernels this handle has launched since creation (host counter). */
 QEVICT_API uint64_t qevict_launch_count(qevict_handle h);
 

@@ -9,6 +9,11 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqevict.so")
+# QEVICT_TRACE_LIB=1 loads the tracing variant (build.build(trace=True)): the same kernels plus %globaltimer
+# stamps, which qevict_kernel_timeline reads.  It is a measuring aid; numbers reported as throughput come from
+# the normal library.
+if os.environ.get("QEVICT_TRACE_LIB", "0") not in ("", "0"):
+    LIB_PATH = os.path.join(_HERE, "libqevict_trace.so")
 
 QEVICT_OK = 0
 DTYPE_FP16, DTYPE_BF16 = 0, 1
@@ -63,6 +68,8 @@ _SIGNATURES = {
     "qevict_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32]),
     "qevict_kernel_time": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
     "qevict_kernel_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
+    "qevict_kernel_timeline": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_double),
+                                        C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
     "qevict_prefill_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -82,7 +89,7 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError("libqevict.so is missing: run `python -m paper_2608_05326_b200.build` "
+            raise RuntimeError(os.path.basename(LIB_PATH) + " is missing: run `python -m paper_2608_05326_b200.build` "
                                "(or __graft_entry__.build()) first; there is no fallback path")
         handle = C.CDLL(LIB_PATH)
         for name, (res, args) in _SIGNATURES.items():
@@ -199,6 +206,15 @@ def qevict_kernel_times(h):
     return {name: (ms[i], n[i]) for i, name in enumerate(KERNEL_NAMES)}
 
 
+def qevict_kernel_timeline(h, max_records=2560):
+    kid = (C.c_int32 * max_records)()
+    t0 = (C.c_double * max_records)()
+    t1 = (C.c_double * max_records)()
+    n = C.c_int32(0)
+    _check(lib().qevict_kernel_timeline(h, max_records, kid, t0, t1, C.byref(n)), h)
+    return [(KERNEL_NAMES[kid[i]] if 0 <= kid[i] < len(KERNEL_NAMES) else "?", t0[i], t1[i]) for i in range(n.value)]
+
+
 def qevict_get_stats(h, layer=-1):
     st = qevict_stats()
     _check(lib().qevict_get_stats(h, layer, C.byref(st)), h)
@@ -282,6 +298,11 @@ class QEvictCache:
     def kernel_times(self):
         """{kernel name: (summed milliseconds, launches)} since the last call."""
         return qevict_kernel_times(self.handle)
+
+    def kernel_timeline(self, max_records=2560):
+        """[(kernel name, start, end)] of the launches since the last call (first 512 API calls), oldest first, in
+        microseconds from the first start; tracing library only (QEVICT_TRACE_LIB=1)."""
+        return qevict_kernel_timeline(self.handle, max_records)
 
     def stats(self, layer=-1):
         return qevict_get_stats(self.handle, layer)

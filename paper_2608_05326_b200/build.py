@@ -10,6 +10,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libqevict.so")
+# the same sources with -DQEVICT_TRACE: every step kernel stamps %globaltimer at its first CTA's start and its
+# last CTA's end (qevict_kernel_timeline reads the stamps); a separate library, so that the normal one carries
+# none of it
+OBJ_TRACE = os.path.join(HERE, "build_trace")
+LIB_TRACE = os.path.join(HERE, "libqevict_trace.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -28,43 +33,46 @@ def _sources():
     return sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
-def _stale():
-    if not os.path.exists(LIB):
+def _stale(lib=LIB):
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "qevict.h"))
     deps.append(os.path.abspath(__file__))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def _compile(nvcc, src, verbose):
-    obj = os.path.join(OBJ, src[:-3] + ".o")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
+def _compile(nvcc, src, verbose, trace=False):
+    obj = os.path.join(OBJ_TRACE if trace else OBJ, src[:-3] + ".o")
+    cmd = [nvcc] + NVCC_FLAGS + (["-DQEVICT_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else []) + \
+          ["-c", os.path.join(CSRC, src), "-o", obj]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s" % (src, r.stderr))
     return obj, r.stderr
 
 
-def build(force=False, verbose=False):
-    """Compile and link the library if any source is newer than it.  Returns the library path."""
-    if not force and not _stale():
-        return LIB
+def build(force=False, verbose=False, trace=False):
+    """Compile and link the library (the tracing variant with trace=True) if any source is newer than it.
+    Returns the library path."""
+    lib = LIB_TRACE if trace else LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = _nvcc()
-    os.makedirs(OBJ, exist_ok=True)
+    os.makedirs(OBJ_TRACE if trace else OBJ, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as ex:
-        results = list(ex.map(lambda s: _compile(nvcc, s, verbose), _sources()))
+        results = list(ex.map(lambda s: _compile(nvcc, s, verbose, trace), _sources()))
     if verbose:
         for _, log in results:
             sys.stderr.write(log)
     objs = [o for o, _ in results]
-    r = subprocess.run([nvcc, "-shared", "-o", LIB] + objs + ["-Xcompiler", "-fvisibility=hidden"],
+    r = subprocess.run([nvcc, "-shared", "-o", lib] + objs + ["-Xcompiler", "-fvisibility=hidden"],
                        capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError("link failed:\n" + r.stderr)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

@@ -157,7 +157,10 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.ml = (float*)take(U * g.Hq * (size_t)MAX_SPLITS * 2 * 4);
   s.wrec = (float2*)take(U * g.Hq * (size_t)g.EMAX * 8);
   s.mass_e = (float*)take(U * (size_t)g.EMAX * 4);
-  s.status = (int32_t*)take(256);
+  s.status = (int32_t*)take(STATUS_BYTES);
+#ifdef QEVICT_TRACE
+  s.trace = (unsigned long long*)take(TRACE_BYTES);
+#endif
   char* sq = take(U * g.Hq * (size_t)g.D * 2);
   char* sk = take(U * g.Hkv * (size_t)g.D * 2);
   char* sv = take(U * g.Hkv * (size_t)g.D * 2);
@@ -174,12 +177,26 @@ bool layer_range(qevict_handle h, int layer, int* l0, int* l1) {
   return true;
 }
 
+#ifdef QEVICT_TRACE
+// {start = all ones, end = 0} in the first `calls` call blocks of the timeline.
+cudaError_t trace_clear(qevict_handle h, uint32_t calls) {
+  if (!calls) return cudaSuccess;
+  std::vector<unsigned long long> init(calls * TRACE_CALL_WORDS);
+  for (size_t i = 0; i < init.size(); i += 2) { init[i] = ~0ull; init[i + 1] = 0ull; }
+  return cudaMemcpy(h->st.trace, init.data(), init.size() * 8, cudaMemcpyHostToDevice);
+}
+#endif
+
 KernelArgs make_args(qevict_handle h, int l0, int l1) {
   KernelArgs a;
   a.geo = h->geo;
   a.st = h->st;
   a.unit0 = l0 * h->geo.batch;
   a.n_units = (l1 - l0) * h->geo.batch;
+#ifdef QEVICT_TRACE
+  const uint32_t call = h->trace_calls < (uint32_t)TRACE_CALLS ? h->trace_calls++ : (uint32_t)TRACE_CALLS;
+  a.trace = h->st.trace + call * TRACE_CALL_WORDS;
+#endif
   return a;
 }
 
@@ -256,6 +273,9 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
+#ifdef QEVICT_TRACE
+  p.trace = a.trace;
+#endif
   QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
   QE_CUDA(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
   h->decode_steps++;
@@ -355,7 +375,10 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
     if (e == cudaSuccess) e = cudaMemset(h->st.mig_count, 0, (size_t)g.n_layers * 2 * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.counters, 0, U * 32);
     if (e == cudaSuccess) e = cudaMemset(h->st.mass_e, 0, U * (size_t)g.EMAX * 4);
-    if (e == cudaSuccess) e = cudaMemset(h->st.status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(h->st.status, 0, STATUS_BYTES);
+#ifdef QEVICT_TRACE
+    if (e == cudaSuccess) e = trace_clear(h, TRACE_CALLS + 1);
+#endif
     if (e == cudaSuccess) e = route_prepare(route_smem_bytes(g, next_pow2(g.NW)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
   }
@@ -378,6 +401,44 @@ QEVICT_API qevict_status qevict_set_kernel_timing(qevict_handle h, int32_t enabl
   if (!h) return QEVICT_ERR_INVALID_ARG;
   h->timing = enable != 0;
   return QEVICT_OK;
+}
+
+QEVICT_API qevict_status qevict_kernel_timeline(qevict_handle h, int32_t max_records, int32_t* kernel, double* start_us,
+                                                double* end_us, int32_t* n_records) {
+  if (!h || !kernel || !start_us || !end_us || !n_records || max_records < 0) return QEVICT_ERR_INVALID_ARG;
+  *n_records = 0;
+#ifdef QEVICT_TRACE
+  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_CUDA(h, cudaDeviceSynchronize());
+  const uint32_t calls = h->trace_calls;
+  std::vector<unsigned long long> buf(calls * TRACE_CALL_WORDS);
+  if (calls) QE_CUDA(h, cudaMemcpy(buf.data(), h->st.trace, buf.size() * 8, cudaMemcpyDeviceToHost));
+  struct Rec { int k; unsigned long long t0, t1; };
+  std::vector<Rec> recs;
+  for (uint32_t c = 0; c < calls; ++c)
+    for (int k = 0; k < TRACE_KERNELS; ++k) {
+      const unsigned long long* b = buf.data() + c * TRACE_CALL_WORDS + (size_t)k * TRACE_SMS * 2;
+      Rec r{k, ~0ull, 0ull};
+      for (int sm = 0; sm < TRACE_SMS; ++sm) {
+        if (b[2 * sm] < r.t0) r.t0 = b[2 * sm];
+        if (b[2 * sm + 1] > r.t1) r.t1 = b[2 * sm + 1];
+      }
+      if (r.t0 != ~0ull) recs.push_back(r);
+    }
+  const size_t n = recs.size() < (size_t)max_records ? recs.size() : (size_t)max_records;
+  const size_t first = recs.size() - n;
+  for (size_t i = 0; i < n; ++i) {
+    kernel[i] = recs[first + i].k;
+    start_us[i] = (double)(long long)(recs[first + i].t0 - recs[first].t0) * 1e-3;
+    end_us[i] = (double)(long long)(recs[first + i].t1 - recs[first].t0) * 1e-3;
+  }
+  *n_records = (int32_t)n;
+  QE_CUDA(h, trace_clear(h, calls));
+  h->trace_calls = 0;
+  return QEVICT_OK;
+#else
+  return fail(h, QEVICT_ERR_UNSUPPORTED, "this library was built without -DQEVICT_TRACE");
+#endif
 }
 
 QEVICT_API qevict_status qevict_kernel_times(qevict_handle h, double* total_ms, uint64_t* n_launches) {

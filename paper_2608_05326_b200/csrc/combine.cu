@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   float* s_invl = s_m + g.Hq;                  // [Hq] 1 / denominator
   float* s_w = s_invl + g.Hq;                  // [Hq][S] weight of a split in its head's output
   pdl_prologue();
+  QE_TRACE_SCOPE(a.trace, 2);
   const float2* ml = reinterpret_cast<const float2*>(a.st.ml) + (size_t)u * g.Hq * MAX_SPLITS;
   const float2* wrec = a.st.wrec + (size_t)u * g.Hq * g.EMAX;
   const uint2* entries = a.st.entries + (size_t)u * g.EMAX;

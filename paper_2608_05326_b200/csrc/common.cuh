@@ -79,6 +79,9 @@ struct State {
   float2* wrec;         // [EMAX][Hq] {window exp-sum, reference max (log2 domain)}
   float* mass_e;        // [EMAX] last step's mass per entry
   int32_t* status;      // [1] (shared by all units)
+#ifdef QEVICT_TRACE
+  unsigned long long* trace;  // [TRACE_CALLS + 1] call blocks (shared by all units)
+#endif
 };
 
 template <class T> struct Tr;
@@ -161,6 +164,40 @@ __device__ __forceinline__ void pdl_prologue() {
   asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
+
+// Kernel timeline (tracing build only, -DQEVICT_TRACE).  The workspace then carries, for each of the first
+// TRACE_CALLS API calls since the timeline was last read, one block per step kernel (0 append, 1 attention,
+// 2 combine, 3 route, 4 migrate) of per-SM {earliest warp start, latest warp end} in %globaltimer nanoseconds;
+// each warp issues two fire-and-forget reductions on its own SM's pair, so nothing waits on the stamps.
+// Block TRACE_CALLS is a sink for the calls beyond the capacity.  In the normal build QE_TRACE_SCOPE is empty.
+constexpr int STATUS_BYTES = 256;
+#ifdef QEVICT_TRACE
+constexpr int TRACE_CALLS = 512;
+constexpr int TRACE_KERNELS = 5;
+constexpr int TRACE_SMS = 160;  // >= SMs of the device; %smid is folded into the range
+constexpr size_t TRACE_CALL_WORDS = (size_t)TRACE_KERNELS * TRACE_SMS * 2;
+constexpr size_t TRACE_BYTES = (TRACE_CALLS + 1) * TRACE_CALL_WORDS * 8;
+struct TraceScope {
+  unsigned long long* slot;
+  static __device__ __forceinline__ unsigned long long now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+  }
+  __device__ __forceinline__ TraceScope(unsigned long long* call_block, int k) {
+    uint32_t smid;
+    asm("mov.u32 %0, %%smid;" : "=r"(smid));
+    slot = call_block + ((size_t)k * TRACE_SMS + smid % TRACE_SMS) * 2;
+    if ((threadIdx.x & 31) == 0) atomicMin(slot, now());
+  }
+  __device__ __forceinline__ ~TraceScope() {
+    if ((threadIdx.x & 31) == 0) atomicMax(slot + 1, now());
+  }
+};
+#define QE_TRACE_SCOPE(block, k) TraceScope qe_trace_scope(block, k)
+#else
+#define QE_TRACE_SCOPE(block, k)
+#endif
 
 template <class... KArgs, class... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

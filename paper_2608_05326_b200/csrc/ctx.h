@@ -40,6 +40,9 @@ struct qevict_ctx {
   char* stage_k = nullptr;
   char* stage_v = nullptr;
   char* stage_out = nullptr;
+#ifdef QEVICT_TRACE
+  uint32_t trace_calls = 0;   // API calls traced since the timeline was last read
+#endif
 };
 
 namespace qevict {

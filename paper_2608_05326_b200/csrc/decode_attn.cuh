@@ -47,6 +47,9 @@ struct DecodeParams {
   int e_bound;            // upper bound of every unit's work-list length (host's mirror of the window counts)
   uint32_t fp_page_bytes, q_page_bytes;
   float scale_log2;
+#ifdef QEVICT_TRACE
+  unsigned long long* trace;  // this call's block of the kernel timeline
+#endif
 };
 
 static constexpr int NSLOT = 2;                   // ring slots per warp
@@ -350,6 +353,7 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   const uint32_t ring = smem_u32(smem) + wid * NSLOT * TT::SLOT_BYTES;
   const uint32_t bars = smem_u32(smem) + TT::RING_BYTES + wid * NSLOT * 8;
   pdl_prologue();
+  QE_TRACE_SCOPE(p.trace, 1);
   if (lane == 0) {
 #pragma unroll
     for (int i = 0; i < NSLOT; ++i) mbar_init(bars + i * 8, 1);

@@ -10,6 +10,9 @@ struct KernelArgs {
   State st;
   int unit0;    // first unit of this call
   int n_units;  // units of this call
+#ifdef QEVICT_TRACE
+  unsigned long long* trace;  // this call's block of the kernel timeline
+#endif
 };
 
 // decode step ---------------------------------------------------------------------------------------

@@ -77,6 +77,9 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   KernelArgs a;
   a.geo = g;
   a.st = h->st;
+#ifdef QEVICT_TRACE
+  a.trace = h->st.trace + (size_t)TRACE_CALLS * TRACE_CALL_WORDS;  // not traced: the sink block
+#endif
   a.st.o_part = reinterpret_cast<float*>(scratch);
   a.st.ml = reinterpret_cast<float*>(scratch + o_bytes);
   a.st.wrec = reinterpret_cast<float2*>(scratch + o_bytes + ml_bytes);
@@ -104,6 +107,9 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   p.q = q; p.entries = a.st.entries; p.n_live = a.st.n_live; p.open_fill = a.st.open_fill;
   p.fp_pool = a.st.fp_pool; p.q_pool = a.st.q_pool; p.o_part = a.st.o_part; p.ml = a.st.ml; p.wrec = a.st.wrec;
   p.status = a.st.status;
+#ifdef QEVICT_TRACE
+  p.trace = a.trace;
+#endif
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
   e = h->decode_fn(p, a.n_units, stream);

@@ -288,6 +288,7 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
                                                                   const T* __restrict__ v_prompt, int ctx) {
   const Geometry& g = a.geo;
   pdl_prologue();
+  QE_TRACE_SCOPE(a.trace, 4);
   int32_t* cnt = a.st.mig_count + 2 * (a.unit0 / g.batch);
   const int4* queue = a.st.mig_queue + (size_t)a.unit0 * (g.PF + g.Kq + g.Kf) * 2;
   const int n_entries = *reinterpret_cast<volatile int32_t*>(cnt);

@@ -108,6 +108,7 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
   const int ul = blockIdx.x, u = a.unit0 + ul, tid = threadIdx.x;
   __shared__ int s_page;
   pdl_prologue();
+  QE_TRACE_SCOPE(a.trace, 0);
   // every thread reads the scalars itself (same addresses: one broadcast transaction each)
   const int ow0 = a.st.open_window[u];
   const int fill0 = a.st.open_fill[u];
@@ -328,6 +329,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   uint8_t* cled = ctier + sort_cap;                                          // [sort_cap] ledger flag
   uint8_t* cnew = cled + sort_cap;                                           // [sort_cap] state after
   pdl_prologue();
+  QE_TRACE_SCOPE(a.trace, 3);
 
   uint8_t* tier = a.st.tier + (size_t)u * g.NW;
   uint8_t* ledger = a.st.ledger + (size_t)u * g.NW;
