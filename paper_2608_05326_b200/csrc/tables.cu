@@ -164,20 +164,35 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
     __syncthreads();
   }
   const int tile = slot >> 5, tk = slot & 31;
+  // The token goes through shared memory so that the scatter into the fragment-major page is two short loops
+  // (keys as channel pairs, values element by element) rather than a long unrolled sequence: this code runs
+  // once per launch with cold instruction caches, so its size is its cost.
+  __shared__ __align__(16) T s_k[128 * MAXV * 8];
+  __shared__ __align__(16) T s_v[128 * MAXV * 8];
 #pragma unroll
   for (int i = 0; i < MAXV; ++i) {
     const int v = tid + i * 128;
     if (v < nvec) {
-      const int h = (v * 8) / g.D, ch0 = v * 8 - h * g.D;
-      T* kt = reinterpret_cast<T*>(pbase + (size_t)h * g.fp_head_bytes + (size_t)tile * 2 * g.fp_tile_bytes);
-      T* vt = reinterpret_cast<T*>(reinterpret_cast<char*>(kt) + g.fp_tile_bytes);
-      const T* ke = reinterpret_cast<const T*>(&kx[i]);
-      const T* ve = reinterpret_cast<const T*>(&vx[i]);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        kt[fpk_off(tk, ch0 + e, g.D)] = ke[e];
-        vt[fpv_off(tk, ch0 + e)] = ve[e];
-      }
+      reinterpret_cast<uint4*>(s_k)[v] = kx[i];
+      reinterpret_cast<uint4*>(s_v)[v] = vx[i];
+    }
+  }
+  __syncthreads();
+  {
+    const int n_stage = (nvec < MAXV * 128 ? nvec : MAXV * 128) * 8;  // elements held in shared memory
+    const int dsh = 31 - __clz(g.D);                                  // the head dimension is a power of two
+    char* tbase = pbase + (size_t)tile * 2 * g.fp_tile_bytes;
+#pragma unroll 1
+    for (int el = 2 * tid; el < n_stage; el += 256) {
+      const int h = el >> dsh, ch = el & (g.D - 1);
+      T* kt = reinterpret_cast<T*>(tbase + (size_t)h * g.fp_head_bytes);
+      *reinterpret_cast<uint32_t*>(kt + fpk_off(tk, ch, g.D)) = *reinterpret_cast<const uint32_t*>(s_k + el);
+    }
+#pragma unroll 1
+    for (int el = tid; el < n_stage; el += 128) {
+      const int h = el >> dsh, ch = el & (g.D - 1);
+      T* vt = reinterpret_cast<T*>(tbase + (size_t)h * g.fp_head_bytes + g.fp_tile_bytes);
+      vt[fpv_off(tk, ch)] = s_v[el];
     }
   }
   for (int v = tid + MAXV * 128; v < nvec; v += 128) {  // wider rows than the register buffer holds
