@@ -212,7 +212,7 @@ def qevict_kernel_timeline(h, max_records=2560):
     t1 = (C.c_double * max_records)()
     n = C.c_int32(0)
     _check(lib().qevict_kernel_timeline(h, max_records, kid, t0, t1, C.byref(n)), h)
-    return [(KERNEL_NAMES[kid[i]] if 0 <= kid[i] < len(KERNEL_NAMES) else "?", t0[i], t1[i]) for i in range(n.value)]
+    return [(KERNEL_NAMES[kid[i]] if 0 <= kid[i] < len(KERNEL_NAMES) else "k%d" % kid[i], t0[i], t1[i]) for i in range(n.value)]
 
 
 def qevict_get_stats(h, layer=-1):
