@@ -193,6 +193,7 @@ KernelArgs make_args(qevict_handle h, int l0, int l1) {
   a.st = h->st;
   a.unit0 = l0 * h->geo.batch;
   a.n_units = (l1 - l0) * h->geo.batch;
+  a.mig_parity = (int)(h->mig_epoch[l0] & 1u);
 #ifdef QEVICT_TRACE
   const uint32_t call = h->trace_calls < (uint32_t)TRACE_CALLS ? h->trace_calls++ : (uint32_t)TRACE_CALLS;
   a.trace = h->st.trace + call * TRACE_CALL_WORDS;
@@ -352,6 +353,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
   }
   if (!h->decode_fn) { delete h; return QEVICT_ERR_UNSUPPORTED; }
   h->layers.resize(g.n_layers);
+  h->mig_epoch.assign(g.n_layers, 0u);
   cudaError_t e = cudaSetDevice(cfg->device);
   if (e == cudaSuccess) {
     int sms = 0;
@@ -497,6 +499,7 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
   QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kfp, s));
   QE_CUDA(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));
+  ++h->mig_epoch[l0];  // the next event of these units counts its queue in the other counter
   h->launches += 2 + (g.Kfp > 0) + (g.Kq > 0);
   for (int l = l0; l < l1; ++l) {
     h->layers[l].prefilled = true;
@@ -561,7 +564,10 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   // quantizations and promotions of the event in one launch (linked where they share a page)
   const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
   const int max_items = (g.Kq > 0 ? g.PF : 0) + max_promote;
-  if (max_items > 0) QE_CUDA(h, timed_launch(h, 4, s, [&] { return launch_migrate(a, nullptr, nullptr, 0, max_items, s); }));
+  if (max_items > 0) {
+    QE_CUDA(h, timed_launch(h, 4, s, [&] { return launch_migrate(a, nullptr, nullptr, 0, max_items, s); }));
+    ++h->mig_epoch[l0];  // the next event of these units counts its queue in the other counter
+  }
   for (int l = l0; l < l1; ++l) h->layers[l].aged = 0;
   return QEVICT_OK;
 }

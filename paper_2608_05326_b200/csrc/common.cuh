@@ -70,7 +70,8 @@ struct State {
   int32_t* n_copy;
   int4* mig_queue;      // [PF + Kq + Kf] records of two int4 per unit; the units of one call share the run
                         // that starts at its first unit (record format: see the migration kernel)
-  int32_t* mig_count;   // [n_layers][2] (not per unit) {entries queued by the routing event, CTAs finished}
+  int32_t* mig_count;   // [n_layers][2] (not per unit) entries queued by the routing event; events alternate
+                        // between the two counters, and the migration kernel clears the one the next event uses
   unsigned long long* counters;  // [4] promotions, quantizations, reactivations, deletions
   char* fp_pool;        // [PF] pages
   char* q_pool;         // [PQ] pages

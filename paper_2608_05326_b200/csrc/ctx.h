@@ -26,6 +26,7 @@ struct qevict_ctx {
   qevict::Geometry geo;
   qevict::State st;
   std::vector<qevict::LayerMirror> layers;
+  std::vector<uint32_t> mig_epoch;    // per layer: routing events launched with this layer first in the call
   std::string last_error;
   uint64_t launches = 0;
   uint64_t decode_steps = 0;

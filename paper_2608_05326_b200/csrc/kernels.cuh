@@ -10,6 +10,7 @@ struct KernelArgs {
   State st;
   int unit0;    // first unit of this call
   int n_units;  // units of this call
+  int mig_parity;  // which of the call's two migration-queue counters this routing event uses
 #ifdef QEVICT_TRACE
   unsigned long long* trace;  // this call's block of the kernel timeline
 #endif

@@ -77,6 +77,7 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   KernelArgs a;
   a.geo = g;
   a.st = h->st;
+  a.mig_parity = 0;  // no routing event on this path
 #ifdef QEVICT_TRACE
   a.trace = h->st.trace + (size_t)TRACE_CALLS * TRACE_CALL_WORDS;  // not traced: the sink block
 #endif

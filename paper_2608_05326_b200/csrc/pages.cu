@@ -282,7 +282,7 @@ __device__ __forceinline__ void promote_value_task(const Geometry& g, int tile, 
 //   kind 2  nothing (a promotion that is linked to a demotion)
 // Every warp of a fixed-size grid takes (record, KV head, keys | values, task) tuples round-robin, so the
 // launch costs the same whether one unit or all of them migrate something, and the tasks are independent
-// (see above), so nothing waits on another warp.  The last CTA to finish empties the queue.
+// (see above), so nothing waits on another warp.
 template <class T>
 __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const KernelArgs a, const T* __restrict__ k_prompt,
                                                                   const T* __restrict__ v_prompt, int ctx) {
@@ -291,7 +291,9 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
   QE_TRACE_SCOPE(a.trace, 4);
   int32_t* cnt = a.st.mig_count + 2 * (a.unit0 / g.batch);
   const int4* queue = a.st.mig_queue + (size_t)a.unit0 * (g.PF + g.Kq + g.Kf) * 2;
-  const int n_entries = *reinterpret_cast<volatile int32_t*>(cnt);
+  const int n_entries = *reinterpret_cast<volatile int32_t*>(cnt + a.mig_parity);
+  // the next routing event of these units counts in the other counter: nothing reads it before this kernel ends
+  if (blockIdx.x == 0 && threadIdx.x == 0) cnt[a.mig_parity ^ 1] = 0;
   const int lane = threadIdx.x & 31;
   const int gw = blockIdx.x * (MIGRATE_THREADS / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (MIGRATE_THREADS / 32);
   const int ks_n = g.D >> 4, ng = g.D / g.group;
@@ -330,11 +332,6 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
       if (part == 0) promote_key_task<T>(g, c0, c1, pq, pf, lane);
       else promote_value_task<T>(g, c0, c1, c2, pq, pf, lane);
     }
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    if (atomicAdd(cnt + 1, 1) == (int)gridDim.x - 1) { cnt[0] = 0; cnt[1] = 0; }
   }
 }
 

@@ -650,7 +650,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     if (n_fp_need > nfp) record_check(a.st.status, CHECK_FP_POOL_EXHAUSTED);
     // this unit's migrations join the call's queue (the order of the units in it does not matter: the
     // items are independent of one another); the reply is needed only at the very end
-    if (n_items > 0) qbase = atomicAdd(a.st.mig_count + 2 * (a.unit0 / g.batch), n_items);
+    if (n_items > 0) qbase = atomicAdd(a.st.mig_count + 2 * (a.unit0 / g.batch) + a.mig_parity, n_items);
   }
   __syncthreads();
 
