@@ -29,16 +29,18 @@ __device__ __forceinline__ void group_params(float mn, float mx, int qmax, T& s_
 }
 
 // code = clamp(rint((x - zero) / scale)) on the IEEE float32 quotient.  The quotient is first estimated with
-// the group's reciprocal (error of a few 1e-6 at most for codes up to 15); only when the estimate lies
-// within 1e-3 of a rounding boundary (or is not finite) is the exact division carried out, so the result
-// is the exact-division result in every case.
-__device__ __forceinline__ uint32_t quant_code(float x, float z, float s, float inv_s, int qmax, bool bad) {
-  if (bad) return 0u;
-  const float d = __fsub_rn(x, z);
-  float r = rintf(__fmul_rn(d, inv_s));
-  if (!(fabsf(fabsf(__fmul_rn(d, inv_s) - r) - 0.5f) >= 1e-3f)) r = rintf(__fdiv_rn(d, s));
-  const int c = (int)fminf(fmaxf(r, 0.f), (float)qmax);
-  return (uint32_t)c;
+// the group's reciprocal (error of a few 1e-6 at most for codes up to 15); only when an estimate of the
+// vector lies within 1e-3 of a rounding boundary (or is not finite) is the exact division carried out, so
+// the result is the exact-division result in every case.  x >= zero (the group minimum), so the estimate
+// needs no lower clamp.  This is run-once code whose length is its cost: one test per vector, not per code.
+__device__ __forceinline__ float code_estimate(float x, float z, float inv_s, bool& near) {
+  const float q = __fmul_rn(__fsub_rn(x, z), inv_s);
+  const float r = rintf(q);
+  near = near || !(fabsf(fabsf(q - r) - 0.5f) >= 1e-3f);
+  return r;
+}
+__device__ __forceinline__ float code_exact(float x, float z, float s) {
+  return fmaxf(rintf(__fdiv_rn(__fsub_rn(x, z), s)), 0.f);
 }
 
 // ---- migration tasks ---------------------------------------------------------------------------------
@@ -82,30 +84,45 @@ __device__ __forceinline__ void fold_minmax(const uint4& v, float (&mn)[4], floa
   }
 }
 
-// codes of one vector: returns sum over (a, e) of code << (bits * a + 16 * e)
+// codes of one vector: returns sum over (a, e) of code << (bits * a + 16 * e); `keep` clears the codes of the
+// slots whose group has no usable scale
 template <class T>
 __device__ __forceinline__ uint32_t vector_codes(const uint4& v, const float (&mn)[4], const float (&sc)[4],
-                                                 const float (&inv)[4], const bool (&bad)[4], int qmax, int bits) {
+                                                 const float (&inv)[4], uint32_t keep, int qmax, int bits) {
   const uint32_t r[4] = {v.x, v.y, v.z, v.w};
-  uint32_t w = 0u;
+  float c[4][2];
+  bool near = false;
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
     float f[2];
     unpack2<T>(r[a], f[0], f[1]);
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int k = (a >> 1) * 2 + e;
-      w |= quant_code(f[e], mn[k], sc[k], inv[k], qmax, bad[k]) << (bits * a + 16 * e);
+    for (int e = 0; e < 2; ++e) c[a][e] = code_estimate(f[e], mn[(a >> 1) * 2 + e], inv[(a >> 1) * 2 + e], near);
+  }
+  if (__builtin_expect(near, 0)) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      float f[2];
+      unpack2<T>(r[a], f[0], f[1]);
+#pragma unroll
+      for (int e = 0; e < 2; ++e) c[a][e] = code_exact(f[e], mn[(a >> 1) * 2 + e], sc[(a >> 1) * 2 + e]);
     }
   }
-  return w;
+  uint32_t w = 0u;
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) w |= (uint32_t)(int)fminf(c[a][e], (float)qmax) << (bits * a + 16 * e);
+  return w & keep;
 }
 
 // Minimum / maximum of the four slots over the 8 lanes of equal lane % 4, then the group parameters of
-// each slot; lanes 0..3 store the 16-byte parameter record (layout (hi * 2 + is_zero) * 2 + e).
+// each slot: the lane with (lane >> 2) & 3 == k works out slot k (one division per lane instead of four) and
+// the others fetch it by shuffle.  Lanes 0..3 store the 16-byte parameter record (layout
+// (hi * 2 + is_zero) * 2 + e).  `keep` gets the code bits of the slots whose scale is usable.
 template <class T>
-__device__ __forceinline__ void slot_params(float (&mn)[4], float (&mx)[4], int qmax, float (&sc)[4], float (&inv)[4],
-                                            bool (&bad)[4], uint4* param_dst, int lane) {
+__device__ __forceinline__ void slot_params(float (&mn)[4], float (&mx)[4], int qmax, int bits, float (&sc)[4],
+                                            float (&inv)[4], uint32_t& keep, uint4* param_dst, int lane) {
 #pragma unroll
   for (int o = 4; o <= 16; o <<= 1) {
 #pragma unroll
@@ -114,11 +131,25 @@ __device__ __forceinline__ void slot_params(float (&mn)[4], float (&mx)[4], int 
       mx[k] = fmaxf(mx[k], __shfl_xor_sync(0xffffffffu, mx[k], o));
     }
   }
+  const int km = (lane >> 2) & 3;
+  const float mn_m = km & 2 ? (km & 1 ? mn[3] : mn[2]) : (km & 1 ? mn[1] : mn[0]);
+  const float mx_m = km & 2 ? (km & 1 ? mx[3] : mx[2]) : (km & 1 ? mx[1] : mx[0]);
+  T st_m, zt_m;
+  float s_m;
+  bool bad_m;
+  group_params<T>(mn_m, mx_m, qmax, st_m, zt_m, s_m, bad_m);
+  const float inv_m = bad_m ? 0.f : __frcp_rn(s_m);  // zero marks an unusable scale (its estimates are 0 or NaN)
   T st[4], zt[4];
+  keep = 0u;
+  const uint32_t pair = (uint32_t)qmax | ((uint32_t)qmax << bits);  // the two registers of one `hi`
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    group_params<T>(mn[k], mx[k], qmax, st[k], zt[k], sc[k], bad[k]);
-    inv[k] = __frcp_rn(sc[k]);
+    const int src = (lane & 3) + 4 * k;
+    sc[k] = __shfl_sync(0xffffffffu, s_m, src);
+    inv[k] = __shfl_sync(0xffffffffu, inv_m, src);
+    st[k] = Tr<T>::from_float(sc[k]);  // exact: the scale is a value of T
+    zt[k] = Tr<T>::from_float(mn[k]);  // exact: the minimum is a value of T
+    if (inv[k] != 0.f) keep |= pair << (2 * bits * (k >> 1) + 16 * (k & 1));
   }
   if (lane < 4) *param_dst = make_uint4(pack2<T>(st[0], st[1]), pack2<T>(zt[0], zt[1]), pack2<T>(st[2], st[3]), pack2<T>(zt[2], zt[3]));
 }
@@ -167,14 +198,15 @@ __device__ __forceinline__ void quant_key_task(const Geometry& g, int blk, int k
     fold_minmax<T>(x[tl][0], mn, mx);
     fold_minmax<T>(x[tl][1], mn, mx);
   }
-  float sc[4], inv[4]; bool bad[4];
-  slot_params<T>(mn, mx, qmax, sc, inv, bad, reinterpret_cast<uint4*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes) + ks * 4 + t, lane);
+  float sc[4], inv[4];
+  uint32_t keep;
+  slot_params<T>(mn, mx, qmax, bits, sc, inv, keep, reinterpret_cast<uint4*>(qb + g.q_kp_off + (size_t)blk * g.q_kp_bytes) + ks * 4 + t, lane);
 #pragma unroll
   for (int tl = 0; tl < 2; ++tl) {
     if (tl >= tpg) continue;
     uint32_t* dstw = reinterpret_cast<uint32_t*>(qb + (size_t)(blk * tpg + tl) * g.q_tile_stride);
-    const uint32_t w0 = vector_codes<T>(x[tl][0], mn, sc, inv, bad, qmax, bits);
-    const uint32_t w1 = vector_codes<T>(x[tl][1], mn, sc, inv, bad, qmax, bits);
+    const uint32_t w0 = vector_codes<T>(x[tl][0], mn, sc, inv, keep, qmax, bits);
+    const uint32_t w1 = vector_codes<T>(x[tl][1], mn, sc, inv, keep, qmax, bits);
     if (bits == 4) {
       dstw[code_word_off(ks * 2 + 0, lane)] = w0;
       dstw[code_word_off(ks * 2 + 1, lane)] = w1;
@@ -235,15 +267,16 @@ __device__ __forceinline__ void quant_value_task(const Geometry& g, int tile, in
     if (ii >= ipg) continue;
     fold_minmax<T>(x[ii], mn, mx);
   }
-  float sc[4], inv[4]; bool bad[4];
+  float sc[4], inv[4];
+  uint32_t keep;
   char* tb = qb + (size_t)tile * g.q_tile_stride;
-  slot_params<T>(mn, mx, qmax, sc, inv, bad, reinterpret_cast<uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes) + (gc * 2 + ks) * 4 + t, lane);
+  slot_params<T>(mn, mx, qmax, bits, sc, inv, keep, reinterpret_cast<uint4*>(tb + g.q_kc_bytes + g.q_vc_bytes) + (gc * 2 + ks) * 4 + t, lane);
   uint32_t* dstw = reinterpret_cast<uint32_t*>(tb + g.q_kc_bytes);
 #pragma unroll
   for (int ii = 0; ii < 4; ++ii) {
     if (ii >= ipg) continue;
     const int i = gc * ipg + ii;
-    const uint32_t w = vector_codes<T>(x[ii], mn, sc, inv, bad, qmax, bits);
+    const uint32_t w = vector_codes<T>(x[ii], mn, sc, inv, keep, qmax, bits);
     if (bits == 4) {
       dstw[code_word_off(i * 2 + ks, lane)] = w;
     } else {
