@@ -355,13 +355,25 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   int32_t* q_owner = a.st.q_owner + (size_t)u * g.PQ;
   const int nw = a.st.n_windows[u];
   const int ow = a.st.open_window[u];
-  const int ow_page = ow >= 0 ? fp_page[ow] : -1;  // the open window is no candidate: its page does not change here
-
+  // The page owner tables: requested here, parked in shared memory only once the gather's loads are in flight
+  // too (a store that waits for its load would hold up every request behind it).  The open window is no
+  // candidate and keeps its page; the page is the one it owns.
+  const int o_f0 = tid < g.PF ? fp_owner[tid] : -1;
+  const int o_q0 = tid < g.PQ ? q_owner[tid] : -1;
   int* s_react = scratch + 100;
   int* s_del = scratch + 101;
+  int* s_ow_page = scratch + 102;  // written by the one thread that sees the open window's page (read only if ow >= 0)
   if (tid == 0) { *s_react = 0; *s_del = 0; }
-  for (int i = tid; i < g.PF; i += NT) ofp[i] = fp_owner[i];
-  for (int i = tid; i < g.PQ; i += NT) oq[i] = q_owner[i];
+  auto park_owners = [&] {
+    if (tid < g.PF) { ofp[tid] = o_f0; if (ow >= 0 && o_f0 == ow) *s_ow_page = tid; }
+    if (tid < g.PQ) oq[tid] = o_q0;
+    for (int i = tid + NT; i < g.PF; i += NT) {
+      const int o = fp_owner[i];
+      ofp[i] = o;
+      if (ow >= 0 && o == ow) *s_ow_page = i;
+    }
+    for (int i = tid + NT; i < g.PQ; i += NT) oq[i] = q_owner[i];
+  };
 
   // ---- ranking functions other than Eq. 1: fold the event accumulator into the score of every stored
   // window (each operation rounded on its own, so that the ranking is taken on reproducible numbers) ----
@@ -422,6 +434,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
       qc[k] = ok ? q_page[b + k] : -1;
       ic[k] = ok ? imp[b + k] : 0.f;
     }
+    park_owners();
     int cnt = 0;  // gathered | candidates << 16
 #pragma unroll
     for (int k = 0; k < PRE; ++k) {
@@ -454,6 +467,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     const int b = tid * chunk;
 #pragma unroll
     for (int k = 0; k < 16; ++k) tc[k] = (k < chunk && b + k < nw) ? tier[b + k] : (uint8_t)QEVICT_TIER_NONE;
+    park_owners();
     int cnt = 0;  // gathered | candidates << 16
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
@@ -471,6 +485,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   } else {
     int* s_real = scratch + 103;
     if (tid == 0) *s_real = 0;
+    park_owners();
     __syncthreads();
     n_all = block_compact(nw, scratch,
                           [&](int w) { const uint8_t t = tier[w]; return is_candidate(t, w, recent_lo) || is_pinned(t, w, recent_lo); },
@@ -748,17 +763,18 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   if (tid == 0) {
     int n = n_f + n_q;
     if (ow >= 0) {
-      if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)ow_page);
+      if (n < g.EMAX) entries[n] = make_uint2((uint32_t)ow | (KIND_OPEN << ENTRY_KIND_SHIFT), (uint32_t)*s_ow_page);
       n += 1;
     }
     if (n > g.EMAX) { record_check(a.st.status, CHECK_ENTRY_OVERFLOW); n = g.EMAX; }
     a.st.n_live[u] = n;
     a.st.n_copy[u] = prefill ? nfp : 0;
+    // reductions, not read-modify-write: nothing at the kernel's end waits for a load
     unsigned long long* c = a.st.counters + (size_t)u * 4;
-    c[0] += prefill ? 0ull : (unsigned long long)nfp;
-    c[1] += (unsigned long long)nq;
-    c[2] += (unsigned long long)*s_react;
-    c[3] += (unsigned long long)*s_del;
+    if (!prefill && nfp) atomicAdd(c + 0, (unsigned long long)nfp);
+    if (nq) atomicAdd(c + 1, (unsigned long long)nq);
+    if (*s_react) atomicAdd(c + 2, (unsigned long long)*s_react);
+    if (*s_del) atomicAdd(c + 3, (unsigned long long)*s_del);
   }
 }
 
