@@ -1,5 +1,7 @@
 // Window tables: append to the recent region, prefill initialisation, and the routing event
 // (rank -> tiers -> page release / allocation -> migration lists -> decode work list).
+#include <type_traits>
+
 #include "kernels.cuh"
 #include "layout.cuh"
 
@@ -415,12 +417,14 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   };
   int n_all, n_real;
   const int chunk = (nw + NT - 1) / NT;
-  constexpr int PRE = 10;
+  constexpr int PRE_MAX = 10;
   const int cs = (g.NW + NT - 1) / NT;  // rows of the table per thread (not of the windows in use)
-  if (cs <= PRE && (g.rank_mode == QEVICT_RANK_CUMULATIVE || g.rank_mode == QEVICT_RANK_KEYNORM || prefill)) {
-    // Small tables: every thread requests all five columns of its rows at once, before it knows how many
-    // windows exist or which of them are candidates (rows past the last window hold state NONE), so the
-    // whole gather costs one global round trip.
+  // Small tables: every thread requests all five columns of its rows at once, before it knows how many
+  // windows exist or which of them are candidates (rows past the last window hold state NONE), so the
+  // whole gather costs one global round trip.  Unrolled for 5 or 10 rows per thread: this is run-once code,
+  // and the shorter variant is half the instructions to fetch.
+  auto gather_small = [&](auto pre_tag) {
+    constexpr int PRE = decltype(pre_tag)::value;
     const int b = tid * cs;
     uint8_t tc[PRE], lc[PRE];
     int32_t fc[PRE], qc[PRE];
@@ -444,23 +448,29 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     int tot;
     int rank = block_exclusive_scan(cnt, scratch, &tot) & 0xFFFF;
     n_all = tot & 0xFFFF; n_real = tot >> 16;
+    if (cnt) {
 #pragma unroll
-    for (int k = 0; k < PRE; ++k) {
-      const int w = b + k;
-      const bool pin = is_pinned(tc[k], w, recent_lo);
-      if ((is_candidate(tc[k], w, recent_lo) || pin) && rank < sort_cap) {
-        cw[rank] = w;
-        ctier[rank] = tc[k];
-        cled[rank] = lc[k];
-        cfp[rank] = fc[k];
-        cq[rank] = qc[k];
-        if (pin) cnew[rank] = PINNED | tc[k];
-        keys[rank] = pin ? (0xFFFFFFFF00000000ull | (uint32_t)rank)
-                         : (((unsigned long long)(~mono_bits(ic[k])) << 32) | (uint32_t)rank);
-        ++rank;
+      for (int k = 0; k < PRE; ++k) {
+        const int w = b + k;
+        const bool pin = is_pinned(tc[k], w, recent_lo);
+        if ((is_candidate(tc[k], w, recent_lo) || pin) && rank < sort_cap) {
+          cw[rank] = w;
+          ctier[rank] = tc[k];
+          cled[rank] = lc[k];
+          cfp[rank] = fc[k];
+          cq[rank] = qc[k];
+          if (pin) cnew[rank] = PINNED | tc[k];
+          keys[rank] = pin ? (0xFFFFFFFF00000000ull | (uint32_t)rank)
+                           : (((unsigned long long)(~mono_bits(ic[k])) << 32) | (uint32_t)rank);
+          ++rank;
+        }
       }
     }
     __syncthreads();
+  };
+  if (cs <= PRE_MAX && (g.rank_mode == QEVICT_RANK_CUMULATIVE || g.rank_mode == QEVICT_RANK_KEYNORM || prefill)) {
+    if (cs <= 5) gather_small(std::integral_constant<int, 5>{});
+    else gather_small(std::integral_constant<int, PRE_MAX>{});
   } else if (chunk <= 16) {
     // every thread reads its (up to 16) window states in one go and keeps them in registers
     uint8_t tc[16];
