@@ -369,11 +369,13 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   auto park_owners = [&] {
     if (tid < g.PF) { ofp[tid] = o_f0; if (ow >= 0 && o_f0 == ow) *s_ow_page = tid; }
     if (tid < g.PQ) oq[tid] = o_q0;
+#pragma unroll 1
     for (int i = tid + NT; i < g.PF; i += NT) {
       const int o = fp_owner[i];
       ofp[i] = o;
       if (ow >= 0 && o == ow) *s_ow_page = i;
     }
+#pragma unroll 1
     for (int i = tid + NT; i < g.PQ; i += NT) oq[i] = q_owner[i];
   };
 
@@ -383,6 +385,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     float* score = a.st.importance + (size_t)u * g.NW;
     float* ev = a.st.event_mass + (size_t)u * g.NW;
     const int p = (int)g.rank_param;
+#pragma unroll 1
     for (int w = tid; w < nw; w += NT) {
       const uint8_t t = tier[w];
       if (t == QEVICT_TIER_NONE || t == QEVICT_TIER_EVICTED) continue;
@@ -392,6 +395,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
         s1 = __fadd_rn(__fmul_rn(g.rank_param, s0), uw);
       } else {
         float v = uw;
+#pragma unroll 1
         for (int i = 1; i < p; ++i) v = __fmul_rn(v, uw);
         s1 = __fadd_rn(s0, v);
       }
@@ -514,22 +518,26 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     // One-way policy (no promotion): the Full tier is drawn from the candidates that are not Quantized, the
     // Quantized tier from everything else.  Two counting ranks (this is a diagnostic policy: no selection path).
     constexpr uint8_t UNDECIDED = 0x7F;
+#pragma unroll 1
     for (int c = tid; c < n_cand; c += NT) {
       const unsigned long long mine = keys[c];
       if ((uint32_t)(mine >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
       uint8_t nt = UNDECIDED;
       if (ctier[c] != QEVICT_TIER_QUANT) {
         int pos = 0;
+#pragma unroll 1
         for (int i = 0; i < n_cand; ++i) pos += (ctier[i] != QEVICT_TIER_QUANT && keys[i] < mine) ? 1 : 0;
         if (pos < g.Kf) nt = QEVICT_TIER_FULL;
       }
       cnew[c] = nt;
     }
     __syncthreads();
+#pragma unroll 1
     for (int c = tid; c < n_cand; c += NT) {
       if (cnew[c] != UNDECIDED) continue;
       const unsigned long long mine = keys[c];
       int pos = 0;  // smaller keys among the candidates outside the new Full tier (pinned windows hold the largest keys)
+#pragma unroll 1
       for (int i = 0; i < n_cand; ++i) pos += (cnew[i] != QEVICT_TIER_FULL && !(cnew[i] & PINNED) && keys[i] < mine) ? 1 : 0;
       // written only after the count: other threads test this entry for "not Full", which holds before and after
       cnew[c] = pos < g.Kq ? QEVICT_TIER_QUANT : QEVICT_TIER_EVICTED;
@@ -538,6 +546,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     // rank of a key = number of smaller keys (all keys are distinct); two adjacent lanes share a key and
     // count over one half of the keys each
     const int half = tid & 1, i0 = half ? n_cand / 2 : 0, i1 = half ? n_cand : n_cand / 2;
+#pragma unroll 1
     for (int cb = 0; cb < n_cand; cb += NT / 2) {  // same trip count for the whole block
       const int c = cb + (tid >> 1);
       const unsigned long long mine = c < n_cand ? keys[c] : ~0ull;
@@ -563,9 +572,11 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
 #pragma unroll 1
     for (int pass = 0; pass < 6; ++pass) {
       const int shift = pass < 4 ? 56 - 8 * pass : (pass == 4 ? 8 : 0);
+#pragma unroll 1
       for (int i = tid; i < 512; i += NT) hist[i] = 0;
       __syncthreads();
       const unsigned long long p0 = ((unsigned long long)sel[1] << 32) | sel[0], p1 = ((unsigned long long)sel[3] << 32) | sel[2];
+#pragma unroll 1
       for (int c = tid; c < n_cand; c += NT) {
         const unsigned long long key = keys[c];
         const int d = (int)((key >> shift) & 255ull);
@@ -604,6 +615,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
       __syncthreads();
     }
     const unsigned long long t0 = ((unsigned long long)sel[1] << 32) | sel[0], t1 = ((unsigned long long)sel[3] << 32) | sel[2];
+#pragma unroll 1
     for (int c = tid; c < n_cand; c += NT) {
       const unsigned long long key = keys[c];
       if ((uint32_t)(key >> 32) == 0xFFFFFFFFu) continue;  // pinned: state already set
@@ -613,6 +625,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   __syncthreads();
 
   // ---- releases (owner tables only; the candidates' page ids stay readable until the lists are built) --
+#pragma unroll 1
   for (int c = tid; c < n_cand; c += NT) {
     const uint8_t old = ctier[c], nt = cnew[c];
     if ((nt == QEVICT_TIER_QUANT && old != QEVICT_TIER_QUANT) || nt == QEVICT_TIER_EVICTED) {
@@ -624,6 +637,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
       atomicAdd(s_react, 1);
     }
   }
+#pragma unroll 1
   for (int i = tid; i < g.PF; i += NT) reader[i] = -1;
   __syncthreads();
 
@@ -642,8 +656,11 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   const int bf = min(g.PF, tid * ch_f), ef = min(g.PF, bf + ch_f), bq = min(g.PQ, tid * ch_q), eq = min(g.PQ, bq + ch_q);
   const int bc = min(n_cand, tid * ch_c), ec = min(n_cand, bc + ch_c);
   int3 cnt = make_int3(0, 0, 0);  // {free fp | free q << 16, need q | need fp << 16, Full | Quantized << 16}
+#pragma unroll 1
   for (int pg = bf; pg < ef; ++pg) cnt.x += ofp[pg] < 0 ? 1 : 0;
+#pragma unroll 1
   for (int pg = bq; pg < eq; ++pg) cnt.x += oq[pg] < 0 ? 0x10000 : 0;
+#pragma unroll 1
   for (int c = bc; c < ec; ++c) {
     cnt.y += (q_needs(c) ? 1 : 0) + (fp_needs(c) ? 0x10000 : 0);
     cnt.z += (lists_as_full(c) ? 1 : 0) + (cnew[c] == QEVICT_TIER_QUANT ? 0x10000 : 0);
@@ -655,10 +672,13 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   int32_t* qlist = flist + n_f;
   {
     int r = rk.x & 0xFFFF;
+#pragma unroll 1
     for (int pg = bf; pg < ef; ++pg) if (ofp[pg] < 0) free_fp[r++] = pg;
     r = rk.x >> 16;
+#pragma unroll 1
     for (int pg = bq; pg < eq; ++pg) if (oq[pg] < 0) free_q[r++] = pg;
     int r0 = rk.y & 0xFFFF, r1 = rk.y >> 16, r2 = rk.z & 0xFFFF, r3 = rk.z >> 16;
+#pragma unroll 1
     for (int c = bc; c < ec; ++c) {
       if (q_needs(c)) need_q[r0++] = c;
       if (fp_needs(c)) need_fp[r1++] = c;
@@ -681,6 +701,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
 
   // first demotions take the free quantized pages in ascending order.  reader[p] = index of the
   // quantization that reads full-precision page p
+#pragma unroll 1
   for (int k = tid; k < nq; k += NT) {
     const int c = need_q[k], pg = free_q[k];
     oq[pg] = cw[c];
@@ -694,6 +715,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   // that receives a page some quantization of this event still has to read is linked to that quantization
   // (the migration kernel runs it right after it, in the same warps).
   int4* copy_list = a.st.copy_list + (size_t)u * g.Kfp;
+#pragma unroll 1
   for (int k = tid; k < nfp; k += NT) {
     const int c = need_fp[k], pg = free_fp[k];
     ofp[pg] = cw[c];
@@ -709,6 +731,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   __syncthreads();
 
   // ---- commit: the candidates' rows and the owner tables go back to global memory --------------------
+#pragma unroll 1
   for (int c = tid; c < n_cand; c += NT) {
     const uint8_t old = ctier[c], nt = cnew[c];
     const int w = cw[c];
@@ -731,13 +754,16 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     fp_page[w] = cfp[c];
     q_page[w] = cq[c];
   }
+#pragma unroll 1
   for (int i = tid; i < g.PF; i += NT) fp_owner[i] = ofp[i];
+#pragma unroll 1
   for (int i = tid; i < g.PQ; i += NT) q_owner[i] = oq[i];
   // the migration records (32 bytes each; format: see the migration kernel), written by the first warp: the
   // reply of the queue reservation reaches the other lanes by shuffle
   if (tid < 32) {
     const int base = __shfl_sync(0xffffffffu, qbase, 0);
     int4* queue = a.st.mig_queue + ((size_t)a.unit0 * (g.PF + g.Kq + g.Kf) + base) * 2;
+#pragma unroll 1
     for (int i = tid; i < n_items; i += 32) {
       if (i < nq) {
         const int4 it = qrec[i];
@@ -758,6 +784,7 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
   uint2* entries = a.st.entries + (size_t)u * g.EMAX;
   {
     const int n = n_f + n_q;
+#pragma unroll 1
     for (int k = tid; k < n && k < g.EMAX; k += NT) {
       const int cf = (int)(((long long)k * n_f) / n);                       // Full windows before position k
       const bool is_f = (int)(((long long)(k + 1) * n_f) / n) > cf;
