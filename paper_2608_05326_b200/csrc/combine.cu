@@ -65,9 +65,11 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   }
 
   // ---- per-head maximum, denominator and split weights (one thread per head) ------------------------------
+#pragma unroll 1
   for (int h = tid; h < g.Hq; h += COMBINE_THREADS) {
     const float2* p = ml + (size_t)h * MAX_SPLITS;
     float mx = -INFINITY, l = 0.f;
+#pragma unroll 1
     for (int s0 = 0; s0 < S; s0 += 8) {
       float2 v[8];
       float cm = -INFINITY;
@@ -88,6 +90,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
       mx = nm;
     }
     const float invl = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll 1
     for (int sp = 0; sp < S; ++sp) {
       const float m = s_w[h * S + sp];
       s_w[h * S + sp] = m > -INFINITY ? ex2a(m - mx) * invl : 0.f;
@@ -107,10 +110,12 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   __syncthreads();
 
   // ---- attention output: out_h = sum_s w_{h,s} O_{h,s}, four channels per task ----------------------------
+#pragma unroll 1
   for (int task = t0; task < n_task; task += t_stride) {
     const int h = task / D4, c4 = task - h * D4;
     const float4* src = reinterpret_cast<const float4*>(op + (size_t)h * MAX_SPLITS * g.D) + c4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
     for (int s0 = 0; s0 < S; s0 += 8) {
       float4 x[8];
 #pragma unroll
@@ -135,6 +140,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
   // run) -------------------------------------------------------------------------------------------------
   auto head_sum = [&](float2 r, int e) -> float {
     float term = 0.f;
+#pragma unroll 1
     for (int hb = 0; hb < g.Hq; hb += 32) {
       const int h = hb + lane;
       float2 rr = r;
