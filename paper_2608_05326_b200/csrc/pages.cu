@@ -332,6 +332,7 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
   const int ks_n = g.D >> 4, ng = g.D / g.group;
   const int n_kt = (g.W / g.group) * ks_n, n_vt = g.tiles * ng * 2, tpp = n_kt > n_vt ? n_kt : n_vt;
   const int per_rec = g.Hkv * 2 * tpp, total = n_entries * per_rec;
+#pragma unroll 1
   for (int id = gw; id < total; id += n_warps) {
     const int rec = id / per_rec, rem = id - rec * per_rec, hp = rem / tpp, task = rem - hp * tpp;
     const int hk = hp >> 1, part = hp & 1;
@@ -345,6 +346,9 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
     int c0, c1, c2 = 0;
     if (part == 0) { c0 = task / ks_n; c1 = task - c0 * ks_n; }                    // (blk, ks)
     else { c2 = task & 1; c1 = (task >> 1) % ng; c0 = (task >> 1) / ng; }           // (tile, gc, ks)
+    // one promotion at most follows: the record's own (kind 1) or the one linked to its quantization
+    const char* pq = nullptr;
+    char* pf = nullptr;
     if (kind == 0) {
       const T* rows = nullptr;
       const char* fp_head = nullptr;
@@ -354,14 +358,14 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
       if (part == 0) quant_key_task<T>(g, c0, c1, rows, fp_head, qb, lane);
       else quant_value_task<T>(g, c0, c1, c2, rows, fp_head, qb, lane);
       if (r1.y >= 0) {
-        const char* pq = q_u + (size_t)r1.y * g.q_page_bytes;
-        char* pf = fp_u + (size_t)r0.w * g.fp_page_bytes;
-        if (part == 0) promote_key_task<T>(g, c0, c1, pq, pf, lane);
-        else promote_value_task<T>(g, c0, c1, c2, pq, pf, lane);
+        pq = q_u + (size_t)r1.y * g.q_page_bytes;
+        pf = fp_u + (size_t)r0.w * g.fp_page_bytes;
       }
     } else {
-      const char* pq = q_u + (size_t)r0.w * g.q_page_bytes;
-      char* pf = fp_u + (size_t)r1.x * g.fp_page_bytes;
+      pq = q_u + (size_t)r0.w * g.q_page_bytes;
+      pf = fp_u + (size_t)r1.x * g.fp_page_bytes;
+    }
+    if (pq) {
       if (part == 0) promote_key_task<T>(g, c0, c1, pq, pf, lane);
       else promote_value_task<T>(g, c0, c1, c2, pq, pf, lane);
     }

@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
     if (tid < 32) {
       int found = -1;
       const int32_t* owner = a.st.fp_owner + (size_t)u * g.PF;
+#pragma unroll 1
       for (int base = 0; base < g.PF && found < 0; base += 32) {
         const int pg = base + tid;
         const bool free_pg = pg < g.PF && owner[pg] < 0;
@@ -162,6 +163,7 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
     // unfilled token slots of the open window must hold finite values (they are multiplied by a zero
     // probability in the PV product)
     uint4* z = reinterpret_cast<uint4*>(pbase);
+#pragma unroll 4
     for (uint32_t i = tid; i < g.fp_page_bytes / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
   }
