@@ -526,15 +526,33 @@ static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void
   const size_t nu = (size_t)(l1 - l0) * g.batch;
   const size_t qb = nu * g.Hq * g.D * 2, kb = nu * g.Hkv * g.D * 2;
   QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  // Page-locked host buffers that the device can address are used in place where each byte is touched once:
+  // the append kernel reads the new token from them and the merge kernel writes `out` into them, which saves
+  // three copy operations (and their hand-overs between the copy engines and the SMs) per step.  The queries
+  // are read by every CTA of the attention kernel, so they always go through device memory.  Pageable buffers
+  // take staged copies throughout.
+  auto device_alias = [](const void* p) -> void* {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+  };
   QE_CUDA(h, cudaMemcpyAsync(h->stage_q, q_host, qb, cudaMemcpyHostToDevice, s));
+  const void* k_dev = nullptr;
+  const void* v_dev = nullptr;
   if (k_new_host) {
-    QE_CUDA(h, cudaMemcpyAsync(h->stage_k, k_new_host, kb, cudaMemcpyHostToDevice, s));
-    QE_CUDA(h, cudaMemcpyAsync(h->stage_v, v_new_host, kb, cudaMemcpyHostToDevice, s));
+    k_dev = device_alias(k_new_host);
+    v_dev = device_alias(v_new_host);
+    if (!k_dev || !v_dev) {
+      QE_CUDA(h, cudaMemcpyAsync(h->stage_k, k_new_host, kb, cudaMemcpyHostToDevice, s));
+      QE_CUDA(h, cudaMemcpyAsync(h->stage_v, v_new_host, kb, cudaMemcpyHostToDevice, s));
+      k_dev = h->stage_k;
+      v_dev = h->stage_v;
+    }
   }
-  const qevict_status st = decode_impl(h, layer, h->stage_q, k_new_host ? h->stage_k : nullptr,
-                                       k_new_host ? h->stage_v : nullptr, h->stage_out, s);
+  void* out_dev = device_alias(out_host);
+  const qevict_status st = decode_impl(h, layer, h->stage_q, k_dev, v_dev, out_dev ? out_dev : h->stage_out, s);
   if (st != QEVICT_OK) return st;
-  QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
+  if (!out_dev) QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
   if (sync) QE_CUDA(h, cudaStreamSynchronize(s));
   return QEVICT_OK;
 }
