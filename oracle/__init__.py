@@ -23,6 +23,7 @@ from .quantizer import (  # noqa: F401
     dequantize_window,
 )
 from .attention import accessible_attention  # noqa: F401
+from .rope import apply_rope, rope_frequencies, rotate_exact  # noqa: F401
 from .diagnostics import retained_windows, selection_churn, tier_mass_share  # noqa: F401
 from .cache import (  # noqa: F401
     OracleConfig,

@@ -59,6 +59,8 @@ it; the reading taken is Algorithm 1 with the Full tier drawn from the candidate
 F' = TopK_{K_f} of the ranked candidates whose state is not Quantized, Q' = TopK_{K_q} of the ranked remainder,
 E' = the rest.
 
+Pre-RoPE keys (rope_base > 0): see rope.py.
+
 Parity unpinned: the page-id assignment order above is this build's own rule (the
 paper never speaks of pages), so nothing outside this file fixes it; and the
 prefill window scores are an input here (the paper only says that prompt attention
@@ -72,6 +74,7 @@ import numpy as np
 from .attention import accessible_attention
 from .numerics import round_to_dtype
 from .quantizer import dequantize_window, quantize_window
+from .rope import apply_rope
 
 TIER_NONE, TIER_OPEN, TIER_AGED, TIER_FULL, TIER_QUANT, TIER_EVICTED, TIER_SINK = 0, 1, 2, 3, 4, 5, 6
 LEDGER_NONE, LEDGER_ACTIVE, LEDGER_DORMANT = 0, 1, 2
@@ -98,6 +101,7 @@ class OracleConfig:
     rank_param: float = 0.0  # lambda of the decayed score, p of the p-norm (integer >= 2)
     one_way: bool = False  # no promotion: a Quantized window never returns to the Full tier
     recent_windows: int = 0  # filled windows kept in the protected recent region
+    rope_base: float = 0.0  # > 0: stored keys are pre-RoPE and are rotated when attention reads them
 
     @property
     def scale(self):
@@ -255,6 +259,10 @@ class UnitOracle:
         mass = np.zeros(cfg.max_windows, dtype=np.float64)
         if not acc:
             return np.zeros((cfg.n_q_heads, cfg.head_dim)), mass
+        if cfg.rope_base > 0:
+            # stored keys are pre-RoPE: the rotation for the key's absolute position is applied when it is read
+            # (Migration-Stable Quantization: "RoPE is reapplied after dequantization")
+            acc = [(w, apply_rope(k, w * cfg.window + np.arange(n), cfg.rope_base, cfg.dtype), v, n) for w, k, v, n in acc]
         k_acc = np.concatenate([a[1] for a in acc], axis=1)
         v_acc = np.concatenate([a[2] for a in acc], axis=1)
         out, probs = accessible_attention(q, k_acc, v_acc, cfg.scale)
