@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--recent-windows", type=int, default=0, help="filled windows kept in the protected recent region")
     ap.add_argument("--rank-mode", type=int, default=0, help="0 cumulative attention (Eq. 1), 1 decayed, 2 p-norm")
     ap.add_argument("--rank-param", type=float, default=0.0, help="lambda of the decayed score / p of the p-norm")
+    ap.add_argument("--rope-base", type=float, default=0.0,
+                    help="> 0: keys are stored pre-RoPE and rotated by the attention kernel (0 in every BASELINE config)")
     ap.add_argument("--prefill-score", type=int, default=0, metavar="N_OBS",
                     help="instead of the decode loop: time qevict_prefill_score (window scores of one layer's prompt from "
                          "N_OBS observation queries per head) and print its own JSON line")
@@ -82,7 +84,7 @@ def make_workload(args, total_steps):
     batch = args.batch if args.batch is not None else wl.batch
     return replace(wl, n_layers=layers, batch=batch, steps=total_steps, rebalance_interval=args.rebalance_interval,
                    sink_windows=args.sink_windows, recent_windows=args.recent_windows, rank_mode=args.rank_mode,
-                   rank_param=args.rank_param)
+                   rank_param=args.rank_param, rope_base=args.rope_base)
 
 
 def peak_hbm_gbs():
@@ -207,7 +209,7 @@ def run_ours(args, rank, world):
                               wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
                               rebalance_interval_hint=args.rebalance_interval, device=dev.index,
                               sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
-                              rank_param=wl.rank_param)
+                              rank_param=wl.rank_param, rope_base=wl.rope_base)
     cache = binding.QEvictCache(cfg)
     if args.splits:
         cache.set_splits(args.splits)
@@ -310,7 +312,7 @@ def run_ours(args, rank, world):
             "units_per_step": wl.n_units, "context": wl.context, "window": wl.window, "quant_bits": wl.quant_bits,
             "group_size": wl.group_size, "fp_budget_windows": wl.fp_budget_windows,
             "q_budget_windows": wl.q_budget_windows, "sink_windows": wl.sink_windows, "recent_windows": wl.recent_windows,
-            "rebalance_interval": R, "append": append,
+            "rebalance_interval": R, "append": append, "rope_base": wl.rope_base,
             "l2": "inputs larger than L2 (KV working set %.0f MB per step)" % (kbytes / 1e6),
         },
         "layer_steps_per_sec": world * K * wl.n_units / (ms * 1e-3),

@@ -113,6 +113,14 @@ typedef struct {
   int32_t one_way;           /* 1: no promotion [promotion ablation: Full -> Quantized -> Evicted].  The paper gives
                                 only the transition diagram; reading: the Full tier is the best K_f candidates that
                                 are not Quantized, the Quantized tier the best K_q of all the others.  0: Algorithm 1 */
+  float rope_base;           /* > 0: the keys handed to the cache (prompt and k_new) are pre-RoPE and stay so in every
+                                tier; the attention kernel rotates each key for its absolute position (slot j of
+                                window w is position w * W + j) when it reads it, after dequantization for the
+                                low-bit tier [Migration-Stable Quantization: keys in the pre-RoPE domain with their
+                                absolute positions, RoPE reapplied after dequantization].  theta_i = rope_base^(-2i/d),
+                                pairs (i, i + d/2); cos, sin and every product and sum rounded to the execution
+                                datatype, as the models' own implementation does.  q arrives rotated.  0: keys are
+                                used as given.  qevict_prefill_score is refused while this is set. */
 } qevict_config;
 
 typedef struct {

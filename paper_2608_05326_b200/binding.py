@@ -38,7 +38,7 @@ class qevict_config(C.Structure):
         ("quant_bits", C.c_int32), ("group_size", C.c_int32), ("fp_budget_windows", C.c_int32),
         ("q_budget_windows", C.c_int32), ("max_context", C.c_int32), ("rebalance_interval_hint", C.c_int32),
         ("softmax_scale", C.c_float), ("device", C.c_int32), ("sink_windows", C.c_int32), ("recent_windows", C.c_int32),
-        ("rank_mode", C.c_int32), ("rank_param", C.c_float), ("one_way", C.c_int32),
+        ("rank_mode", C.c_int32), ("rank_param", C.c_float), ("one_way", C.c_int32), ("rope_base", C.c_float),
     ]
 
 
@@ -108,12 +108,12 @@ def _check(status, handle=None):
 
 def make_config(batch, n_layers, n_q_heads, n_kv_heads, head_dim, dtype, window, quant_bits, group_size,
                 fp_budget_windows, q_budget_windows, max_context, rebalance_interval_hint=0, softmax_scale=0.0,
-                device=0, sink_windows=0, recent_windows=0, rank_mode=0, rank_param=0.0, one_way=0):
+                device=0, sink_windows=0, recent_windows=0, rank_mode=0, rank_param=0.0, one_way=0, rope_base=0.0):
     dt = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, torch.float16: DTYPE_FP16, torch.bfloat16: DTYPE_BF16}[dtype]
     return qevict_config(C.sizeof(qevict_config), batch, n_layers, n_q_heads, n_kv_heads, head_dim, dt, window,
                          quant_bits, group_size, fp_budget_windows, q_budget_windows, max_context,
                          rebalance_interval_hint, softmax_scale, device, sink_windows, recent_windows, rank_mode,
-                         rank_param, int(one_way))
+                         rank_param, int(one_way), float(rope_base))
 
 
 # --- plain function wrappers, same names as the C entry points -----------------------------------------

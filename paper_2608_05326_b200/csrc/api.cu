@@ -79,6 +79,7 @@ const char* validate(const qevict_config* c) {
   if (c->sink_windows < 0 || c->recent_windows < 0) return "sink_windows and recent_windows must be >= 0";
   if (c->sink_windows + c->recent_windows > c->max_context / c->window) return "protected windows exceed max_context";
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return "softmax_scale must be finite and >= 0";
+  if (!(c->rope_base >= 0.f) || isinf(c->rope_base) || (c->rope_base > 0.f && c->rope_base < 1.f)) return "rope_base must be 0 or >= 1";
   return nullptr;
 }
 
@@ -102,6 +103,7 @@ void make_geometry(const qevict_config& c, Geometry& g) {
   g.aged_cap = (r + g.W - 1) / g.W + 1;
   g.n_sink = c.sink_windows; g.n_recent = c.recent_windows;
   g.rank_mode = c.rank_mode; g.rank_param = c.rank_param; g.one_way = c.one_way != 0;
+  g.rope_base = c.rope_base;
   g.Kfp = g.Kf + g.n_sink + g.n_recent;
   g.PF = g.Kfp + g.aged_cap + 1;
   g.PQ = g.Kq + g.Kf;
@@ -158,6 +160,7 @@ size_t carve(const Geometry& g, char* base, State* st, qevict_ctx* ctx) {
   s.wrec = (float2*)take(U * g.Hq * (size_t)g.EMAX * 8);
   s.mass_e = (float*)take(U * (size_t)g.EMAX * 4);
   s.status = (int32_t*)take(STATUS_BYTES);
+  s.rope_table = (uint4*)take(g.rope_base > 0.f ? (size_t)g.NW * g.tiles * 32u * (g.D / 2) * 4u : 0);
 #ifdef QEVICT_TRACE
   s.trace = (unsigned long long*)take(TRACE_BYTES);
 #endif
@@ -215,7 +218,7 @@ int qevict::choose_splits(const qevict_ctx* h, int n_units) {
   }
   const int entries = g.Kfp + g.Kq + 1;
   const long pairs = (long)n_units * g.Hkv;
-  const long slots = (long)h->sm_count * 3;  // resident CTAs
+  const long slots = (long)h->sm_count * (g.rope_base > 0.f ? 2 : 3);  // resident CTAs
   int best = smin;
   double best_cost = 1e30;
   const int smax = entries / DECODE_WARPS < 1 ? 1 : (entries / DECODE_WARPS > MAX_SPLITS ? MAX_SPLITS : entries / DECODE_WARPS);
@@ -274,6 +277,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
+  p.rope = reinterpret_cast<const char*>(h->st.rope_table);
 #ifdef QEVICT_TRACE
   p.trace = a.trace;
 #endif
@@ -346,10 +350,10 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
   const size_t need = carve(g, (char*)device_mem, &h->st, h);
   if (need > bytes) { delete h; return QEVICT_ERR_NO_MEMORY; }
   switch ((g.dtype == QEVICT_DTYPE_BF16 ? 2 : 0) + (g.D == 128 ? 1 : 0)) {
-    case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles, g.G); break;
-    case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles, g.G); break;
-    case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles, g.G); break;
-    default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles, g.G); break;
+    case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
+    case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
+    case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
+    default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
   }
   if (!h->decode_fn) { delete h; return QEVICT_ERR_UNSUPPORTED; }
   h->layers.resize(g.n_layers);
@@ -381,6 +385,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
 #ifdef QEVICT_TRACE
     if (e == cudaSuccess) e = trace_clear(h, TRACE_CALLS + 1);
 #endif
+    if (e == cudaSuccess) e = launch_rope_table(g, h->st, 0);
     if (e == cudaSuccess) e = route_prepare(route_smem_bytes(g, next_pow2(g.NW)));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
   }

@@ -40,6 +40,7 @@ struct Geometry {
   int n_sink, n_recent;  // protected windows: sink prefix, recent region (besides the open window)
   int rank_mode;     // QEVICT_RANK_*
   int one_way;       // 1: a Quantized window never returns to the Full tier
+  float rope_base;   // > 0: stored keys are pre-RoPE, rotated by the attention kernel
   float rank_param;  // lambda or p
   int Kfp;       // K_f + n_sink + n_recent: windows that may need a full-precision page in one event
   int tiles;     // W / 32
@@ -80,6 +81,7 @@ struct State {
   float2* wrec;         // [EMAX][Hq] {window exp-sum, reference max (log2 domain)}
   float* mass_e;        // [EMAX] last step's mass per entry
   int32_t* status;      // [1] (shared by all units)
+  uint4* rope_table;    // [NW * tiles] blocks of cos / sin pairs in the key tile's fragment order (shared by all units)
 #ifdef QEVICT_TRACE
   unsigned long long* trace;  // [TRACE_CALLS + 1] call blocks (shared by all units)
 #endif

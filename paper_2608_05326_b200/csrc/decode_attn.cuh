@@ -47,16 +47,18 @@ struct DecodeParams {
   int e_bound;            // upper bound of every unit's work-list length (host's mirror of the window counts)
   uint32_t fp_page_bytes, q_page_bytes;
   float scale_log2;
+  const char* rope;       // pre-RoPE keys: blocks of cos / sin pairs, one per 32 positions, in the key tile's fragment order
 #ifdef QEVICT_TRACE
   unsigned long long* trace;  // this call's block of the kernel timeline
 #endif
 };
 
-static constexpr int NSLOT = 2;                   // ring slots per warp
 static constexpr uint32_t WAIT_LIMIT = 1u << 20;  // mbarrier try_wait attempts before giving up
 
-template <class T, int D, int BITS, int GROUP, int TILES>
+template <class T, int D, int BITS, int GROUP, int TILES, bool ROPE>
 struct DecodeTraits {
+  // ring slots per warp: with pre-RoPE keys a tile's rotation block sits in the ring beside the key tile
+  static constexpr int NSLOT = ROPE ? 3 : 2;
   static constexpr int KG = D / 32;   // 16-byte key vectors per 8-token row block
   static constexpr int KS = D / 16;   // k-steps of the QK product
   static constexpr int MT = D / 16;   // m-tiles (16 channels) of the PV product
@@ -73,6 +75,8 @@ struct DecodeTraits {
   // a ring slot holds a full-precision key tile or value tile, or a whole quantized tile
   // (key codes, value codes, value params as they lie in the page, then the key params)
   static constexpr uint32_t SLOT_BYTES = FP_TILE_BYTES;
+  static constexpr uint32_t ROPE_BLOCK_BYTES = 32 * (D / 2) * 4;  // (cos, sin) of 32 positions x d/2 frequencies
+  static_assert(ROPE_BLOCK_BYTES <= SLOT_BYTES, "a rotation block must fit a slot");
   static constexpr uint32_t RING_BYTES = DECODE_WARPS * NSLOT * SLOT_BYTES;
   static constexpr uint32_t SMEM_BYTES = RING_BYTES + DECODE_WARPS * NSLOT * 8;
   static_assert(Q_TILE_STRIDE + KP_BYTES <= SLOT_BYTES, "a quantized tile must fit a slot");
@@ -122,6 +126,14 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst),
       "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
+}
+
+// The same without a cache hint: the rotation table of pre-RoPE keys is shared by every unit and KV head and
+// should stay in L2.
+__device__ __forceinline__ void bulk_g2s_plain(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -174,6 +186,83 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[2][4], const uint32_t (&qa)
         const uint32_t a3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
         mma16816<T>(s[mt], a0, a1, a2, a3, qa[ks][0], qa[ks][1]);
       }
+    }
+  }
+}
+
+// ---- pre-RoPE keys: S^T = R(K) Q^T ---------------------------------------------------------------------------
+// The partner of channel c < d/2 is channel c + d/2: the same lane, the same register, KS/2 k-steps further on.
+// A rotation block holds, for k-step ks' < KS/2 and token block mt, two 16-byte vectors per lane:
+// {C r0, S r0, C r1, S r1} and {C r2, S r2, C r3, S r3}, C / S = the (cos, sin) pairs of register r's two channels
+// at register r's token row.  x' = RN(RN(x c) - RN(y s)), y' = RN(RN(y c) + RN(x s)) in the execution datatype,
+// every operation rounded on its own (the _rn intrinsics are never contracted into a fused multiply-add).
+template <class T>
+__device__ __forceinline__ void rope_pair(uint32_t& x, uint32_t& y, uint32_t c, uint32_t s) {
+  using T2 = typename Tr<T>::T2;
+  const T2 X = as_t2<T2>(x), Y = as_t2<T2>(y), C = as_t2<T2>(c), S = as_t2<T2>(s);
+  x = as_u32(__hsub2_rn(__hmul2_rn(X, C), __hmul2_rn(Y, S)));
+  y = as_u32(__hadd2_rn(__hmul2_rn(Y, C), __hmul2_rn(X, S)));
+}
+template <class T>
+__device__ __forceinline__ void rope_fragments(uint4& a, uint4& b, uint32_t rslot, int ksp, int mt, int lane) {
+  const uint4 c0 = lds16(rslot + (((ksp * 2 + mt) * 2 + 0) * 32 + lane) * 16);
+  const uint4 c1 = lds16(rslot + (((ksp * 2 + mt) * 2 + 1) * 32 + lane) * 16);
+  rope_pair<T>(a.x, b.x, c0.x, c0.y);
+  rope_pair<T>(a.y, b.y, c0.z, c0.w);
+  rope_pair<T>(a.z, b.z, c1.x, c1.y);
+  rope_pair<T>(a.w, b.w, c1.z, c1.w);
+}
+
+template <class T, int D>
+__device__ __forceinline__ void qk_fp_tile_rope(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot,
+                                                uint32_t rslot, int lane) {
+  constexpr int KS = D / 16;
+#pragma unroll
+  for (int ksp = 0; ksp < KS / 2; ++ksp) {
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      uint4 a = lds16(slot + ((ksp * 2 + mt) * 32 + lane) * 16);
+      uint4 b = lds16(slot + (((ksp + KS / 2) * 2 + mt) * 32 + lane) * 16);
+      rope_fragments<T>(a, b, rslot, ksp, mt, lane);
+      mma16816<T>(s[mt], a.x, a.y, a.z, a.w, qa[ksp][0], qa[ksp][1]);
+      mma16816<T>(s[mt], b.x, b.y, b.z, b.w, qa[ksp + KS / 2][0], qa[ksp + KS / 2][1]);
+    }
+  }
+}
+
+template <class T, int D, int BITS>
+__device__ __forceinline__ void qk_q_tile_rope(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
+                                               uint32_t rslot, int lane) {
+  constexpr int KS = D / 16;
+  constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
+  constexpr uint32_t MG = Tr<T>::MAGIC;
+  constexpr int KPV = (BITS == 4) ? 2 : 4;  // k-steps per code vector
+  const int t = lane & 3;
+  uint32_t cw[KS / KPV][4];
+#pragma unroll
+  for (int v = 0; v < KS / KPV; ++v) {
+    const uint4 cv = lds16(slot + (v * 32 + lane) * 16);
+    cw[v][0] = cv.x; cw[v][1] = cv.y; cw[v][2] = cv.z; cw[v][3] = cv.w;
+  }
+  auto fragment = [&](int ks, int mt, const uint4& pr) -> uint4 {
+    const uint32_t w = (BITS == 4) ? cw[ks / KPV][(ks % KPV) * 2 + mt] : cw[ks / KPV][ks % KPV];
+    const int sh = (BITS == 4) ? 0 : mt * 8;
+    uint4 a;
+    a.x = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
+    a.y = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
+    a.z = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
+    a.w = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
+    return a;
+  };
+#pragma unroll
+  for (int ksp = 0; ksp < KS / 2; ++ksp) {
+    const uint4 pra = lds16(kp + (ksp * 4 + t) * 16), prb = lds16(kp + ((ksp + KS / 2) * 4 + t) * 16);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      uint4 a = fragment(ksp, mt, pra), b = fragment(ksp + KS / 2, mt, prb);
+      rope_fragments<T>(a, b, rslot, ksp, mt, lane);
+      mma16816<T>(s[mt], a.x, a.y, a.z, a.w, qa[ksp][0], qa[ksp][1]);
+      mma16816<T>(s[mt], b.x, b.y, b.z, b.w, qa[ksp + KS / 2][0], qa[ksp + KS / 2][1]);
     }
   }
 }
@@ -342,10 +431,10 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
   }
 }
 
-template <class T, int D, int BITS, int GROUP, int TILES, bool PACK>
-__global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const DecodeParams p) {
-  using TT = DecodeTraits<T, D, BITS, GROUP, TILES>;
-  constexpr int KS = TT::KS, MT = TT::MT;
+template <class T, int D, int BITS, int GROUP, int TILES, bool PACK, bool ROPE>
+__global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_kernel(const DecodeParams p) {
+  using TT = DecodeTraits<T, D, BITS, GROUP, TILES, ROPE>;
+  constexpr int KS = TT::KS, MT = TT::MT, NSLOT = TT::NSLOT;
   extern __shared__ __align__(128) unsigned char smem[];
   const int s = blockIdx.x, hk = blockIdx.y, ul = blockIdx.z;
   const int u = p.unit0 + ul;
@@ -384,9 +473,11 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   if (lane >= my_n) my_ent = make_uint2(0u, 0u);
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------
-  // pieces per tile: full precision = 2 (key tile, value tile), quantized = 1 (the whole tile)
+  // pieces per tile: full precision = key tile, value tile; quantized = the whole tile; with pre-RoPE keys the
+  // tile's rotation block follows the piece that holds the keys
   int pr_ci = 0, pr_tile = 0, pr_part = 0, issued = 0, consumed = 0;
   bool dead = false, pr_isq = false;
+  uint32_t pr_win = 0;
   const char* pr_base = nullptr;  // page of the producer's current entry (this KV head), set on its first piece
   const char* const fp_unit = p.fp_pool + (size_t)u * p.PF * p.fp_page_bytes + (size_t)hk * TT::FP_HEAD_BYTES;
   const char* const q_unit = p.q_pool + (size_t)u * p.PQ * p.q_page_bytes + (size_t)hk * TT::Q_HEAD_BYTES;
@@ -396,14 +487,20 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
     if (pr_tile == 0 && pr_part == 0) {
       const uint32_t ex = __shfl_sync(0xffffffffu, my_ent.x, pr_ci), ey = __shfl_sync(0xffffffffu, my_ent.y, pr_ci);
       pr_isq = (ex >> ENTRY_KIND_SHIFT) == KIND_Q;
+      pr_win = ex & ENTRY_WINDOW_MASK;
       pr_base = pr_isq ? q_unit + (size_t)ey * p.q_page_bytes : fp_unit + (size_t)ey * p.fp_page_bytes;
     }
+    const bool is_rope = ROPE && pr_part == 1;
     if (lane == 0) {
       const int slot = issued % NSLOT;
       const uint32_t dst = ring + slot * TT::SLOT_BYTES, bar = bars + slot * 8;
-      if (!pr_isq) {
+      if (is_rope) {
+        mbar_expect_tx(bar, TT::ROPE_BLOCK_BYTES);
+        bulk_g2s_plain(dst, p.rope + ((size_t)pr_win * TILES + pr_tile) * TT::ROPE_BLOCK_BYTES, TT::ROPE_BLOCK_BYTES, bar);
+      } else if (!pr_isq) {
+        const int half = pr_part ? 1 : 0;  // key tile, then value tile
         mbar_expect_tx(bar, TT::FP_TILE_BYTES);
-        bulk_g2s(dst, pr_base + (size_t)(pr_tile * 2 + pr_part) * TT::FP_TILE_BYTES, TT::FP_TILE_BYTES, bar, l2pol);
+        bulk_g2s(dst, pr_base + (size_t)(pr_tile * 2 + half) * TT::FP_TILE_BYTES, TT::FP_TILE_BYTES, bar, l2pol);
       } else {
         mbar_expect_tx(bar, TT::Q_TILE_STRIDE + TT::KP_BYTES);
         bulk_g2s(dst, pr_base + (size_t)pr_tile * TT::Q_TILE_STRIDE, TT::Q_TILE_STRIDE, bar, l2pol);
@@ -411,15 +508,15 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
       }
     }
     ++issued;
-    if (++pr_part == (pr_isq ? 1 : 2)) {
+    if (++pr_part == (pr_isq ? 1 : 2) + (ROPE ? 1 : 0)) {
       pr_part = 0;
       if (++pr_tile == TILES) { pr_tile = 0; ++pr_ci; }
     }
   };
-  // wait for the next piece in order; returns its slot address
-  auto acquire = [&]() -> uint32_t {
-    const int slot = consumed % NSLOT;
-    if (!dead && !mbar_wait(bars + slot * 8, (consumed / NSLOT) & 1)) {
+  // wait for the piece `ahead` places after the next one in order; returns its slot address
+  auto acquire = [&](int ahead = 0) -> uint32_t {
+    const int k = consumed + ahead, slot = k % NSLOT;
+    if (!dead && !mbar_wait(bars + slot * 8, (k / NSLOT) & 1)) {
       dead = true;
       if (lane == 0) record_check(p.status, CHECK_COPY_TIMEOUT);
     }
@@ -465,7 +562,14 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
       uint32_t pa[2][2], pb[2][2];
       if (kind != KIND_Q) {
         uint32_t sl = acquire();
-        if (!dead && ntok > 0) {
+        if (ROPE) {
+          const uint32_t rs = acquire(1);
+          if (!dead && ntok > 0) {
+            qk_fp_tile_rope<T, D>(sacc, qa, sl, rs, lane);
+            softmax_tile<T, MT, PACK>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
+          }
+          release();
+        } else if (!dead && ntok > 0) {
           qk_fp_tile<T, D>(sacc, qa, sl, lane);
           softmax_tile<T, MT, PACK>(sacc, ntok, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
         }
@@ -475,12 +579,15 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
         release();
       } else {
         const uint32_t sl = acquire();
+        const uint32_t rs = ROPE ? acquire(1) : 0u;
         if (!dead) {
-          qk_q_tile<T, D, BITS>(sacc, qa, sl, sl + TT::Q_TILE_STRIDE, lane);
+          if (ROPE) qk_q_tile_rope<T, D, BITS>(sacc, qa, sl, sl + TT::Q_TILE_STRIDE, rs, lane);
+          else qk_q_tile<T, D, BITS>(sacc, qa, sl, sl + TT::Q_TILE_STRIDE, lane);
           softmax_tile<T, MT, PACK>(sacc, 32, p.scale_log2, lane, m_run, l_run, wsum, o, pa, pb);
           pv_q_tile<T, D, BITS, GROUP, PACK>(o, pa, pb, sl + TT::KC_BYTES, lane);
         }
         release();
+        if (ROPE) release();
       }
     }
     if (g == 0) {
@@ -535,33 +642,34 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, 3) decode_attn_kernel(const
   }
 }
 
-template <class T, int D, int BITS, int GROUP, int TILES, bool PACK>
+template <class T, int D, int BITS, int GROUP, int TILES, bool PACK, bool ROPE>
 cudaError_t launch_decode_attn(const DecodeParams& p, int n_units, cudaStream_t stream) {
-  using TT = DecodeTraits<T, D, BITS, GROUP, TILES>;
+  using TT = DecodeTraits<T, D, BITS, GROUP, TILES, ROPE>;
   static bool prepared = false;
   if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK>,
+    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK, ROPE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TT::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     prepared = true;
   }
   dim3 grid(p.S, p.Hkv, n_units);
-  return launch_pdl(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK>, grid, dim3(DECODE_WARPS * 32), TT::SMEM_BYTES, stream, p);
+  return launch_pdl(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK, ROPE>, grid, dim3(DECODE_WARPS * 32), TT::SMEM_BYTES, stream, p);
 }
 
 // explicit dispatch table entry points, one per (dtype, D) translation unit
 typedef cudaError_t (*decode_launch_fn)(const DecodeParams&, int, cudaStream_t);
-decode_launch_fn decode_dispatch_h64(int bits, int group, int tiles, int heads_per_kv);
-decode_launch_fn decode_dispatch_h128(int bits, int group, int tiles, int heads_per_kv);
-decode_launch_fn decode_dispatch_b64(int bits, int group, int tiles, int heads_per_kv);
-decode_launch_fn decode_dispatch_b128(int bits, int group, int tiles, int heads_per_kv);
+decode_launch_fn decode_dispatch_h64(int bits, int group, int tiles, int heads_per_kv, bool rope);
+decode_launch_fn decode_dispatch_h128(int bits, int group, int tiles, int heads_per_kv, bool rope);
+decode_launch_fn decode_dispatch_b64(int bits, int group, int tiles, int heads_per_kv, bool rope);
+decode_launch_fn decode_dispatch_b128(int bits, int group, int tiles, int heads_per_kv, bool rope);
 
 #define QEVICT_DECODE_CASE(T, D, B, G, TL)    \
   if (bits == B && group == G && tiles == TL) \
-    return heads_per_kv <= 4 ? launch_decode_attn<T, D, B, G, TL, true> : launch_decode_attn<T, D, B, G, TL, false>;
+    return rope ? (heads_per_kv <= 4 ? launch_decode_attn<T, D, B, G, TL, true, true> : launch_decode_attn<T, D, B, G, TL, false, true>) \
+                : (heads_per_kv <= 4 ? launch_decode_attn<T, D, B, G, TL, true, false> : launch_decode_attn<T, D, B, G, TL, false, false>);
 
 #define QEVICT_DECODE_DISPATCH(NAME, T, D)                                  \
-  decode_launch_fn NAME(int bits, int group, int tiles, int heads_per_kv) { \
+  decode_launch_fn NAME(int bits, int group, int tiles, int heads_per_kv, bool rope) { \
     QEVICT_DECODE_CASE(T, D, 4, 32, 1)                                      \
     QEVICT_DECODE_CASE(T, D, 2, 32, 1)                                      \
     QEVICT_DECODE_CASE(T, D, 4, 32, 2)                                      \

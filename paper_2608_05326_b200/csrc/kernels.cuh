@@ -16,6 +16,9 @@ struct KernelArgs {
 #endif
 };
 
+// cache set-up: the rotation table of pre-RoPE keys (nothing to do when rope_base is 0)
+cudaError_t launch_rope_table(const Geometry& g, const State& st, cudaStream_t s);
+
 // decode step ---------------------------------------------------------------------------------------
 // A0: append one token per unit to its open window (opens one first if needed, zeroing the page).
 cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s);

@@ -108,6 +108,7 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   p.q = q; p.entries = a.st.entries; p.n_live = a.st.n_live; p.open_fill = a.st.open_fill;
   p.fp_pool = a.st.fp_pool; p.q_pool = a.st.q_pool; p.o_part = a.st.o_part; p.ml = a.st.ml; p.wrec = a.st.wrec;
   p.status = a.st.status;
+  p.rope = reinterpret_cast<const char*>(a.st.rope_table);
 #ifdef QEVICT_TRACE
   p.trace = a.trace;
 #endif

@@ -278,6 +278,7 @@ QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, co
   const Geometry& g = h->geo;
   auto bad = [&](const char* msg) { h->last_error = msg; return QEVICT_ERR_INVALID_ARG; };
   if (!k || !q_obs || !window_scores || !scratch) return bad("k, q_obs, window_scores and scratch must not be NULL");
+  if (g.rope_base > 0.f) { h->last_error = "prefill scoring is not built for pre-RoPE keys"; return QEVICT_ERR_UNSUPPORTED; }
   if (n_obs < 1 || n_obs > 64) return bad("n_obs must be in 1..64");
   if (ctx_tokens < g.W || ctx_tokens % g.W || ctx_tokens > h->cfg.max_context) return bad("ctx_tokens must be a multiple of window within max_context");
   uint64_t need = 0;

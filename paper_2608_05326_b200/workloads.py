@@ -47,6 +47,7 @@ class Workload:
     rank_mode: int = 0       # 0 cumulative attention, 1 exponentially decayed, 2 attention p-norm
     rank_param: float = 0.0  # lambda or p
     one_way: bool = False    # no promotion (promotion ablation)
+    rope_base: float = 0.0   # > 0: keys are pre-RoPE and rotated at attention time
 
     @property
     def n_units(self):

@@ -22,7 +22,7 @@ def oracle_config(wl, aged_windows):
     return OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits, wl.group_size,
                         wl.fp_budget_windows, wl.q_budget_windows, wl.max_context, aged_windows=aged_windows,
                         sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
-                        rank_param=wl.rank_param, one_way=wl.one_way)
+                        rank_param=wl.rank_param, one_way=wl.one_way, rope_base=wl.rope_base)
 
 
 def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
@@ -31,7 +31,8 @@ def gpu_config(wl, batch=None, n_layers=None, rebalance_interval=None):
                                wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window, wl.quant_bits,
                                wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
                                rebalance_interval_hint=r, sink_windows=wl.sink_windows, recent_windows=wl.recent_windows,
-                               rank_mode=wl.rank_mode, rank_param=wl.rank_param, one_way=wl.one_way)
+                               rank_mode=wl.rank_mode, rank_param=wl.rank_param, one_way=wl.one_way,
+                               rope_base=wl.rope_base)
 
 
 def aged_capacity(wl, rebalance_interval=None):

@@ -471,3 +471,40 @@ def test_random_configurations_lockstep(wl):
     assert st["deletions"] == sum(x.stats["deletions"] for x in run.oracles.values())
     assert st["promotions"] == sum(x.stats["promotions"] for x in run.oracles.values())
     run.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, rope_base=10000.0),
+    dict(dtype="fp16", head_dim=64, n_q_heads=4, n_kv_heads=2, rope_base=500000.0),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1, quant_bits=2, rope_base=500000.0),
+    dict(dtype="fp16", head_dim=128, n_q_heads=7, n_kv_heads=1, window=64, group_size=64, quant_bits=2, rope_base=10000.0),
+    dict(dtype="bf16", head_dim=64, n_q_heads=3, n_kv_heads=1, window=64, quant_bits=4, rope_base=1000000.0,
+         context=64 * 2040, fp_budget_windows=5, q_budget_windows=9),
+])
+def test_pre_rope_keys_rotated_at_attention_time(kw):
+    # the cache holds pre-RoPE keys in every tier (they are quantized and promoted as such: codes and pages must
+    # still match bit for bit) and the attention kernel rotates each key for its absolute position when it reads
+    # it, after dequantization; the last case puts the positions near 130000
+    ls = _lockstep()
+    wl = _small("rope", steps=70, **kw)
+    run = ls.LockstepRun(wl, rebalance_interval=2)
+    run.check_state("all", "after prefill")
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    o = run.oracles[0]
+    st = run.cache.stats()
+    assert st["promotions"] == o.stats["promotions"] and st["quantizations"] == o.stats["quantizations"] > 0
+    run.close()
+
+
+def test_pre_rope_keys_change_the_result():
+    # the same inputs with and without the rotation must not give the same output (a kernel that ignored the
+    # rotation table would pass a comparison against itself, not this one)
+    ls = _lockstep()
+    a = ls.LockstepRun(_small("norope", steps=3), oracle_units=[])
+    b = ls.LockstepRun(_small("norope", steps=3, rope_base=10000.0), oracle_units=[])
+    oa = a.step(append=True, check_mass=False)
+    ob = b.step(append=True, check_mass=False)
+    assert (oa.float() - ob.float()).abs().max() > 1e-2
+    a.close(); b.close()
