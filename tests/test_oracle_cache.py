@@ -537,3 +537,39 @@ def test_tier_capacities_closed_form():
     assert (k_f, k_q) == (22, 170)
     assert k_f * m_f <= 0.3 * 10_000_000 < (k_f + 1) * m_f
     assert k_q * m_q <= 0.7 * 10_000_000 < (k_q + 1) * m_q
+
+
+# ------------------------------------------------------------------------------- pre-RoPE keys
+def test_pre_rope_cache_with_full_budget_equals_attention_over_rotated_keys():
+    """With every window in the Full tier the cache must give plain attention over the keys rotated for their
+    absolute positions (complex multiplication of the half-split pairs, here in float64): the stored keys stay
+    pre-RoPE, positions count from the start of the prompt through the appended tokens, values are untouched.
+    The rounding of the rotated keys to the execution datatype bounds the difference."""
+    from dataclasses import replace as dc_replace
+
+    dtype = "fp16"
+    rng = np.random.default_rng(21)
+    cfg = dc_replace(_small_cfg(dtype, k_f=64, k_q=4), rope_base=10000.0)
+    u, k, v, _ = _prefilled(cfg, rng)
+    ks, vs = [k], [v]
+    d = cfg.head_dim
+    freq = 10000.0 ** (-2.0 * np.arange(d // 2) / d)
+    for t in range(12):
+        q = _rand_T(rng, (cfg.n_q_heads, d), dtype)
+        kn = _rand_T(rng, (cfg.n_kv_heads, d), dtype)
+        vn = _rand_T(rng, (cfg.n_kv_heads, d), dtype)
+        ks.append(kn[:, None]); vs.append(vn[:, None])
+        out, mass = u.decode_attn(q, kn, vn)
+        kk = np.concatenate(ks, 1)
+        z = (kk[..., : d // 2] + 1j * kk[..., d // 2 :]) * np.exp(1j * np.outer(np.arange(kk.shape[1]), freq))
+        ref, p = _full_attention_reference(q, np.concatenate([z.real, z.imag], -1), np.concatenate(vs, 1), cfg.scale)
+        assert np.abs(out - ref).max() < 2e-2 and np.abs(out - ref).mean() < 2e-3
+        assert np.isclose(mass.sum(), cfg.n_q_heads, rtol=1e-12)
+        # the stored keys are still the ones that were handed in
+        assert np.array_equal(u.fp[0][0], k[:, : cfg.window])
+    # and the rotation matters: without it the same cache state gives a different answer
+    u2 = UnitOracle(dc_replace(cfg, rope_base=0.0))
+    u2.prefill_assign(k, v, np.zeros(k.shape[1] // cfg.window))
+    o2, _ = u2.decode_attn(q)
+    o1, _ = u.decode_attn(q)
+    assert np.abs(o1 - o2).max() > 1e-2
