@@ -425,8 +425,9 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
 
 def _random_workloads(n, seed=20260805):
     """Seeded draws over the supported configuration space (shapes, tiers, protected regions, ranking
-    functions, routing intervals)."""
+    functions, routing intervals, pre-RoPE keys in two draws of five)."""
     rng = np.random.default_rng(seed)
+    rope_rng = np.random.default_rng(seed + 1)  # its own stream: the other draws stay what they were
     out = []
     for i in range(n):
         window = int(rng.choice([32, 64]))
@@ -447,7 +448,8 @@ def _random_workloads(n, seed=20260805):
                     context=n_win * window, fp_budget_windows=k_f, q_budget_windows=k_q,
                     sink_windows=int(rng.integers(0, 3)), recent_windows=int(rng.integers(0, 3)),
                     rank_mode=mode, rank_param=param, steps=2 * window + int(rng.integers(3, 20)),
-                    batch=int(rng.choice([1, 2])), rebalance_interval=interval)
+                    batch=int(rng.choice([1, 2])), rebalance_interval=interval,
+                    rope_base=float(rope_rng.choice([0.0, 0.0, 0.0, 10000.0, 500000.0])))
         out.append(wl)
     return out
 
