@@ -120,7 +120,7 @@ typedef struct {
                                 absolute positions, RoPE reapplied after dequantization].  theta_i = rope_base^(-2i/d),
                                 pairs (i, i + d/2); cos, sin and every product and sum rounded to the execution
                                 datatype, as the models' own implementation does.  q arrives rotated.  0: keys are
-                                used as given.  qevict_prefill_score is refused while this is set. */
+                                used as given. */
 } qevict_config;
 
 typedef struct {
@@ -175,8 +175,10 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
  *   k             device, [batch][H_kv][ctx_tokens][d] in the execution datatype (one layer)
  *   q_obs         device, [batch][n_obs][H_q][d], n_obs in 1..64
  *   window_scores device, float32 [batch][ctx_tokens / W] (output)
- *   scratch       device, at least qevict_prefill_score_scratch_bytes(...) bytes, 8-byte aligned; contents
+ *   scratch       device, at least qevict_prefill_score_scratch_bytes(...) bytes, 16-byte aligned; contents
  *                 are overwritten
+ * With rope_base > 0 the keys are pre-RoPE like everything the cache is given: the scores are taken over a copy
+ * rotated for positions 0 .. ctx_tokens - 1, kept in the scratch buffer (which is that much larger).
  * Deterministic (fixed summation order). */
 QEVICT_API qevict_status qevict_prefill_score_scratch_bytes(qevict_handle h, int32_t n_obs, int32_t ctx_tokens,
                                                             uint64_t* bytes);

@@ -18,6 +18,8 @@ struct KernelArgs {
 
 // cache set-up: the rotation table of pre-RoPE keys (nothing to do when rope_base is 0)
 cudaError_t launch_rope_table(const Geometry& g, const State& st, cudaStream_t s);
+// prompt keys [rows][ctx][d] (pre-RoPE) -> rotated for positions 0 .. ctx-1 (prefill scoring with pre-RoPE keys)
+cudaError_t launch_rope_rotate_prompt(const Geometry& g, const void* k, void* out, long rows, int ctx, cudaStream_t s);
 
 // decode step ---------------------------------------------------------------------------------------
 // A0: append one token per unit to its open window (opens one first if needed, zeroing the page).

@@ -269,6 +269,8 @@ extern "C" {
 QEVICT_API qevict_status qevict_prefill_score_scratch_bytes(qevict_handle h, int32_t n_obs, int32_t ctx_tokens, uint64_t* bytes) {
   if (!h || !bytes || n_obs < 1 || ctx_tokens < 32 || ctx_tokens % 32) return QEVICT_ERR_INVALID_ARG;
   *bytes = (uint64_t)h->geo.batch * ((uint64_t)(ctx_tokens / 32) + 1) * n_obs * h->geo.Hq * sizeof(float2);
+  // pre-RoPE keys: room for a rotated copy of the prompt keys behind the records
+  if (h->geo.rope_base > 0.f) *bytes = ((*bytes + 255) & ~(uint64_t)255) + (uint64_t)h->geo.batch * h->geo.Hkv * ctx_tokens * h->geo.D * 2;
   return QEVICT_OK;
 }
 
@@ -278,7 +280,6 @@ QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, co
   const Geometry& g = h->geo;
   auto bad = [&](const char* msg) { h->last_error = msg; return QEVICT_ERR_INVALID_ARG; };
   if (!k || !q_obs || !window_scores || !scratch) return bad("k, q_obs, window_scores and scratch must not be NULL");
-  if (g.rope_base > 0.f) { h->last_error = "prefill scoring is not built for pre-RoPE keys"; return QEVICT_ERR_UNSUPPORTED; }
   if (n_obs < 1 || n_obs > 64) return bad("n_obs must be in 1..64");
   if (ctx_tokens < g.W || ctx_tokens % g.W || ctx_tokens > h->cfg.max_context) return bad("ctx_tokens must be a multiple of window within max_context");
   uint64_t need = 0;
@@ -289,6 +290,14 @@ QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, co
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSetDevice(h->cfg.device);
   float2* rec = static_cast<float2*>(scratch);
+  if (g.rope_base > 0.f) {
+    // the keys are pre-RoPE: the scores are taken over a rotated copy (prompt positions 0 .. ctx_tokens - 1)
+    const uint64_t rec_bytes = ((uint64_t)g.batch * ((uint64_t)n_tiles + 1) * n_obs * g.Hq * sizeof(float2) + 255) & ~(uint64_t)255;
+    void* k_rot = static_cast<char*>(scratch) + rec_bytes;
+    if (e == cudaSuccess) e = launch_rope_rotate_prompt(g, k, k_rot, (long)g.batch * g.Hkv, ctx_tokens, s);
+    k = k_rot;
+    h->launches += 1;
+  }
   if (nqh <= 128 && ctx_tokens % 128 == 0) {
     // tensor-core path: NP = queries padded to a power of two (tensor-memory columns)
     const int NP = nqh <= 32 ? 32 : (nqh <= 64 ? 64 : 128);

@@ -382,12 +382,14 @@ def test_config1_llama_shape_lockstep():
     (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1, context=1024), 12),              # 96 queries: N = 128
     (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, context=1056), 5),               # not a multiple of 128: CUDA cores
     (dict(dtype="fp16", head_dim=128, n_q_heads=8, n_kv_heads=1, context=1024), 20),              # 160 queries: CUDA cores
-], ids=["bf16-d128-g4", "fp16-d64-w64", "bf16-96q", "bf16-ctx1056", "fp16-160q"])
+    (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2, context=1024, rope_base=500000.0), 8),   # pre-RoPE keys
+    (dict(dtype="fp16", head_dim=64, n_q_heads=4, n_kv_heads=2, context=1056, rope_base=10000.0), 5),     # same, CUDA cores
+], ids=["bf16-d128-g4", "fp16-d64-w64", "bf16-96q", "bf16-ctx1056", "fp16-160q", "bf16-rope", "fp16-rope-ctx1056"])
 def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
     """Window scores of the prompt from observation queries: the GPU routine against the oracle's attention
     (raw mass per window summed over observers and heads); then a prefill_assign on both sides from the
     oracle's scores."""
-    from oracle import accessible_attention
+    from oracle import accessible_attention, apply_rope
     ls = _lockstep()
     wl = _small("pscore", steps=4, **kw)
     cache = binding.QEvictCache(ls.gpu_config(wl))
@@ -405,6 +407,8 @@ def test_prefill_scores_on_the_gpu_match_the_oracle(kw, n_obs):
     ref_all = []
     for u in range(wl.n_units):
         k64 = ks[u].double().numpy()
+        if wl.rope_base > 0:  # the prompt keys are pre-RoPE: attention sees them rotated for their positions
+            k64 = apply_rope(k64, np.arange(k64.shape[1]), wl.rope_base, wl.dtype)
         ref = np.zeros(wl.n_prompt_windows)
         for o in range(n_obs):
             _, p = accessible_attention(qs[u][o].double().numpy(), k64, np.zeros_like(k64[:, :, :1]), scale)
