@@ -218,7 +218,8 @@ int qevict::choose_splits(const qevict_ctx* h, int n_units) {
   }
   const int entries = g.Kfp + g.Kq + 1;
   const long pairs = (long)n_units * g.Hkv;
-  const long slots = (long)h->sm_count * (g.rope_base > 0.f ? 2 : 3);  // resident CTAs
+  // resident CTAs: three per SM; two where the third ring slot of the pre-RoPE variant makes the ring 96 KB
+  const long slots = (long)h->sm_count * (g.rope_base > 0.f && g.D == 128 ? 2 : 3);
   int best = smin;
   double best_cost = 1e30;
   const int smax = entries / DECODE_WARPS < 1 ? 1 : (entries / DECODE_WARPS > MAX_SPLITS ? MAX_SPLITS : entries / DECODE_WARPS);
