@@ -11,7 +11,7 @@
 // warp runs an independent online softmax over its windows; the four warps are merged in shared
 // memory and the CTA writes one partial (m, l, O) per query head of its KV head.
 //
-// Data movement: every warp owns a ring of NSLOT shared-memory slots.  Lane 0 streams the warp's
+// Data movement: every warp owns a ring of shared-memory slots (two; three with pre-RoPE keys).  Lane 0 streams the warp's
 // pages into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on one
 // mbarrier per slot) one piece ahead of the math; a page is stored fragment-major (layout.cuh),
 // so a piece is one contiguous run in global memory and every lane reads its operands from shared
@@ -26,6 +26,12 @@
 // head the residuals ride in the unused N columns 4..7 of the same product (PACK), otherwise they take
 // a second product.  A quantized tile is read as packed words, and codes become operands in
 // registers with one exact subtract and one fused multiply-add per pair.
+//
+// Pre-RoPE keys (ROPE instantiations) [Migration-Stable Quantization: keys in the pre-RoPE domain with their
+// absolute positions, RoPE reapplied after dequantization]: the ring has a third slot, into which the
+// rotation block of the tile's 32 positions follows the piece that holds the keys; the key fragments of
+// k-steps ks and ks + KS/2 (rotation partners sit in the same lane and register) are rotated in registers,
+// full-precision tiles as loaded and low-bit tiles after dequantization, before the products.
 #pragma once
 
 #include "common.cuh"
