@@ -55,6 +55,17 @@ def test_config3_long_context_window64_sampled_unit():
     _run(wl, oracle_units=[2], steps=70, check_all_units_mass=True)
 
 
+def test_config3_long_context_pre_rope_keys_sampled_unit():
+    # the 128k configuration with the keys stored pre-RoPE: positions up to 131 072 go through the rotation table
+    wl = replace(workloads.config(3), rope_base=500000.0)
+    _run(wl, oracle_units=[1], steps=24, check_all_units_mass=True)
+
+
+def test_config1_x32_layers_pre_rope_keys_sampled_unit():
+    wl = replace(workloads.config(1, n_layers=32), rope_base=500000.0)
+    _run(wl, oracle_units=[7], steps=34)
+
+
 @pytest.mark.parametrize("bits,fp_frac", [(4, 0.10), (2, 0.20)])
 def test_config4_qwen_gqa7_sampled_unit(bits, fp_frac):
     wl = workloads.config(4, bits=bits, fp_frac=fp_frac)
