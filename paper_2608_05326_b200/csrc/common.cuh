@@ -91,12 +91,14 @@ template <class T> struct Tr;
 template <> struct Tr<__half> {
   using T2 = __half2;
   static constexpr uint32_t MAGIC = 0x64006400u;  // 1024.0 in both halves: 1024 + code is exact
+  static constexpr int MANT = 10, EXP_BIAS = 15;   // significand bits, exponent bias
   static __device__ __forceinline__ __half from_float(float x) { return __float2half_rn(x); }
   static __device__ __forceinline__ float to_float(__half x) { return __half2float(x); }
 };
 template <> struct Tr<__nv_bfloat16> {
   using T2 = __nv_bfloat162;
   static constexpr uint32_t MAGIC = 0x43004300u;  // 128.0 in both halves: 128 + code is exact
+  static constexpr int MANT = 7, EXP_BIAS = 127;   // significand bits, exponent bias
   static __device__ __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
   static __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 };
@@ -120,6 +122,23 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
 template <class T> __device__ __forceinline__ uint32_t dequant2(uint32_t x, uint32_t s2, uint32_t z2) {
   using T2 = typename Tr<T>::T2;
   T2 c = __hsub2(as_t2<T2>(x), as_t2<T2>(Tr<T>::MAGIC));  // exact
+  return as_u32(__hfma2(c, as_t2<T2>(s2), as_t2<T2>(z2)));
+}
+
+// Two codes of BITS bits at bit position `pos` of each 16-bit half of `w` -> two dequantized values.  A code that
+// lies wholly inside the significand field of T needs no shift to become a number: planted at significand bit p
+// under the exponent of 2^(MANT - p), the half reads 2^(MANT - p) + code, and subtracting that power of two
+// leaves the code, exactly.  So only every CAP-th bit position costs a shift (CAP = the multiple of BITS that
+// fits the significand: 6 of 7 bits for 2-bit codes in bf16), and the shifted word serves CAP / BITS positions.
+// `pos` must be a compile-time constant after unrolling.
+template <class T, int BITS>
+__device__ __forceinline__ uint32_t dequant_at(uint32_t w, int pos, uint32_t s2, uint32_t z2) {
+  using T2 = typename Tr<T>::T2;
+  constexpr int MANT = Tr<T>::MANT, CAP = (MANT / BITS) * BITS;
+  const int sh = (pos / CAP) * CAP, p = pos - sh;
+  const uint32_t mask = (((1u << BITS) - 1u) << p) * 0x00010001u;
+  const uint32_t magic = ((uint32_t)(Tr<T>::EXP_BIAS + MANT - p) << MANT) * 0x00010001u;
+  const T2 c = __hsub2(as_t2<T2>(and_or(w >> sh, mask, magic)), as_t2<T2>(magic));  // exact
   return as_u32(__hfma2(c, as_t2<T2>(s2), as_t2<T2>(z2)));
 }
 

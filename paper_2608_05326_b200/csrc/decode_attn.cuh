@@ -170,8 +170,6 @@ template <class T, int D, int BITS>
 __device__ __forceinline__ void qk_q_tile(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
                                           int lane) {
   constexpr int KS = D / 16;
-  constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
-  constexpr uint32_t MG = Tr<T>::MAGIC;
   constexpr int KPV = (BITS == 4) ? 2 : 4;  // k-steps per code vector
   const int t = lane & 3;
 #pragma unroll
@@ -186,10 +184,10 @@ __device__ __forceinline__ void qk_q_tile(float (&s)[2][4], const uint32_t (&qa)
       for (int mt = 0; mt < 2; ++mt) {
         const uint32_t w = (BITS == 4) ? cw[kk * 2 + mt] : cw[kk];
         const int sh = (BITS == 4) ? 0 : mt * 8;
-        const uint32_t a0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
-        const uint32_t a1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
-        const uint32_t a2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
-        const uint32_t a3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
+        const uint32_t a0 = dequant_at<T, BITS>(w, sh + 0 * BITS, pr.x, pr.y);
+        const uint32_t a1 = dequant_at<T, BITS>(w, sh + 1 * BITS, pr.x, pr.y);
+        const uint32_t a2 = dequant_at<T, BITS>(w, sh + 2 * BITS, pr.z, pr.w);
+        const uint32_t a3 = dequant_at<T, BITS>(w, sh + 3 * BITS, pr.z, pr.w);
         mma16816<T>(s[mt], a0, a1, a2, a3, qa[ks][0], qa[ks][1]);
       }
     }
@@ -240,8 +238,6 @@ template <class T, int D, int BITS>
 __device__ __forceinline__ void qk_q_tile_rope(float (&s)[2][4], const uint32_t (&qa)[D / 16][2], uint32_t slot, uint32_t kp,
                                                uint32_t rslot, int lane) {
   constexpr int KS = D / 16;
-  constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
-  constexpr uint32_t MG = Tr<T>::MAGIC;
   constexpr int KPV = (BITS == 4) ? 2 : 4;  // k-steps per code vector
   const int t = lane & 3;
   uint32_t cw[KS / KPV][4];
@@ -254,10 +250,10 @@ __device__ __forceinline__ void qk_q_tile_rope(float (&s)[2][4], const uint32_t 
     const uint32_t w = (BITS == 4) ? cw[ks / KPV][(ks % KPV) * 2 + mt] : cw[ks / KPV][ks % KPV];
     const int sh = (BITS == 4) ? 0 : mt * 8;
     uint4 a;
-    a.x = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
-    a.y = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
-    a.z = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
-    a.w = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
+    a.x = dequant_at<T, BITS>(w, sh + 0 * BITS, pr.x, pr.y);
+    a.y = dequant_at<T, BITS>(w, sh + 1 * BITS, pr.x, pr.y);
+    a.z = dequant_at<T, BITS>(w, sh + 2 * BITS, pr.z, pr.w);
+    a.w = dequant_at<T, BITS>(w, sh + 3 * BITS, pr.z, pr.w);
     return a;
   };
 #pragma unroll
@@ -296,8 +292,6 @@ __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t 
                                           uint32_t slot, int lane) {
   constexpr int MT = D / 16;
   constexpr uint32_t VC_BYTES = 32 * D * BITS / 8;
-  constexpr uint32_t MASK = (BITS == 4) ? 0x000F000Fu : 0x00030003u;
-  constexpr uint32_t MG = Tr<T>::MAGIC;
   constexpr int IPV = (BITS == 4) ? 2 : 4;  // channel blocks (of 16) per code vector
   const int t = lane & 3;
   const uint32_t vp = slot + VC_BYTES;
@@ -319,10 +313,10 @@ __device__ __forceinline__ void pv_q_tile(float (&o)[D / 16][4], const uint32_t 
         const uint4 pr = ks ? pr1 : pr0;
         const uint32_t w = (BITS == 4) ? vw[ii * 2 + ks] : vw[ii];
         const int sh = (BITS == 4) ? 0 : ks * 8;
-        const uint32_t a0 = dequant2<T>(and_or(w >> (sh + 0 * BITS), MASK, MG), pr.x, pr.y);
-        const uint32_t a1 = dequant2<T>(and_or(w >> (sh + 1 * BITS), MASK, MG), pr.x, pr.y);
-        const uint32_t a2 = dequant2<T>(and_or(w >> (sh + 2 * BITS), MASK, MG), pr.z, pr.w);
-        const uint32_t a3 = dequant2<T>(and_or(w >> (sh + 3 * BITS), MASK, MG), pr.z, pr.w);
+        const uint32_t a0 = dequant_at<T, BITS>(w, sh + 0 * BITS, pr.x, pr.y);
+        const uint32_t a1 = dequant_at<T, BITS>(w, sh + 1 * BITS, pr.x, pr.y);
+        const uint32_t a2 = dequant_at<T, BITS>(w, sh + 2 * BITS, pr.z, pr.w);
+        const uint32_t a3 = dequant_at<T, BITS>(w, sh + 3 * BITS, pr.z, pr.w);
         mma16816<T>(o[i], a0, a1, a2, a3, pa[ks][0], pa[ks][1]);
         if (!PACK) mma16816<T>(o[i], a0, a1, a2, a3, pb[ks][0], pb[ks][1]);
       }
@@ -352,12 +346,20 @@ __device__ __forceinline__ uint32_t transpose8x8(uint32_t x) {
   return y;
 }
 
-// Online softmax update for one tile.  A lane owns heads 2t and 2t+1 (index 0 / 1 of m_run, l_run, wsum)
-// and tokens g, g+8, g+16, g+24 of the tile; the statistics of a head are replicated over the 8 lanes of
-// equal t.  Leaves the probability fragments for the PV product in pa / pb.
+// Online softmax update for one tile.  A lane owns heads 2t and 2t+1 (index 0 / 1 of m_run, l_part, wsum)
+// and tokens g, g+8, g+16, g+24 of the tile; the reference exponent m_run of a head is the same in the 8 lanes
+// of equal t, while l_part and wsum are the lane's own share of the sums (added over the 8 lanes by the caller,
+// once per window and once at the end).  m_run is a reference, not necessarily the maximum: a tile whose
+// logits stay below m_run + REF_SLACK keeps it (its probabilities are then at most 2^REF_SLACK, far inside
+// the range of every format they pass through), so the common tile costs no reduction over lanes and no
+// rescaling; only a tile that exceeds the slack moves the reference to the true maximum so far.
+// With PACK the query heads sit in columns 0..3 of the products and once more in columns 4..7, so lanes
+// t >= 2 see the same logits as lanes t - 2 and contribute the rounding residuals of the same probabilities.
+// Leaves the probability fragments for the PV product in pa / pb.
+constexpr float REF_SLACK = 8.f;
 template <class T, int MT, bool PACK>
 __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float scale_log2, int lane, float (&m_run)[2],
-                                             float (&l_run)[2], float (&wsum)[2], float (&o)[MT][4],
+                                             float (&l_part)[2], float (&wsum)[2], float (&o)[MT][4],
                                              uint32_t (&pa)[2][2], uint32_t (&pb)[2][2]) {
   const int g = lane >> 2;
   float x[2][2][2];  // [token block][row half][head]
@@ -378,43 +380,43 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
       }
     }
   }
-  float alpha[2], p[2][2][2];
+  float lm[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) lm[h] = fmaxf(fmaxf(x[0][0][h], x[0][1][h]), fmaxf(x[1][0][h], x[1][1][h]));
+  if (__any_sync(0xffffffffu, lm[0] > m_run[0] + REF_SLACK || lm[1] > m_run[1] + REF_SLACK)) {
+    float alpha[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float tmax = lm[h];
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+      const float m_new = fmaxf(m_run[h], tmax);  // finite: the caller guarantees ntok >= 1
+      alpha[h] = ex2(m_run[h] - m_new);
+      l_part[h] *= alpha[h];
+      wsum[h] *= alpha[h];
+      m_run[h] = m_new;
+    }
+    // the accumulators hold O^T with the lane's own two heads as its columns
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+      o[i][0] *= alpha[0]; o[i][1] *= alpha[1]; o[i][2] *= alpha[0]; o[i][3] *= alpha[1];
+    }
+  }
+  float p[2][2][2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    float tmax = fmaxf(fmaxf(x[0][0][h], x[0][1][h]), fmaxf(x[1][0][h], x[1][1][h]));
-    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
-    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
-    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
-    const float m_new = fmaxf(m_run[h], tmax);  // finite: the caller guarantees ntok >= 1
-    alpha[h] = ex2(m_run[h] - m_new);
     float rs = 0.f;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
-        p[mt][r][h] = ex2(x[mt][r][h] - m_new);
+        p[mt][r][h] = ex2(x[mt][r][h] - m_run[h]);
         rs += p[mt][r][h];
       }
     }
-    rs += __shfl_xor_sync(0xffffffffu, rs, 4);
-    rs += __shfl_xor_sync(0xffffffffu, rs, 8);
-    rs += __shfl_xor_sync(0xffffffffu, rs, 16);
-    l_run[h] = l_run[h] * alpha[h] + rs;
-    wsum[h] = wsum[h] * alpha[h] + rs;
-    m_run[h] = m_new;
-  }
-  if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
-    // the accumulators hold O^T with the lane's own two heads as its columns; with PACK the columns of
-    // lanes t >= 2 hold the residual products of heads 2(t-2), 2(t-2)+1
-    float a0 = alpha[0], a1 = alpha[1];
-    if (PACK) {
-      const float b0 = __shfl_sync(0xffffffffu, a0, (lane - 2) & 31), b1 = __shfl_sync(0xffffffffu, a1, (lane - 2) & 31);
-      if ((lane & 3) >= 2) { a0 = b0; a1 = b1; }
-    }
-#pragma unroll
-    for (int i = 0; i < MT; ++i) {
-      o[i][0] *= a0; o[i][1] *= a1; o[i][2] *= a0; o[i][3] *= a1;
-    }
+    l_part[h] += rs;
+    wsum[h] += rs;
   }
   // probabilities as (token, head) pairs -> 16-bit value + residual -> transposed into the B operand
   // (k = token, n = head): block (mt, r) becomes register r of k-step mt
@@ -425,16 +427,22 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
       uint32_t main, res;
       split_pair<T>(p[mt][r][0], p[mt][r][1], main, res);
       if (PACK) {
-        // heads live in columns 0..3; columns 4..7 carry the residuals of heads 0..3 in the same product
-        const uint32_t left = __shfl_sync(0xffffffffu, res, (lane - 2) & 31);
-        if ((lane & 3) >= 2) main = left;
-        pa[mt][r] = transpose8x8(main);
+        // columns 0..3 carry the probabilities, columns 4..7 their residuals, in the same product
+        pa[mt][r] = transpose8x8((lane & 3) >= 2 ? res : main);
       } else {
         pa[mt][r] = transpose8x8(main);
         pb[mt][r] = transpose8x8(res);
       }
     }
   }
+}
+
+// sum over the 8 lanes of equal lane % 4
+__device__ __forceinline__ float sum_over_g(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 4);
+  v += __shfl_xor_sync(0xffffffffu, v, 8);
+  v += __shfl_xor_sync(0xffffffffu, v, 16);
+  return v;
 }
 
 template <class T, int D, int BITS, int GROUP, int TILES, bool PACK, bool ROPE>
@@ -536,13 +544,15 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_k
 #pragma unroll 1
   for (int i = 0; i < NSLOT; ++i) issue_next();
 
-  // query fragments: row g of the A operand = head hk*G + g (rows >= G are zero)
+  // query fragments: column g of the B operand = head hk*G + g (columns >= G are zero)
   uint32_t qa[KS][2];
   {
-    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)ul * p.Hq + (size_t)hk * p.G + g) * D;
+    // with PACK (at most 4 heads per KV head) the heads fill columns 0..3 and, again, columns 4..7
+    const int gh = PACK ? (g & 3) : g;
+    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)ul * p.Hq + (size_t)hk * p.G + gh) * D;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      if (g < p.G) {
+      if (gh < p.G) {
         qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * t);
         qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * t);
       } else {
@@ -596,6 +606,8 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_k
         if (ROPE) release();
       }
     }
+    wsum[0] = sum_over_g(wsum[0]);
+    wsum[1] = sum_over_g(wsum[1]);
     if (g == 0) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -613,6 +625,8 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_k
   constexpr int OSTR = D + 4;
   float* my_o = reinterpret_cast<float*>(smem + wid * NSLOT * TT::SLOT_BYTES);
   float* my_ml = my_o + 8 * OSTR;
+  l_run[0] = sum_over_g(l_run[0]);
+  l_run[1] = sum_over_g(l_run[1]);
   if (g == 0) { my_ml[2 * t] = m_run[0]; my_ml[2 * t + 1] = m_run[1]; my_ml[8 + 2 * t] = l_run[0]; my_ml[8 + 2 * t + 1] = l_run[1]; }
 #pragma unroll
   for (int i = 0; i < MT; ++i) {
