@@ -26,10 +26,19 @@
  *     enqueue work unless the comment says "synchronises".
  *   - A "unit" is one (layer, sequence) pair; unit = layer * batch + sequence.  `layer == -1` means
  *     every layer in one launch; tensors then carry a leading [n_layers] dimension.
- *   - Errors are returned as qevict_status; a failed call enqueues nothing.  Kernels never trap:
- *     device-side checks record a code that the synchronising getters report as
+ *   - Errors are returned as qevict_status; a call refused for its arguments or its place in the call order
+ *     enqueues nothing.  If a CUDA launch fails after an earlier kernel of the same call has been enqueued,
+ *     the cache is marked broken and every later compute call on it returns QEVICT_ERR_BAD_STATE.  Kernels
+ *     never trap: device-side checks record a code that qevict_get_stats reports as
  *     QEVICT_ERR_DEVICE_CHECK.
- *   - The library holds no global state; one handle must not be used from two threads at once.
+ *   - Every call makes the cache's device current while it runs and puts the caller's current device back
+ *     before it returns.
+ *   - Process-wide state is limited to three things, none of which a caller can observe through results:
+ *     the text qevict_last_error(NULL) returns (per thread: the last failure of qevict_create or
+ *     qevict_workspace_bytes, which have no handle to keep it in); the per-device record of the
+ *     shared-memory limits already granted to the kernels (only ever raised); and the built-in scratch
+ *     array of qevict_decode_attn_noalloc with its per-device address.  One handle must not be used from
+ *     two threads at once; different handles may be.
  *   - There is no CPU fallback: without a CUDA device every compute call returns QEVICT_ERR_CUDA.
  */
 #ifndef QEVICT_H_
@@ -143,7 +152,11 @@ typedef struct {
 QEVICT_API qevict_status qevict_budget_from_bytes(const qevict_config* cfg, uint64_t hist_bytes, double q_frac,
                                        int32_t* k_f, int32_t* k_q, uint64_t* m_f, uint64_t* m_q);
 
-/* Size of the device buffer qevict_create needs for this configuration (pools, tables, scratch). */
+/* Size of the device buffer qevict_create needs for this configuration (pools, tables, scratch).
+ * QEVICT_ERR_UNSUPPORTED for shapes the kernels are not built for: head_dim other than 64 / 128, window other
+ * than 32 / 64, more than 8 query heads per KV head, more than 8192 windows per sequence, budgets whose decode
+ * work list (K_f + K_q + protected windows + waiting windows + 1) exceeds 8192 entries, routing tables that do
+ * not fit the shared memory of an SM; qevict_last_error(NULL) says which. */
 QEVICT_API qevict_status qevict_workspace_bytes(const qevict_config* cfg, uint64_t* bytes);
 
 /* Build a cache inside `device_mem` (device pointer, 256-byte aligned, `bytes` long, owned by the
@@ -230,10 +243,16 @@ QEVICT_API qevict_status qevict_decode_attn_host_async(qevict_handle h, int32_t 
  * or freed by the call (no cudaMalloc / cudaFree, no allocating library routine).
  *
  * Arguments, results and state changes are those of qevict_decode_attn.  Differences:
- *   - A call whose scratch (partials for all units up to the last unit of the call) does not fit the
- *     array returns QEVICT_ERR_NO_MEMORY and enqueues nothing; qevict_last_error states the size needed.
+ *   - A call whose scratch (the partials of the units of THIS call: one layer's sequences, or all of them
+ *     with layer == -1) does not fit the array returns QEVICT_ERR_NO_MEMORY and enqueues nothing;
+ *     qevict_last_error states the size needed.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) before it
- *     launches anything.  Make that first call before any stream capture begins.
+ *     launches anything.  Where the CUDA runtime loads modules lazily, that look-up is also the moment the
+ *     runtime places the library's device image -- the array included -- in device memory, so the first
+ *     call can fail with an out-of-memory error on a device whose memory has already been handed out in
+ *     full: make it once at start-up, before the memory plan is committed and before any stream capture
+ *     begins.  Later calls allocate nothing.
+ *   - qevict_set_kernel_timing does not cover this entry point (its launches are not bracketed by events).
  *   - All calls, on all handles and streams of a device, share the one array, which keeps the last
  *     call's contents.  Nothing in it has to start at zero -- every slot a call reads it has written
  *     first -- but two calls that overlap on the GPU race on it: keep them in one stream, or order them
@@ -281,6 +300,63 @@ QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, in
 QEVICT_API qevict_status qevict_export_event_mass(qevict_handle h, int32_t layer, int32_t seq, float* event_mass,
                                                   void* stream);
 
+/* Snapshot and restore of one unit [Migration-Stable Quantization: the ledger is a persistent low-bit store;
+ * codes written at a window's first demotion stay valid for the window's whole life, so a cache can be put
+ * away and brought back without requantizing anything].  A snapshot holds what the kernels read for one
+ * (layer, sequence) pair -- window tables, page-owner tables, decode work list, the unit's pages of both pools
+ * and the host's bookkeeping for the layer -- and restores into any cache created with the same
+ * configuration, after which decode steps and routing events continue bit for bit as they would have.
+ *
+ * All arrays are HOST memory owned by the caller, sized by qevict_state_layout_of:
+ *   tier, ledger uint8 [n_window_slots]; fp_page, q_page int32 [n_window_slots] (-1 = none); importance,
+ *   event_mass float32 [n_window_slots]; fp_owner int32 [n_fp_pages], q_owner int32 [n_q_pages] (window that
+ *   holds the page, -1 = free); entries uint32 [n_entries][2] ({window | kind << 28, page}; kind 0 full
+ *   precision, 1 quantized, 2 open window); last_mass float32 [n_entries] (mass of the last decode step per
+ *   work-list entry); fp_pool [fp_pool_bytes], q_pool [q_pool_bytes]: the unit's pages in the library's own
+ *   page layout (opaque; use qevict_export_fp_page / qevict_export_q_page for plain layouts).
+ * qevict_export_state synchronises the device, fills the scalars and the arrays.  qevict_import_state checks
+ * every index in the snapshot against the configuration (a snapshot that fails a check changes nothing),
+ * synchronises the device and overwrites the unit.  The sequences of a layer step together, so the layer's
+ * bookkeeping (windows, fill of the open window, filled windows waiting for a routing event) is taken from the
+ * first snapshot imported into a layer that has not been prefilled, and every later import into that layer
+ * must agree with it (QEVICT_ERR_BAD_STATE otherwise); import every sequence of a layer before using it. */
+typedef struct {
+  int32_t n_window_slots;  /* max_context / W */
+  int32_t n_fp_pages;      /* full-precision pages per unit */
+  int32_t n_q_pages;       /* quantized pages per unit */
+  int32_t n_entries;       /* capacity of the decode work list */
+  uint64_t fp_pool_bytes;  /* n_fp_pages * bytes of a full-precision page */
+  uint64_t q_pool_bytes;   /* n_q_pages * bytes of a quantized page */
+} qevict_state_layout;
+
+typedef struct {
+  uint32_t struct_size;    /* sizeof(qevict_state_view) of the caller */
+  int32_t n_windows;       /* windows created so far */
+  int32_t open_window;     /* index of the window being filled, -1 if none */
+  int32_t open_fill;       /* tokens in it */
+  int32_t n_live;          /* entries of the decode work list */
+  int32_t layer_prefilled, layer_has_open, layer_open_fill, layer_n_windows, layer_aged; /* host bookkeeping of the layer */
+  float knorm_acc;         /* key-norm ranking: running sum of the open window */
+  uint64_t counters[4];    /* promotions, quantizations, reactivations, deletions of the unit */
+  uint64_t decode_steps;   /* of the handle */
+  uint8_t* tier;
+  uint8_t* ledger;
+  int32_t* fp_page;
+  int32_t* q_page;
+  float* importance;
+  float* event_mass;
+  int32_t* fp_owner;
+  int32_t* q_owner;
+  uint32_t* entries;
+  float* last_mass;
+  void* fp_pool;
+  void* q_pool;
+} qevict_state_view;
+
+QEVICT_API qevict_status qevict_state_layout_of(qevict_handle h, qevict_state_layout* out);
+QEVICT_API qevict_status qevict_export_state(qevict_handle h, int32_t layer, int32_t seq, qevict_state_view* view);
+QEVICT_API qevict_status qevict_import_state(qevict_handle h, int32_t layer, int32_t seq, const qevict_state_view* view);
+
 /* Tuning: force the number of KV splits per (unit, KV head) of the decode kernel (1..64); 0 restores
  * the built-in choice, which fills the GPU in whole waves.  Results do not depend on it beyond
  * floating-point summation order. */
@@ -311,7 +387,8 @@ QEVICT_API qevict_status qevict_kernel_timeline(qevict_handle h, int32_t max_rec
 /* Number of kernels this handle has launched since creation (host counter). */
 QEVICT_API uint64_t qevict_launch_count(qevict_handle h);
 
-/* Text of the last error on this handle (never NULL). */
+/* Text of the last error on this handle (never NULL).  With h == NULL: the calling thread's last failure of
+ * qevict_create or qevict_workspace_bytes. */
 QEVICT_API const char* qevict_last_error(qevict_handle h);
 QEVICT_API const char* qevict_status_string(qevict_status s);
 /* Library version, "major.minor". */

@@ -48,6 +48,23 @@ class qevict_stats(C.Structure):
         "n_evicted", "decode_steps", "n_sink")]
 
 
+class qevict_state_layout(C.Structure):
+    _fields_ = [("n_window_slots", C.c_int32), ("n_fp_pages", C.c_int32), ("n_q_pages", C.c_int32), ("n_entries", C.c_int32),
+                ("fp_pool_bytes", C.c_uint64), ("q_pool_bytes", C.c_uint64)]
+
+
+_STATE_SCALARS = ("n_windows", "open_window", "open_fill", "n_live", "layer_prefilled", "layer_has_open", "layer_open_fill",
+                  "layer_n_windows", "layer_aged")
+_STATE_ARRAYS = ("tier", "ledger", "fp_page", "q_page", "importance", "event_mass", "fp_owner", "q_owner", "entries",
+                 "last_mass", "fp_pool", "q_pool")
+
+
+class qevict_state_view(C.Structure):
+    _fields_ = ([("struct_size", C.c_uint32)] + [(n, C.c_int32) for n in _STATE_SCALARS] +
+                [("knorm_acc", C.c_float), ("counters", C.c_uint64 * 4), ("decode_steps", C.c_uint64)] +
+                [(n, C.c_void_p) for n in _STATE_ARRAYS])
+
+
 _lib = None
 
 _SIGNATURES = {
@@ -76,6 +93,9 @@ _SIGNATURES = {
     "qevict_decode_attn_host_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_rebalance": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
+    "qevict_state_layout_of": (C.c_int, [C.c_void_p, C.POINTER(qevict_state_layout)]),
+    "qevict_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(qevict_state_view)]),
+    "qevict_import_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(qevict_state_view)]),
     "qevict_get_stats": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(qevict_stats)]),
     "qevict_export_tables": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 7),
     "qevict_export_last_mass": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
@@ -102,7 +122,8 @@ def lib():
 
 def _check(status, handle=None):
     if status != QEVICT_OK:
-        msg = lib().qevict_last_error(handle).decode() if handle else lib().qevict_status_string(status).decode()
+        # without a handle: the calling thread's last failure of qevict_create / qevict_workspace_bytes
+        msg = lib().qevict_last_error(handle).decode()
         raise QEvictError(status, msg or lib().qevict_status_string(status).decode())
 
 
@@ -180,6 +201,62 @@ def qevict_decode_attn_noalloc(h, layer, q, k_new, v_new, out, stream=None):
 
 def qevict_rebalance(h, layer, stream=None):
     _check(lib().qevict_rebalance(h, layer, _stream(stream)), h)
+
+
+def qevict_state_layout_of(h):
+    lay = qevict_state_layout()
+    _check(lib().qevict_state_layout_of(h, C.byref(lay)), h)
+    return lay
+
+
+def _state_buffers(lay):
+    """Host tensors of a snapshot, sized by the layout."""
+    nw, i32, f32, u8 = lay.n_window_slots, torch.int32, torch.float32, torch.uint8
+    return {
+        "tier": torch.zeros(nw, dtype=u8), "ledger": torch.zeros(nw, dtype=u8),
+        "fp_page": torch.zeros(nw, dtype=i32), "q_page": torch.zeros(nw, dtype=i32),
+        "importance": torch.zeros(nw, dtype=f32), "event_mass": torch.zeros(nw, dtype=f32),
+        "fp_owner": torch.zeros(lay.n_fp_pages, dtype=i32), "q_owner": torch.zeros(lay.n_q_pages, dtype=i32),
+        "entries": torch.zeros((lay.n_entries, 2), dtype=i32), "last_mass": torch.zeros(lay.n_entries, dtype=f32),
+        "fp_pool": torch.zeros(lay.fp_pool_bytes, dtype=u8), "q_pool": torch.zeros(lay.q_pool_bytes, dtype=u8),
+    }
+
+
+def _state_view(arrays):
+    view = qevict_state_view()
+    view.struct_size = C.sizeof(qevict_state_view)
+    for n in _STATE_ARRAYS:
+        t = arrays[n]
+        assert not t.is_cuda and t.is_contiguous()
+        setattr(view, n, t.data_ptr())
+    return view
+
+
+def qevict_export_state(h, layer, seq):
+    """Snapshot of one unit: a dict of host tensors (tables, owner tables, work list, the unit's pages of both pools
+    in the library's page layout) and scalars.  Synchronises."""
+    arrays = _state_buffers(qevict_state_layout_of(h))
+    view = _state_view(arrays)
+    _check(lib().qevict_export_state(h, layer, seq, C.byref(view)), h)
+    state = dict(arrays)
+    for n in _STATE_SCALARS:
+        state[n] = int(getattr(view, n))
+    state["knorm_acc"] = float(view.knorm_acc)
+    state["counters"] = [int(x) for x in view.counters]
+    state["decode_steps"] = int(view.decode_steps)
+    return state
+
+
+def qevict_import_state(h, layer, seq, state):
+    """Restores a unit from a snapshot made by qevict_export_state on a cache of the same configuration."""
+    view = _state_view(state)
+    for n in _STATE_SCALARS:
+        setattr(view, n, int(state[n]))
+    view.knorm_acc = float(state["knorm_acc"])
+    for i in range(4):
+        view.counters[i] = int(state["counters"][i])
+    view.decode_steps = int(state["decode_steps"])
+    _check(lib().qevict_import_state(h, layer, seq, C.byref(view)), h)
 
 
 def qevict_set_splits(h, splits):
@@ -311,6 +388,12 @@ class QEvictCache:
         return qevict_launch_count(self.handle)
 
     # -- exports (parity checks, snapshots) -------------------------------------------------------
+    def export_state(self, layer, seq):
+        return qevict_export_state(self.handle, layer, seq)
+
+    def import_state(self, layer, seq, state):
+        qevict_import_state(self.handle, layer, seq, state)
+
     def export_tables(self, layer, seq):
         n = self.max_windows
         dev = self.device

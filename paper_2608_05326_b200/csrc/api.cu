@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -26,8 +27,13 @@ int next_pow2(int x) {
 
 namespace {
 
+// Text of the last failure of a call that has no handle to keep it in (qevict_create, qevict_workspace_bytes),
+// per calling thread; qevict_last_error(NULL) returns it.
+thread_local std::string t_create_error;
+
 qevict_status fail(qevict_handle h, qevict_status s, const std::string& msg) {
   if (h) h->last_error = msg;
+  else t_create_error = msg;
   return s;
 }
 
@@ -90,6 +96,17 @@ const char* unsupported(const qevict_config* c) {
   if (c->quant_bits != 2 && c->quant_bits != 4) return "quant_bits must be 2 or 4";
   if (c->group_size != 32 && c->group_size != 64) return "group_size must be 32 or 64";
   if (c->max_context / c->window > 8192) return "more than 8192 windows per sequence";
+  {
+    // the attention kernel keeps a warp's work-list entries one per lane and runs at most MAX_SPLITS splits of
+    // DECODE_WARPS warps per (unit, KV head): longer work lists cannot be walked
+    const int r = c->rebalance_interval_hint > 0 ? c->rebalance_interval_hint : c->window;
+    const long long emax = (long long)c->fp_budget_windows + c->q_budget_windows + c->sink_windows + c->recent_windows +
+                           (r + c->window - 1) / c->window + 2;
+    if (emax > 32LL * DECODE_WARPS * MAX_SPLITS)
+      return "fp_budget_windows + q_budget_windows + protected windows exceed the 8192 work-list entries per sequence the attention kernel walks";
+  }
+  if (c->rank_mode == QEVICT_RANK_KEYNORM && (long long)c->n_kv_heads * c->head_dim > 4096)
+    return "key-norm ranking supports n_kv_heads * head_dim <= 4096";
   return nullptr;
 }
 
@@ -206,12 +223,36 @@ KernelArgs make_args(qevict_handle h, int l0, int l1) {
 
 }  // namespace
 
+const char* qevict::decode_precheck(const qevict_ctx* h, int layer, const void* q, const void* k_new, const void* v_new,
+                                    const void* out, int* l0, int* l1, qevict_status* st) {
+  const Geometry& g = h->geo;
+  *st = QEVICT_ERR_INVALID_ARG;
+  if (layer == -1) { *l0 = 0; *l1 = g.n_layers; }
+  else if (layer >= 0 && layer < g.n_layers) { *l0 = layer; *l1 = layer + 1; }
+  else return "layer out of range";
+  if (!q || !out) return "q and out must not be NULL";
+  if ((k_new == nullptr) != (v_new == nullptr)) return "k_new and v_new must both be given or both be NULL";
+  *st = QEVICT_ERR_BAD_STATE;
+  if (h->broken) return "an earlier call failed after it had started to enqueue work: destroy this cache";
+  for (int l = *l0; l < *l1; ++l) {
+    const LayerMirror& m = h->layers[l];
+    if (!m.prefilled) return "decode before prefill_assign";
+    if (k_new && !m.has_open) {
+      if (m.aged > g.aged_cap) return "too many filled windows are waiting: call qevict_rebalance";
+      if (m.n_windows + 1 > g.NW) return "context would exceed max_context";
+    }
+  }
+  *st = QEVICT_OK;
+  return nullptr;
+}
+
 // Splits per (unit, KV head): enough CTAs to fill the GPU in whole waves while every warp still walks
 // several windows.
 int qevict::choose_splits(const qevict_ctx* h, int n_units) {
   const Geometry& g = h->geo;
   // a warp holds its work-list entries one per lane: at most 32 entries per warp
-  const int smin = (g.EMAX + 32 * DECODE_WARPS - 1) / (32 * DECODE_WARPS);
+  int smin = (g.EMAX + 32 * DECODE_WARPS - 1) / (32 * DECODE_WARPS);
+  if (smin > MAX_SPLITS) smin = MAX_SPLITS;  // (configurations that would need more are refused at create)
   if (h->forced_splits > 0) {
     const int f = h->forced_splits < smin ? smin : h->forced_splits;
     return f < MAX_SPLITS ? f : MAX_SPLITS;
@@ -235,6 +276,21 @@ int qevict::choose_splits(const qevict_ctx* h, int n_units) {
 
 namespace {
 
+#define QE_DEVICE(h)                        \
+  DeviceGuard qe_device_guard((h)->cfg.device); \
+  QE_CUDA(h, qe_device_guard.err)
+
+// the same for a launch that follows one that has already been enqueued in this call: a failure here leaves the
+// device tables ahead of (or behind) the host's mirror, so the cache refuses every later call
+#define QE_CUDA_MID(h, expr)                                                              \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess) {                                                             \
+      (h)->broken = true;                                                                 \
+      return fail(h, QEVICT_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+    }                                                                                     \
+  } while (0)
+
 #define QE_CUDA(h, expr)                                                                  \
   do {                                                                                    \
     cudaError_t e__ = (expr);                                                             \
@@ -244,19 +300,10 @@ namespace {
 qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                           cudaStream_t stream) {
   int l0, l1;
-  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
-  if (!q || !out) return fail(h, QEVICT_ERR_INVALID_ARG, "q and out must not be NULL");
-  if ((k_new == nullptr) != (v_new == nullptr)) return fail(h, QEVICT_ERR_INVALID_ARG, "k_new and v_new must both be given or both be NULL");
+  qevict_status pst;
+  if (const char* msg = decode_precheck(h, layer, q, k_new, v_new, out, &l0, &l1, &pst)) return fail(h, pst, msg);
   const Geometry& g = h->geo;
-  for (int l = l0; l < l1; ++l) {
-    const LayerMirror& m = h->layers[l];
-    if (!m.prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "decode before prefill_assign");
-    if (k_new && !m.has_open) {
-      if (m.aged > g.aged_cap) return fail(h, QEVICT_ERR_BAD_STATE, "too many filled windows are waiting: call qevict_rebalance");
-      if (m.n_windows + 1 > g.NW) return fail(h, QEVICT_ERR_BAD_STATE, "context would exceed max_context");
-    }
-  }
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   const KernelArgs a = make_args(h, l0, l1);
   if (k_new) {
     QE_CUDA(h, timed_launch(h, 0, stream, [&] { return launch_append(a, k_new, v_new, stream); }));
@@ -282,8 +329,9 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
 #ifdef QEVICT_TRACE
   p.trace = a.trace;
 #endif
-  QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
-  QE_CUDA(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
+  if (k_new) QE_CUDA_MID(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
+  else QE_CUDA(h, timed_launch(h, 1, stream, [&] { return h->decode_fn(p, a.n_units, stream); }));
+  QE_CUDA_MID(h, timed_launch(h, 2, stream, [&] { return launch_combine(a, p.S, e_bound, out, stream); }));
   h->decode_steps++;
   return QEVICT_OK;
 }
@@ -307,7 +355,7 @@ QEVICT_API const char* qevict_status_string(qevict_status s) {
   return "unknown status";
 }
 
-QEVICT_API const char* qevict_last_error(qevict_handle h) { return h ? h->last_error.c_str() : "handle is NULL"; }
+QEVICT_API const char* qevict_last_error(qevict_handle h) { return h ? h->last_error.c_str() : t_create_error.c_str(); }
 
 QEVICT_API uint64_t qevict_launch_count(qevict_handle h) { return h ? h->launches : 0; }
 
@@ -327,39 +375,60 @@ QEVICT_API qevict_status qevict_budget_from_bytes(const qevict_config* cfg, uint
   return QEVICT_OK;
 }
 
+// Shapes the kernels cannot run with although every single field is in range; nullptr if fine.
+static const char* unsupported_geometry(const Geometry& g) {
+  // the routing kernel keeps one unit's candidate tables in shared memory (227 KB per CTA on this architecture)
+  if (route_smem_bytes(g, next_pow2(g.NW)) > 227u * 1024u)
+    return "the routing tables of one sequence (max_context / window windows, the budgets' pages) exceed the shared memory of an SM";
+  return nullptr;
+}
+
 QEVICT_API qevict_status qevict_workspace_bytes(const qevict_config* cfg, uint64_t* bytes) {
-  if (!bytes) return QEVICT_ERR_INVALID_ARG;
-  if (validate(cfg)) return QEVICT_ERR_INVALID_ARG;
-  if (unsupported(cfg)) return QEVICT_ERR_UNSUPPORTED;
+  if (!bytes) return fail(nullptr, QEVICT_ERR_INVALID_ARG, "bytes is NULL");
+  if (const char* m = validate(cfg)) return fail(nullptr, QEVICT_ERR_INVALID_ARG, m);
+  if (const char* m = unsupported(cfg)) return fail(nullptr, QEVICT_ERR_UNSUPPORTED, m);
   Geometry g;
   make_geometry(*cfg, g);
+  if (const char* m = unsupported_geometry(g)) return fail(nullptr, QEVICT_ERR_UNSUPPORTED, m);
   *bytes = carve(g, nullptr, nullptr, nullptr);
   return QEVICT_OK;
 }
 
 QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_mem, uint64_t bytes, qevict_handle* out) {
-  if (!out) return QEVICT_ERR_INVALID_ARG;
+  if (!out) return fail(nullptr, QEVICT_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
-  if (validate(cfg)) return QEVICT_ERR_INVALID_ARG;
-  if (unsupported(cfg)) return QEVICT_ERR_UNSUPPORTED;
-  if (!device_mem || ((uintptr_t)device_mem & 255)) return QEVICT_ERR_INVALID_ARG;
+  if (const char* m = validate(cfg)) return fail(nullptr, QEVICT_ERR_INVALID_ARG, m);
+  if (const char* m = unsupported(cfg)) return fail(nullptr, QEVICT_ERR_UNSUPPORTED, m);
+  {
+    Geometry g0;
+    make_geometry(*cfg, g0);
+    if (const char* m = unsupported_geometry(g0)) return fail(nullptr, QEVICT_ERR_UNSUPPORTED, m);
+  }
+  if (!device_mem || ((uintptr_t)device_mem & 255)) return fail(nullptr, QEVICT_ERR_INVALID_ARG, "device_mem must be a 256-byte aligned device pointer");
   qevict_ctx* h = new (std::nothrow) qevict_ctx();
-  if (!h) return QEVICT_ERR_NO_MEMORY;
+  if (!h) return fail(nullptr, QEVICT_ERR_NO_MEMORY, "host allocation failed");
   h->cfg = *cfg;
   make_geometry(*cfg, h->geo);
   const Geometry& g = h->geo;
   const size_t need = carve(g, (char*)device_mem, &h->st, h);
-  if (need > bytes) { delete h; return QEVICT_ERR_NO_MEMORY; }
+  if (need > bytes) {
+    delete h;
+    return fail(nullptr, QEVICT_ERR_NO_MEMORY, "device_mem is smaller than qevict_workspace_bytes");
+  }
   switch ((g.dtype == QEVICT_DTYPE_BF16 ? 2 : 0) + (g.D == 128 ? 1 : 0)) {
     case 0: h->decode_fn = decode_dispatch_h64(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
     case 1: h->decode_fn = decode_dispatch_h128(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
     case 2: h->decode_fn = decode_dispatch_b64(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
     default: h->decode_fn = decode_dispatch_b128(g.bits, g.group, g.tiles, g.G, g.rope_base > 0.f); break;
   }
-  if (!h->decode_fn) { delete h; return QEVICT_ERR_UNSUPPORTED; }
+  if (!h->decode_fn) {
+    delete h;
+    return fail(nullptr, QEVICT_ERR_UNSUPPORTED, "no attention kernel is built for this combination of quant_bits, group_size and window");
+  }
   h->layers.resize(g.n_layers);
   h->mig_epoch.assign(g.n_layers, 0u);
-  cudaError_t e = cudaSetDevice(cfg->device);
+  DeviceGuard guard(cfg->device);
+  cudaError_t e = guard.err;
   if (e == cudaSuccess) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) h->sm_count = sms;
@@ -392,7 +461,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
   }
   if (e != cudaSuccess) {
     delete h;
-    return QEVICT_ERR_CUDA;
+    return fail(nullptr, QEVICT_ERR_CUDA, std::string("set-up on the device failed: ") + cudaGetErrorString(e));
   }
   *out = h;
   return QEVICT_OK;
@@ -416,7 +485,7 @@ QEVICT_API qevict_status qevict_kernel_timeline(qevict_handle h, int32_t max_rec
   if (!h || !kernel || !start_us || !end_us || !n_records || max_records < 0) return QEVICT_ERR_INVALID_ARG;
   *n_records = 0;
 #ifdef QEVICT_TRACE
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   QE_CUDA(h, cudaDeviceSynchronize());
   const uint32_t calls = h->trace_calls;
   std::vector<unsigned long long> buf(calls * TRACE_CALL_WORDS);
@@ -493,7 +562,7 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
   if (ctx_tokens > h->cfg.max_context) return fail(h, QEVICT_ERR_INVALID_ARG, "ctx_tokens exceeds max_context");
   for (int l = l0; l < l1; ++l)
     if (h->layers[l].prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "prefill_assign called twice for a layer");
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   cudaStream_t s = (cudaStream_t)stream;
   const KernelArgs a = make_args(h, l0, l1);
   const int n_prompt = ctx_tokens / g.W;
@@ -502,9 +571,9 @@ QEVICT_API qevict_status qevict_prefill_assign(qevict_handle h, int32_t layer, c
     QE_CUDA(h, launch_key_norm_scores(a, k, ctx_tokens, n_prompt, s));
     h->launches++;
   }
-  QE_CUDA(h, launch_route(a, 1, next_pow2(n_prompt), s));
-  QE_CUDA(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kfp, s));
-  QE_CUDA(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));
+  QE_CUDA_MID(h, launch_route(a, 1, next_pow2(n_prompt), s));
+  QE_CUDA_MID(h, launch_copy_prompt(a, k, v, ctx_tokens, g.Kfp, s));
+  QE_CUDA_MID(h, launch_migrate(a, k, v, ctx_tokens, g.Kq, s));
   ++h->mig_epoch[l0];  // the next event of these units counts its queue in the other counter
   h->launches += 2 + (g.Kfp > 0) + (g.Kq > 0);
   for (int l = l0; l < l1; ++l) {
@@ -524,14 +593,14 @@ static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void
                                       const void* v_new_host, void* out_host, void* stream, bool sync) {
   if (!h) return QEVICT_ERR_INVALID_ARG;
   int l0, l1;
-  if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
-  if (!q_host || !out_host) return fail(h, QEVICT_ERR_INVALID_ARG, "q_host and out_host must not be NULL");
-  if ((k_new_host == nullptr) != (v_new_host == nullptr)) return fail(h, QEVICT_ERR_INVALID_ARG, "k_new and v_new must both be given or both be NULL");
+  qevict_status pst;
+  // every argument and call-order check comes before the first copy: a refused call enqueues nothing
+  if (const char* msg = decode_precheck(h, layer, q_host, k_new_host, v_new_host, out_host, &l0, &l1, &pst)) return fail(h, pst, msg);
   const Geometry& g = h->geo;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t nu = (size_t)(l1 - l0) * g.batch;
   const size_t qb = nu * g.Hq * g.D * 2, kb = nu * g.Hkv * g.D * 2;
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   // Page-locked host buffers that the device can address are used in place where each byte is touched once:
   // the append kernel reads the new token from them and the merge kernel writes `out` into them, which saves
   // three copy operations (and their hand-overs between the copy engines and the SMs) per step.  The queries
@@ -578,10 +647,11 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   if (!h) return QEVICT_ERR_INVALID_ARG;
   int l0, l1;
   if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
+  if (h->broken) return fail(h, QEVICT_ERR_BAD_STATE, "an earlier call failed after it had started to enqueue work: destroy this cache");
   for (int l = l0; l < l1; ++l)
     if (!h->layers[l].prefilled) return fail(h, QEVICT_ERR_BAD_STATE, "rebalance before prefill_assign");
   const Geometry& g = h->geo;
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   cudaStream_t s = (cudaStream_t)stream;
   const KernelArgs a = make_args(h, l0, l1);
   QE_CUDA(h, timed_launch(h, 3, s, [&] { return launch_route(a, 0, next_pow2(g.Kfp + g.Kq + g.aged_cap + 1), s); }));
@@ -589,7 +659,7 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
   const int max_promote = g.Kf < g.Kq ? g.Kf : g.Kq;
   const int max_items = (g.Kq > 0 ? g.PF : 0) + max_promote;
   if (max_items > 0) {
-    QE_CUDA(h, timed_launch(h, 4, s, [&] { return launch_migrate(a, nullptr, nullptr, 0, max_items, s); }));
+    QE_CUDA_MID(h, timed_launch(h, 4, s, [&] { return launch_migrate(a, nullptr, nullptr, 0, max_items, s); }));
     ++h->mig_epoch[l0];  // the next event of these units counts its queue in the other counter
   }
   for (int l = l0; l < l1; ++l) h->layers[l].aged = 0;
@@ -601,7 +671,7 @@ QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict
   int l0, l1;
   if (!layer_range(h, layer, &l0, &l1)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer out of range");
   const Geometry& g = h->geo;
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   QE_CUDA(h, cudaDeviceSynchronize());
   memset(out, 0, sizeof(*out));
   const size_t u0 = (size_t)l0 * g.batch, nu = (size_t)(l1 - l0) * g.batch;
@@ -649,7 +719,7 @@ QEVICT_API qevict_status qevict_export_tables(qevict_handle h, int32_t layer, in
   const Geometry& g = h->geo;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t o = (size_t)u * g.NW;
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   if (n_windows) QE_CUDA(h, cudaMemcpyAsync(n_windows, h->st.n_windows + u, 4, cudaMemcpyDeviceToDevice, s));
   if (tier) QE_CUDA(h, cudaMemcpyAsync(tier, h->st.tier + o, g.NW, cudaMemcpyDeviceToDevice, s));
   if (ledger) QE_CUDA(h, cudaMemcpyAsync(ledger, h->st.ledger + o, g.NW, cudaMemcpyDeviceToDevice, s));
@@ -663,7 +733,7 @@ QEVICT_API qevict_status qevict_export_event_mass(qevict_handle h, int32_t layer
   if (!h || !event_mass) return QEVICT_ERR_INVALID_ARG;
   int u;
   if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   QE_CUDA(h, cudaMemcpyAsync(event_mass, h->st.event_mass + (size_t)u * h->geo.NW, (size_t)h->geo.NW * 4,
                              cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return QEVICT_OK;
@@ -673,7 +743,7 @@ QEVICT_API qevict_status qevict_export_last_mass(qevict_handle h, int32_t layer,
   if (!h || !mass) return QEVICT_ERR_INVALID_ARG;
   int u;
   if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   const KernelArgs a = make_args(h, 0, h->geo.n_layers);
   QE_CUDA(h, launch_export_mass(a, u, mass, (cudaStream_t)stream));
   h->launches++;
@@ -686,7 +756,7 @@ QEVICT_API qevict_status qevict_export_fp_page(qevict_handle h, int32_t layer, i
   int u;
   if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
   if (fp_page < 0 || fp_page >= h->geo.PF) return fail(h, QEVICT_ERR_INVALID_ARG, "fp_page out of range");
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   const KernelArgs a = make_args(h, 0, h->geo.n_layers);
   QE_CUDA(h, launch_export_fp_page(a, u, fp_page, k_out, v_out, (cudaStream_t)stream));
   h->launches++;
@@ -699,7 +769,7 @@ QEVICT_API qevict_status qevict_export_q_page(qevict_handle h, int32_t layer, in
   int u;
   if (!unit_of(h, layer, seq, &u)) return fail(h, QEVICT_ERR_INVALID_ARG, "layer or seq out of range");
   if (q_page < 0 || q_page >= h->geo.PQ) return fail(h, QEVICT_ERR_INVALID_ARG, "q_page out of range");
-  QE_CUDA(h, cudaSetDevice(h->cfg.device));
+  QE_DEVICE(h);
   const KernelArgs a = make_args(h, 0, h->geo.n_layers);
   QE_CUDA(h, launch_export_q_page(a, u, q_page, k_codes, k_params, v_codes, v_params, (cudaStream_t)stream));
   h->launches++;

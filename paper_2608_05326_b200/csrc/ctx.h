@@ -19,6 +19,25 @@ struct LayerMirror {  // what the host must know without reading device memory (
 
 constexpr int SM_COUNT_FALLBACK = 148;
 
+// Makes the cache's device current for the duration of an API call and puts the caller's device back afterwards.
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) {
+      err = cudaSetDevice(dev);
+      switched = err == cudaSuccess;
+    }
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+  DeviceGuard(const DeviceGuard&) = delete;
+  DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
+
 }  // namespace qevict
 
 struct qevict_ctx {
@@ -34,6 +53,8 @@ struct qevict_ctx {
   int forced_splits = 0;
   int sm_count = qevict::SM_COUNT_FALLBACK;
   bool timing = false;
+  bool broken = false;                // a launch failed half way through a step: the tables and the host's mirror may
+                                      // disagree from here on, every later call is refused
   std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
   std::vector<int> ev_kind;           // kernel index of each pair
   size_t ev_used = 0;
@@ -50,5 +71,9 @@ namespace qevict {
 
 // Splits per (unit, KV head) of the attention kernel for a call over `n_units` units.
 int choose_splits(const qevict_ctx* h, int n_units);
+// Argument and call-order checks of a decode step over layers [l0, l1); nullptr if the step may run (nothing is
+// enqueued before this has passed), else the status in *st and the message.
+const char* decode_precheck(const qevict_ctx* h, int layer, const void* q, const void* k_new, const void* v_new,
+                            const void* out, int* l0, int* l1, qevict_status* st);
 
 }  // namespace qevict

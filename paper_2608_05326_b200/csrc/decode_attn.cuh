@@ -34,6 +34,8 @@
 // full-precision tiles as loaded and low-bit tiles after dequantization, before the products.
 #pragma once
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace qevict {
@@ -665,12 +667,18 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_k
 template <class T, int D, int BITS, int GROUP, int TILES, bool PACK, bool ROPE>
 cudaError_t launch_decode_attn(const DecodeParams& p, int n_units, cudaStream_t stream) {
   using TT = DecodeTraits<T, D, BITS, GROUP, TILES, ROPE>;
-  static bool prepared = false;
-  if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK, ROPE>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TT::SMEM_BYTES);
+  // the shared-memory attribute of a kernel is kept per device: set it the first time this instantiation is
+  // launched on the current device (one bit per device ordinal; ordinals past 63 set it every time)
+  static std::atomic<unsigned long long> prepared{0ull};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = dev < 64 ? 1ull << dev : 0ull;
+  if (!(prepared.load(std::memory_order_acquire) & bit) || !bit) {
+    e = cudaFuncSetAttribute(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK, ROPE>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TT::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    prepared = true;
+    prepared.fetch_or(bit, std::memory_order_release);
   }
   dim3 grid(p.S, p.Hkv, n_units);
   return launch_pdl(decode_attn_kernel<T, D, BITS, GROUP, TILES, PACK, ROPE>, grid, dim3(DECODE_WARPS * 32), TT::SMEM_BYTES, stream, p);

@@ -6,6 +6,8 @@
 // inside this library's device image instead of in memory that somebody had to allocate.
 #include <stdio.h>
 
+#include <atomic>
+
 #include "ctx.h"
 
 using namespace qevict;
@@ -17,9 +19,10 @@ constexpr size_t NOALLOC_SCRATCH_BYTES = (size_t)QEVICT_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 // In host code `g_noalloc_scratch` is only a stand-in for the symbol, not a device address; the address is
-// asked for once per device, with that device current, and remembered here.
+// asked for once per device, with that device current, and remembered here (atomically: two handles on two
+// threads may make their first call at the same time; both would store the same address).
 constexpr int MAX_DEVICES = 64;
-void* g_scratch_addr[MAX_DEVICES] = {};
+std::atomic<void*> g_scratch_addr[MAX_DEVICES];
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -32,23 +35,17 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   cudaStream_t stream = (cudaStream_t)stream_;
   const Geometry& g = h->geo;
   int l0, l1;
-  if (layer == -1) { l0 = 0; l1 = g.n_layers; }
-  else if (layer >= 0 && layer < g.n_layers) { l0 = layer; l1 = layer + 1; }
-  else { h->last_error = "layer out of range"; return QEVICT_ERR_INVALID_ARG; }
-  if (!q || !out) { h->last_error = "q and out must not be NULL"; return QEVICT_ERR_INVALID_ARG; }
-  if ((k_new == nullptr) != (v_new == nullptr)) {
-    h->last_error = "k_new and v_new must both be given or both be NULL";
-    return QEVICT_ERR_INVALID_ARG;
-  }
+  qevict_status pst;
+  if (const char* msg = decode_precheck(h, layer, q, k_new, v_new, out, &l0, &l1, &pst)) { h->last_error = msg; return pst; }
   const int dev = h->cfg.device;
   if (dev < 0 || dev >= MAX_DEVICES) { h->last_error = "device ordinal not supported by the no-allocation entry point"; return QEVICT_ERR_UNSUPPORTED; }
 
-  // The scratch is indexed by unit exactly like the handle's own scratch, so it has to span the units up
-  // to the last one of the call.
-  const size_t units_spanned = (size_t)l1 * g.batch;
-  const size_t o_bytes = align256(units_spanned * g.Hq * (size_t)MAX_SPLITS * g.D * sizeof(float));
-  const size_t ml_bytes = align256(units_spanned * g.Hq * (size_t)MAX_SPLITS * 2 * sizeof(float));
-  const size_t w_bytes = align256(units_spanned * g.Hq * (size_t)g.EMAX * sizeof(float2));
+  // The array holds the partial results of this call's units only: unit u of the call uses slot u - unit0.
+  const size_t unit0 = (size_t)l0 * g.batch, n_units = (size_t)(l1 - l0) * g.batch;
+  const size_t o_unit = g.Hq * (size_t)MAX_SPLITS * g.D * sizeof(float);
+  const size_t ml_unit = g.Hq * (size_t)MAX_SPLITS * 2 * sizeof(float);
+  const size_t w_unit = g.Hq * (size_t)g.EMAX * sizeof(float2);
+  const size_t o_bytes = align256(n_units * o_unit), ml_bytes = align256(n_units * ml_unit), w_bytes = align256(n_units * w_unit);
   if (o_bytes + ml_bytes + w_bytes > NOALLOC_SCRATCH_BYTES) {
     char buf[192];
     snprintf(buf, sizeof(buf), "this call needs %zu bytes of attention scratch; the built-in array holds %zu (use qevict_decode_attn)",
@@ -56,23 +53,18 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
     h->last_error = buf;
     return QEVICT_ERR_NO_MEMORY;
   }
-  for (int l = l0; l < l1; ++l) {
-    const LayerMirror& m = h->layers[l];
-    if (!m.prefilled) { h->last_error = "decode before prefill_assign"; return QEVICT_ERR_BAD_STATE; }
-    if (k_new && !m.has_open) {
-      if (m.aged > g.aged_cap) { h->last_error = "too many filled windows are waiting: call qevict_rebalance"; return QEVICT_ERR_BAD_STATE; }
-      if (m.n_windows + 1 > g.NW) { h->last_error = "context would exceed max_context"; return QEVICT_ERR_BAD_STATE; }
-    }
-  }
-  cudaError_t e = cudaSetDevice(dev);
-  if (e == cudaSuccess && !g_scratch_addr[dev]) {
-    // set-up, once per device: ask the runtime where the array lives on this device
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-    if (e == cudaSuccess) g_scratch_addr[dev] = p;
+  DeviceGuard guard(dev);
+  cudaError_t e = guard.err;
+  void* addr = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (e == cudaSuccess && !addr) {
+    // set-up, once per device: ask the runtime where the array lives on this device (with lazy module loading
+    // this is also what makes the runtime place the library's device image, array included, on the device)
+    e = cudaGetSymbolAddress(&addr, g_noalloc_scratch);
+    if (e == cudaSuccess) g_scratch_addr[dev].store(addr, std::memory_order_release);
   }
   if (e != cudaSuccess) { h->last_error = std::string("no-allocation set-up: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
-  unsigned char* scratch = static_cast<unsigned char*>(g_scratch_addr[dev]);
+  // the kernels index their scratch by absolute unit: hand them the array's address moved back by unit0 slots
+  const uintptr_t base = reinterpret_cast<uintptr_t>(addr);
 
   KernelArgs a;
   a.geo = g;
@@ -81,11 +73,11 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
 #ifdef QEVICT_TRACE
   a.trace = h->st.trace + (size_t)TRACE_CALLS * TRACE_CALL_WORDS;  // not traced: the sink block
 #endif
-  a.st.o_part = reinterpret_cast<float*>(scratch);
-  a.st.ml = reinterpret_cast<float*>(scratch + o_bytes);
-  a.st.wrec = reinterpret_cast<float2*>(scratch + o_bytes + ml_bytes);
-  a.unit0 = l0 * g.batch;
-  a.n_units = (l1 - l0) * g.batch;
+  a.st.o_part = reinterpret_cast<float*>(base - unit0 * o_unit);
+  a.st.ml = reinterpret_cast<float*>(base + o_bytes - unit0 * ml_unit);
+  a.st.wrec = reinterpret_cast<float2*>(base + o_bytes + ml_bytes - unit0 * w_unit);
+  a.unit0 = (int)unit0;
+  a.n_units = (int)n_units;
 
   if (k_new) {
     e = launch_append(a, k_new, v_new, stream);
@@ -115,10 +107,10 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
   p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
   e = h->decode_fn(p, a.n_units, stream);
-  if (e != cudaSuccess) { h->last_error = std::string("attention: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
+  if (e != cudaSuccess) { h->broken = k_new != nullptr; h->last_error = std::string("attention: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
   h->launches++;
   e = launch_combine(a, p.S, e_bound, out, stream);
-  if (e != cudaSuccess) { h->last_error = std::string("combine: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
+  if (e != cudaSuccess) { h->broken = true; h->last_error = std::string("combine: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
   h->launches++;
   h->decode_steps++;
   return QEVICT_OK;

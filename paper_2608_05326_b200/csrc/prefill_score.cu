@@ -288,7 +288,8 @@ QEVICT_API qevict_status qevict_prefill_score(qevict_handle h, const void* k, co
   const int nqh = n_obs * g.G, NQ = n_obs * g.Hq, n_tiles = ctx_tokens / 32;
   const size_t sm_a = (size_t)nqh * g.D * sizeof(float);
   cudaStream_t s = (cudaStream_t)stream;
-  cudaError_t e = cudaSetDevice(h->cfg.device);
+  DeviceGuard guard(h->cfg.device);
+  cudaError_t e = guard.err;
   float2* rec = static_cast<float2*>(scratch);
   if (g.rope_base > 0.f) {
     // the keys are pre-RoPE: the scores are taken over a rotated copy (prompt positions 0 .. ctx_tokens - 1)

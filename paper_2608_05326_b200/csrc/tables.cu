@@ -1,5 +1,6 @@
 // Window tables: append to the recent region, prefill initialisation, and the routing event
 // (rank -> tiers -> page release / allocation -> migration lists -> decode work list).
+#include <mutex>
 #include <type_traits>
 
 #include "kernels.cuh"
@@ -834,11 +835,22 @@ size_t route_smem_bytes(const Geometry& g, int sort_cap) {
          (size_t)(3 * g.PF + 2 * g.PQ + g.EMAX + 128 + 512) * 4 + 16;
 }
 
+// The dynamic shared-memory limit of a kernel is a per-device attribute shared by every cache of the process:
+// it is only ever raised, to the largest size any cache on that device has asked for.
 cudaError_t route_prepare(size_t max_smem) {
+  static std::mutex mu;
+  static size_t granted[64] = {};
   if (max_smem <= 48 * 1024) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(route_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(route_kernel<ROUTE_MAX_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev >= 0 && dev < 64 && granted[dev] >= max_smem) return cudaSuccess;
+  e = cudaFuncSetAttribute(route_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(route_kernel<ROUTE_MAX_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) granted[dev] = max_smem;
+  return e;
 }
 
 cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s) {

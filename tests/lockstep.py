@@ -108,8 +108,9 @@ class LockstepRun:
     """One workload instance on the GPU (all its units in one cache) and oracles for a subset of units."""
 
     def __init__(self, wl, oracle_units=None, score_mode="observation", rebalance_interval=None, device="cuda",
-                 gen_device="cpu", score_levels=None, free_running=False):
+                 gen_device="cpu", score_levels=None, free_running=False, entry="decode_attn"):
         self.wl = wl
+        self.entry = entry  # which decode entry point the steps go through: "decode_attn" or "noalloc"
         self.R = wl.rebalance_interval if rebalance_interval is None else rebalance_interval
         self.units = list(range(wl.n_units)) if oracle_units is None else list(oracle_units)
         self.cache = binding.QEvictCache(gpu_config(wl, rebalance_interval=self.R))
@@ -159,7 +160,15 @@ class LockstepRun:
             compare_state(self.cache, layer, seq, orc, self.wl, None if pages == "all" else pages.get(u, []),
                           what="%s unit %d" % (what, u))
 
-    def step(self, append=True, check_mass=True):
+    def _decode(self, layer, q, kn, vn):
+        if self.entry == "noalloc":
+            out = torch.empty_like(q)
+            binding.qevict_decode_attn_noalloc(self.cache.handle, layer, q, kn, vn, out)
+            return out
+        return self.cache.decode_attn(layer, q, kn, vn)
+
+    def step(self, append=True, check_mass=True, per_layer=False):
+        """One decode step of every unit; per_layer=True issues one call per layer instead of one for all."""
         wl, t = self.wl, self.step_idx
         shape_q = (wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim)
         shape_kv = (wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim)
@@ -168,7 +177,12 @@ class LockstepRun:
         if append:
             kn = torch.stack([self.new_kv[u][0][t] for u in range(wl.n_units)]).reshape(shape_kv).to(self.dev)
             vn = torch.stack([self.new_kv[u][1][t] for u in range(wl.n_units)]).reshape(shape_kv).to(self.dev)
-        out = self.cache.decode_attn(-1, q, kn, vn).cpu().reshape(wl.n_units, wl.n_q_heads, wl.head_dim)
+        if per_layer:
+            out = torch.stack([self._decode(l, q[l].contiguous(), None if kn is None else kn[l].contiguous(),
+                                            None if vn is None else vn[l].contiguous()) for l in range(wl.n_layers)])
+        else:
+            out = self._decode(-1, q, kn, vn)
+        out = out.cpu().reshape(wl.n_units, wl.n_q_heads, wl.head_dim)
         for u, orc in self.oracles.items():
             layer, seq = self.unit_ls(u)
             ref_out, ref_mass = orc.decode_attn(self.queries[u][t].double().numpy(),
@@ -192,14 +206,18 @@ class LockstepRun:
                 orc.importance[:] = imp  # lockstep: route on the GPU's float32 scores
         self.step_idx += 1
         if self.step_idx % self.R == 0:
-            self.rebalance()
+            self.rebalance(per_layer=per_layer)
         return out
 
-    def rebalance(self, full_check=False):
+    def rebalance(self, full_check=False, per_layer=False):
         if self.free_running:
             return self._rebalance_free()
         before = {u: (o.tier.copy(), o.ledger_flag.copy()) for u, o in self.oracles.items()}
-        self.cache.rebalance(-1)
+        if per_layer:
+            for l in range(self.wl.n_layers):
+                self.cache.rebalance(l)
+        else:
+            self.cache.rebalance(-1)
         changed = {}
         for u, orc in self.oracles.items():
             orc.rebalance()

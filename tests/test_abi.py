@@ -68,6 +68,24 @@ def test_workspace_and_validation(lib):
     assert e.value.status in (1, 4)
 
 
+def test_shapes_the_kernels_cannot_walk_are_refused_with_a_reason(lib):
+    def refused(cfg, word):
+        with pytest.raises(binding.QEvictError) as e:
+            binding.qevict_workspace_bytes(cfg)
+        assert e.value.status == 4 and word in str(e.value), str(e.value)
+        assert word in lib.qevict_last_error(None).decode()
+
+    # budgets whose decode work list would exceed 32 entries x 4 warps x 64 splits
+    refused(binding.make_config(1, 1, 8, 8, 64, "bf16", 32, 4, 32, 4096, 4100, 8192 * 32), "work-list")
+    # routing tables of one sequence beyond the shared memory of an SM
+    refused(binding.make_config(1, 1, 8, 8, 64, "bf16", 32, 4, 32, 4000, 4000, 8192 * 32), "shared memory")
+    # key-norm ranking stages H_kv * d <= 4096 elements of the token
+    refused(binding.make_config(1, 1, 64, 64, 128, "bf16", 32, 4, 32, 8, 8, 4096, rank_mode=3), "key-norm")
+    # a failed call does not disturb a good one, and the largest BASELINE shape passes
+    ok = binding.make_config(4, 8, 32, 8, 128, "bf16", 64, 4, 64, 64, 256, 131072 + 1024)
+    assert binding.qevict_workspace_bytes(ok) > 0
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device error path")
 def test_create_without_a_device_fails_loudly(lib):
     cfg = binding.make_config(1, 1, 4, 2, 64, "fp16", 32, 4, 32, 2, 2, 1024)
@@ -75,3 +93,4 @@ def test_create_without_a_device_fails_loudly(lib):
     fake = C.c_void_p(256 * 1024)  # never dereferenced on the host; no device to clear it on
     st = lib.qevict_create(C.byref(cfg), fake, 1 << 30, C.byref(h))
     assert st == 5 and not h.value  # QEVICT_ERR_CUDA, no handle, no fallback
+    assert b"device" in lib.qevict_last_error(None)
