@@ -31,13 +31,6 @@ from paper_2608_05326_b200 import sharding, workloads  # noqa: E402
 METRIC = "decode_steps_per_sec"
 UNIT = "steps/s"
 HBM_FALLBACK_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures
-# summarised under profiles/ (bytes per launch, keyed by workload name); None = not captured.
-NCU_TRAFFIC_BYTES = {
-    # profiles/decode_attn_c1x32.md: 440.83 MB read + 6.50 MB written per launch
-    "c1-llama3-8b-32k": 446_080_000,
-}
-
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -68,6 +61,7 @@ def parse_args():
     ap.add_argument("--fixed-context", action="store_true", help="no appends (k_new = NULL)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="default run only: skip the second target configuration (config 3 x 8 layers)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     return ap.parse_args()
 
@@ -148,7 +142,15 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ ours
-def build_inputs(wl, device):
+INPUT_POOL = 384        # distinct decode steps of inputs held on the device; longer runs go round the pool
+SETTLE_STEPS = 32       # untimed steps right after prefill (state preparation, not warm-up): the first routing
+                        # events after a prefill quantize every window that leaves the full-precision tier for the
+                        # first time, a burst that later steps do not see
+MIN_TIMED_SECONDS = 0.5 # a K-step loop shorter than this is repeated and the median repeat is reported
+MAX_REPEATS = 9
+
+
+def build_inputs(wl, n_input_steps, device):
     """All inputs of the run, resident on `device`: prompts are consumed by prefill layer by layer."""
     scores, queries, knew, vnew = [], [], [], []
     prompts = {}
@@ -157,8 +159,8 @@ def build_inputs(wl, device):
         s = workloads.place_planted(workloads.synthetic_window_scores(wl, u), workloads.planted_windows(wl, u),
                                     wl.fp_budget_windows, wl.q_budget_windows)
         scores.append(s)
-        queries.append(workloads.gen_queries(wl, u, k, s, device=device))
-        kn, vn = workloads.gen_new_kv(wl, u, device=device)
+        queries.append(workloads.gen_queries(wl, u, k, s, n_steps=n_input_steps, device=device))
+        kn, vn = workloads.gen_new_kv(wl, u, n_steps=n_input_steps, device=device)
         knew.append(kn); vnew.append(vn)
         prompts[u] = (k, v)
         yield_layer = (u + 1) % wl.batch == 0
@@ -171,9 +173,9 @@ def build_inputs(wl, device):
                 del prompts[x]
     shape_q = (wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim)
     shape_kv = (wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim)
-    q = torch.stack(queries, 1).reshape((wl.steps,) + shape_q).contiguous()
-    kn = torch.stack(knew, 1).reshape((wl.steps,) + shape_kv).contiguous()
-    vn = torch.stack(vnew, 1).reshape((wl.steps,) + shape_kv).contiguous()
+    q = torch.stack(queries, 1).reshape((n_input_steps,) + shape_q).contiguous()
+    kn = torch.stack(knew, 1).reshape((n_input_steps,) + shape_kv).contiguous()
+    vn = torch.stack(vnew, 1).reshape((n_input_steps,) + shape_kv).contiguous()
     yield ("steps", q, kn, vn)
 
 
@@ -190,31 +192,43 @@ def attention_kernel_bytes(wl, stats, n_splits_hint=None):
     return kv + q_bytes + lists
 
 
-def run_ours(args, rank, world):
-    if args.timeline:
-        os.environ["QEVICT_TRACE_LIB"] = "1"  # read when the binding is first imported
-    from paper_2608_05326_b200 import binding, build
-    if rank == 0:
-        build.build(trace=args.timeline)  # no-op when the in-tree library is newer than its sources
-    if world > 1:
-        torch.distributed.barrier()
-    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
-    torch.cuda.set_device(dev)
-    K, W = args.steps, args.warmup
-    phases = 2 + (0 if args.no_e2e else 1)
-    total_steps = W + phases * K
-    wl = make_workload(args, total_steps)
-    wl = sharding.rank_workload(wl, rank)  # every rank owns its own sequences (weak scaling, no exchange)
+def dram_traffic_bytes(wl):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch on this workload, as recorded
+    from an ncu capture in profiles/dram_traffic.txt (one line per workload: key, read bytes, write bytes, the
+    summary the figures come from); None for a workload without a capture."""
+    key = "%s/L%d/B%d/rope%d" % (wl.name, wl.n_layers, wl.batch, 1 if wl.rope_base > 0 else 0)
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 3 and parts[0] == key:
+                    return int(parts[1]) + int(parts[2])
+    except OSError:
+        pass
+    return None
+
+
+def measure_workload(args, wl, rank, world, dev, K, W, with_e2e, timeline=False):
+    """Builds the cache of `wl` on `dev`, runs the decode loop and returns the measurements of one workload."""
+    from paper_2608_05326_b200 import binding
+    Wwin = wl.window
+    R = args.rebalance_interval
+    append = not args.fixed_context
+    # steps the run may take at most: settle + warm-up + the repeated timed loop + the event-bracketed loop + the
+    # loop at the paper's interval (one routing event per filled window) + the end-to-end loop
+    total_steps = SETTLE_STEPS + W + (MAX_REPEATS + 1) * K + max(K, 4 * Wwin) + (K if with_e2e else 0) + 2 * Wwin
+    n_in = min(total_steps, INPUT_POOL)
+    wl = replace(wl, steps=total_steps)  # sizes max_context for every token the run appends
     cfg = binding.make_config(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, wl.window,
                               wl.quant_bits, wl.group_size, wl.fp_budget_windows, wl.q_budget_windows, wl.max_context,
-                              rebalance_interval_hint=args.rebalance_interval, device=dev.index,
+                              rebalance_interval_hint=max(R, 1), device=dev.index,
                               sink_windows=wl.sink_windows, recent_windows=wl.recent_windows, rank_mode=wl.rank_mode,
                               rank_param=wl.rank_param, rope_base=wl.rope_base)
     cache = binding.QEvictCache(cfg)
     if args.splits:
         cache.set_splits(args.splits)
     q = kn = vn = None
-    for item in build_inputs(wl, dev):
+    for item in build_inputs(wl, n_in, dev):
         if item[0] == "layer":
             _, layer, k, v, s = item
             cache.prefill_assign(layer, k, v, s)
@@ -223,58 +237,79 @@ def run_ours(args, rank, world):
         else:
             _, q, kn, vn = item
     out = torch.empty_like(q[0])
-    R = args.rebalance_interval
-    append = not args.fixed_context
+    state = {"t": 0}
 
-    def step(t):
-        cache.decode_attn(-1, q[t], kn[t] if append else None, vn[t] if append else None, out)
-        if (t + 1) % R == 0:
+    def step(interval=R):
+        t = state["t"]
+        i = t % n_in
+        cache.decode_attn(-1, q[i], kn[i] if append else None, vn[i] if append else None, out)
+        if (t + 1) % interval == 0:
             cache.rebalance(-1)
+        state["t"] = t + 1
 
     def barrier():
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
-    t = 0
-    for _ in range(W):
-        step(t); t += 1
-    if args.timeline:
+    def timed_loop(n, interval=R):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        h0 = time.perf_counter()
+        for _ in range(n):
+            step(interval)
+        host_s = time.perf_counter() - h0   # host time to enqueue the steps (no synchronisation)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1), host_s
+
+    for _ in range(SETTLE_STEPS + W):
+        step()
+    if timeline:
         cache.kernel_timeline()  # restart the record after the warm-up
         for _ in range(min(K, 250)):  # the library records 512 calls (two per step)
-            step(t); t += 1
+            step()
         line = timeline_summary(cache.kernel_timeline(), wl)
         cache.close()
-        return line, wl
-    # ---- timed region: device-resident inputs ----
+        return line
+    # ---- timed region: device-resident inputs; K steps, repeated while a loop is shorter than MIN_TIMED_SECONDS ----
     launches0 = cache.launch_count()
     sampler = ClockSampler(dev.index)
     sampler.start()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    host_t0 = time.perf_counter()
-    for _ in range(K):
-        step(t); t += 1
-    host_enqueue_s = time.perf_counter() - host_t0   # host time to enqueue the K steps (no synchronisation)
-    e1.record()
-    barrier()
+    loops = [timed_loop(K)]
+    first_ms = sharding.max_over_ranks([loops[0][0]], device=dev)[0]
+    repeats = 1 if first_ms * 1e-3 >= MIN_TIMED_SECONDS else MAX_REPEATS
+    while len(loops) < repeats:
+        loops.append(timed_loop(K))
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
     launches = cache.launch_count() - launches0
-    # ---- same loop with the attention kernel bracketed by events ----
+    rep_ms = sorted(sharding.max_over_ranks([ms for ms, _ in loops], device=dev)) if world > 1 else sorted(ms for ms, _ in loops)
+    ms = statistics.median(rep_ms)
+    host_enqueue_s = statistics.median(h for _, h in loops)
+    # ---- same loop with every kernel bracketed by events ----
     cache.set_kernel_timing(True)
     for _ in range(K):
-        step(t); t += 1
+        step()
     torch.cuda.synchronize()
     ktimes = cache.kernel_times()
     kernel_ms, kernel_n = ktimes["decode_attn"]
     cache.set_kernel_timing(False)
     stats = cache.stats()
+    # ---- the paper's coupling of window and interval: one routing event per filled window (every W steps) ----
+    interval_w = None
+    if R != Wwin and not args.fixed_context:
+        while state["t"] % Wwin:
+            step()  # reach a window boundary with routing after every step, as before
+        n_w = max(K, 4 * Wwin) // Wwin * Wwin
+        ms_w, _ = timed_loop(n_w, interval=Wwin)
+        ms_w = sharding.max_over_ranks([ms_w], device=dev)[0]
+        interval_w = (ms_w, n_w)
     # ---- end to end: host buffers through the host entry point ----
     e2e = None
-    if not args.no_e2e:
-        qh = q[t:t + K].cpu().pin_memory(); knh = kn[t:t + K].cpu().pin_memory(); vnh = vn[t:t + K].cpu().pin_memory()
+    if with_e2e:
+        idx = [(state["t"] + i) % n_in for i in range(K)]
+        qh = q[idx].cpu().pin_memory(); knh = kn[idx].cpu().pin_memory(); vnh = vn[idx].cpu().pin_memory()
         outh = torch.empty_like(qh[0]).pin_memory()
         barrier()
         t0 = time.perf_counter()
@@ -285,55 +320,108 @@ def run_ours(args, rank, world):
         for i in range(K):
             cache.decode_attn_host_async(-1, qh[i], knh[i] if append else None, vnh[i] if append else None, outh)
             got.record()          # the result is in host memory once this event has passed
-            if (t + i + 1) % R == 0:
+            if (state["t"] + i + 1) % R == 0:
                 cache.rebalance(-1)
             got.synchronize()     # the routing event keeps running while the host turns around
         barrier()
-        e2e_s = time.perf_counter() - t0
+        e2e_s = sharding.max_over_ranks([time.perf_counter() - t0], device=dev)[0]
+        state["t"] += K
         h2d = qh[0].numel() * 2 + (2 * knh[0].numel() * 2 if append else 0)
         e2e = {"seconds": e2e_s, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": outh.numel() * 2}
-
-    ms, e2e_s = sharding.max_over_ranks([ms, e2e["seconds"] if e2e else 0.0], device=dev)
-    if e2e:
-        e2e["seconds"] = e2e_s
+    cache.close()
     if rank != 0:
-        cache.close()
         return None
     peak, peak_kind = peak_hbm_gbs()
     kbytes = attention_kernel_bytes(wl, stats)
     k_avg_ms = kernel_ms / max(kernel_n, 1)
     achieved = kbytes / (k_avg_ms * 1e-3) / 1e9 if k_avg_ms > 0 else 0.0
-    line = {
-        "metric": METRIC, "value": sharding.aggregate_steps_per_second(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
-        "data": "synthetic",
-        "config": {
-            "workload": "%s x %d layers x batch %d (layer-batched launches)" % (wl.name, wl.n_layers, wl.batch),
-            "units_per_step": wl.n_units, "context": wl.context, "window": wl.window, "quant_bits": wl.quant_bits,
-            "group_size": wl.group_size, "fp_budget_windows": wl.fp_budget_windows,
-            "q_budget_windows": wl.q_budget_windows, "sink_windows": wl.sink_windows, "recent_windows": wl.recent_windows,
-            "rebalance_interval": R, "append": append, "rope_base": wl.rope_base,
-            "l2": "inputs larger than L2 (KV working set %.0f MB per step)" % (kbytes / 1e6),
-        },
-        "layer_steps_per_sec": world * K * wl.n_units / (ms * 1e-3),
-        "clocks": clocks,
-        "gpu_launches": int(launches),
+    step_gbs = kbytes / (ms / K * 1e-3) / 1e9
+    res = {
+        "workload": "%s x %d layers x batch %d (layer-batched launches)" % (wl.name, wl.n_layers, wl.batch),
+        "wl": wl, "K": K, "ms": ms, "rep_ms": rep_ms, "repeats": len(rep_ms), "launches": int(launches), "clocks": clocks,
+        "host_enqueue_us_per_step": round(host_enqueue_s * 1e6 / K, 2),
+        "kernel_us_per_step": {k: round(v[0] * 1e3 / K, 2) for k, v in ktimes.items()},
+        "stats": stats, "e2e": e2e, "kbytes": kbytes,
         "roofline": {
             "bound": "hbm", "kernel": "decode_attn_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth", "frac_of_8TBs": achieved / 8000.0,
             "bytes_per_launch": kbytes, "kernel_ms": k_avg_ms, "kernel_launches_timed": int(kernel_n),
             "kernel_share_of_step": k_avg_ms / (ms / K),
-            "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+            # the whole step (append + attention + combine + route + migrate) against the same algorithmic bytes
+            "step_frac": step_gbs / peak, "step_frac_of_8TBs": step_gbs / 8000.0,
+            "traffic": dram_traffic_bytes(wl),
         },
-        "host_enqueue_us_per_step": round(host_enqueue_s * 1e6 / K, 2),
-        "kernel_us_per_step": {k: round(v[0] * 1e3 / K, 2) for k, v in ktimes.items()},
-        "tier_state": {k: stats[k] for k in ("n_full", "n_quant", "n_aged", "n_sink", "n_open", "n_evicted", "promotions",
-                                             "quantizations", "reactivations", "deletions")},
     }
-    if e2e:
+    if interval_w:
+        ms_w, n_w = interval_w
+        gbs_w = kbytes / (ms_w / n_w * 1e-3) / 1e9
+        res["interval_w"] = {"rebalance_interval": Wwin, "steps": n_w, "ms_per_step": ms_w / n_w,
+                             "value": world * n_w / (ms_w * 1e-3), "step_frac": gbs_w / peak, "step_frac_of_8TBs": gbs_w / 8000.0}
+    return res
+
+
+def run_ours(args, rank, world):
+    if args.timeline:
+        os.environ["QEVICT_TRACE_LIB"] = "1"  # read when the binding is first imported
+    from paper_2608_05326_b200 import build
+    if rank == 0:
+        build.build(trace=args.timeline)  # no-op when the in-tree library is newer than its sources
+    if world > 1:
+        torch.distributed.barrier()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    K, W = args.steps, args.warmup
+    wl = sharding.rank_workload(make_workload(args, K), rank)  # every rank owns its own sequences (weak scaling, no exchange)
+    res = measure_workload(args, wl, rank, world, dev, K, W, with_e2e=not args.no_e2e, timeline=args.timeline)
+    if args.timeline:
+        return res, wl
+    # the default run also carries the second target configuration (128k context, 8 layers in one launch)
+    also = None
+    default_run = (args.config == 1 and args.layers is None and args.batch is None and args.rope_base == 0.0 and
+                   not args.fixed_context and args.rank_mode == 0 and not args.sink_windows and not args.recent_windows and
+                   not args.no_also)
+    if default_run:
+        wl3 = sharding.rank_workload(replace(workloads.config(3), n_layers=8, rebalance_interval=args.rebalance_interval), rank)
+        also = measure_workload(args, wl3, rank, world, dev, K, W, with_e2e=False)
+    if rank != 0:
+        return None
+    wl, ms, R = res["wl"], res["ms"], args.rebalance_interval
+    line = {
+        "metric": METRIC, "value": sharding.aggregate_steps_per_second(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+        "data": "synthetic",
+        "repeats": res["repeats"], "ms_per_step_min": res["rep_ms"][0] / K, "ms_per_step_max": res["rep_ms"][-1] / K,
+        "config": {
+            "workload": res["workload"],
+            "units_per_step": wl.n_units, "context": wl.context, "window": wl.window, "quant_bits": wl.quant_bits,
+            "group_size": wl.group_size, "fp_budget_windows": wl.fp_budget_windows,
+            "q_budget_windows": wl.q_budget_windows, "sink_windows": wl.sink_windows, "recent_windows": wl.recent_windows,
+            "rebalance_interval": R, "append": not args.fixed_context, "rope_base": wl.rope_base,
+            "l2": "inputs larger than L2 (KV working set %.0f MB per step)" % (res["kbytes"] / 1e6),
+            "settle_steps": SETTLE_STEPS, "input_pool_steps": min(INPUT_POOL, wl.steps),
+            "timing": "median of %d repeats of the %d-step loop (a loop shorter than %.1f s is repeated)" % (res["repeats"], K, MIN_TIMED_SECONDS),
+        },
+        "layer_steps_per_sec": world * K * wl.n_units / (ms * 1e-3),
+        "clocks": res["clocks"],
+        "gpu_launches": res["launches"],
+        "roofline": res["roofline"],
+        "host_enqueue_us_per_step": res["host_enqueue_us_per_step"],
+        "kernel_us_per_step": res["kernel_us_per_step"],
+        "tier_state": {k: res["stats"][k] for k in ("n_full", "n_quant", "n_aged", "n_sink", "n_open", "n_evicted", "promotions",
+                                                     "quantizations", "reactivations", "deletions")},
+    }
+    if "interval_w" in res:
+        line["rebalance_every_window"] = res["interval_w"]
+    if res["e2e"]:
+        e2e = res["e2e"]
         line["e2e"] = {"value": world * K / e2e["seconds"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d_bytes_per_step"],
                        "d2h_bytes_per_step": e2e["d2h_bytes_per_step"]}
-    cache.close()
+    if also:
+        line["also"] = {"workload": also["workload"], "value": sharding.aggregate_steps_per_second(world, K, also["ms"]),
+                        "unit": UNIT, "ms_per_step": also["ms"] / K, "repeats": also["repeats"], "roofline": also["roofline"],
+                        "kernel_us_per_step": also["kernel_us_per_step"], "gpu_launches": also["launches"]}
+        if "interval_w" in also:
+            line["also"]["rebalance_every_window"] = also["interval_w"]
     return line, wl
 
 
@@ -362,12 +450,18 @@ def timeline_summary(records, wl):
 
 
 def oracle_threads():
+    """Size of the BLAS thread pool the oracle's matrix products may use (its element-wise numpy code is single-threaded)."""
     try:
         from threadpoolctl import threadpool_info
         n = [p.get("num_threads", 1) for p in threadpool_info()]
         return max(n) if n else 1
     except Exception:
         return 1
+
+
+def _cpu_seconds():
+    t = os.times()
+    return t.user + t.system
 
 
 def time_oracle(wl, n_steps, warmup, budget_s):
@@ -394,6 +488,7 @@ def time_oracle(wl, n_steps, warmup, budget_s):
     for _ in range(warmup):
         orc.decode_attn(q[t], kn[t], vn[t]); orc.rebalance(); t += 1
     done = 0
+    c0 = _cpu_seconds()
     t0 = time.perf_counter()
     while done < n_steps and t < q.shape[0] and time.perf_counter() - t0 < budget_s:
         orc.decode_attn(q[t], kn[t], vn[t])
@@ -401,10 +496,16 @@ def time_oracle(wl, n_steps, warmup, budget_s):
             orc.rebalance()
         t += 1; done += 1
     dt = time.perf_counter() - t0
+    busy = (_cpu_seconds() - c0) / dt if dt > 0 else 1.0   # cores kept busy on average (process CPU time / wall time)
     unit_steps_per_s = done / dt
     value = unit_steps_per_s / wl.n_units
     sample = "unit 0 of %d, %d decode+rebalance steps in %.1f s" % (wl.n_units, done, dt)
-    return value, sample, done, dt
+    return value, sample, done, dt, busy
+
+
+def cpu_baseline_record(value, sample, busy):
+    return {"value": value, "unit": UNIT, "cores": max(1, round(busy)), "kind": "oracle", "sample": sample,
+            "cores_busy_avg": round(busy, 2), "blas_threads": oracle_threads(), "host_cores": os.cpu_count()}
 
 
 def run_reference(args, rank):
@@ -412,14 +513,13 @@ def run_reference(args, rank):
         return None
     K, W = args.steps, args.warmup
     wl = make_workload(args, max(W + K, 8))
-    value, sample, done, dt = time_oracle(wl, K, W, budget_s=180.0)
-    cores = oracle_threads()
+    value, sample, done, dt, busy = time_oracle(wl, K, W, budget_s=180.0)
     return {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": done,
         "warmup": W, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": "%s x %d layers x batch %d" % (wl.name, wl.n_layers, wl.batch), "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": cpu_baseline_record(value, sample, busy),
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -458,10 +558,32 @@ def run_prefill_score(args):
     return line
 
 
+def spawn_ranks(args):
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script, one per GPU, under
+    torch.distributed.run (rank 0 prints the one JSON line).  Returns the launcher's exit code."""
+    import socket
+    if args.impl == "ours":
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            sys.stderr.write("bench.py: --gpus %d asked for, %d CUDA device(s) visible; not running fewer ranks than asked\n" % (args.gpus, have))
+            return 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if world != max(args.gpus, 1):
+        sys.stderr.write("bench.py: --gpus %d does not match the launcher's WORLD_SIZE %d\n" % (args.gpus, world))
+        sys.exit(2)
     if args.prefill_score > 0:
         if rank == 0:
             print(json.dumps(run_prefill_score(args)))
@@ -472,14 +594,15 @@ def main():
             print(json.dumps(line))
         return
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "WARN")
         torch.distributed.init_process_group("nccl")
     res = run_ours(args, rank, world)
     if rank == 0:
         line, wl = res
         if not args.timeline and not args.no_cpu_baseline and world >= 1:
             small = replace(wl, steps=256, seed=wl.seed)
-            value, sample, _, _ = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds)
-            line["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample}
+            value, sample, _, _, busy = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds)
+            line["cpu_baseline"] = cpu_baseline_record(value, sample, busy)
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()

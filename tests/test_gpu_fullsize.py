@@ -26,7 +26,7 @@ def _run(wl, oracle_units, steps, rebalance_interval=1, check_all_units_mass=Tru
             for u in range(wl.n_units):
                 m = run.cache.export_last_mass(u // wl.batch, u % wl.batch).double().sum().item()
                 assert abs(m - wl.n_q_heads) < 1e-4 * wl.n_q_heads, (u, m)
-    run.rebalance(full_check=False)
+    run.rebalance(full_check=True)  # every live page, code and table of the followed units
     st = run.cache.stats()
     assert st["n_full"] <= wl.n_units * wl.fp_budget_windows and st["n_quant"] <= wl.n_units * wl.q_budget_windows
     for u in oracle_units:
@@ -44,15 +44,22 @@ def test_config1_llama_32k_x32_layers_sampled_units():
 
 
 def test_config2_stacked_2bit_sampled_units():
-    # 16 sequences x 4 of the 32 layers (the per-unit work is the full-size one; fewer layers keep the
-    # test short), 2-bit codes, rebalance every step
-    wl = workloads.config(2, n_layers=4)
-    _run(wl, oracle_units=[5, 37, 63], steps=36)
+    # 16 sequences x 8 of the 32 layers = 128 of the 512 units (the per-unit work and the split count are those
+    # of the full configuration -- the launch fills the GPU several times over either way; 8 layers keep the
+    # prompts of the test within a few GB and its run time short), 2-bit codes, rebalance every step
+    wl = workloads.config(2, n_layers=8)
+    _run(wl, oracle_units=[5, 37, 63, 127], steps=36)
 
 
 def test_config3_long_context_window64_sampled_unit():
     wl = workloads.config(3)
     _run(wl, oracle_units=[2], steps=70, check_all_units_mass=True)
+
+
+def test_config3_x8_layers_sampled_units():
+    # the launch configuration the 128k roofline figure is quoted on: 8 layers x 4 sequences in one launch
+    wl = workloads.config(3, n_layers=8)
+    _run(wl, oracle_units=[3, 30], steps=40)
 
 
 def test_config3_long_context_pre_rope_keys_sampled_unit():
@@ -66,7 +73,7 @@ def test_config1_x32_layers_pre_rope_keys_sampled_unit():
     _run(wl, oracle_units=[7], steps=34)
 
 
-@pytest.mark.parametrize("bits,fp_frac", [(4, 0.10), (2, 0.20)])
+@pytest.mark.parametrize("bits,fp_frac", [(4, 0.05), (4, 0.10), (4, 0.20), (2, 0.05), (2, 0.10), (2, 0.20)])
 def test_config4_qwen_gqa7_sampled_unit(bits, fp_frac):
     wl = workloads.config(4, bits=bits, fp_frac=fp_frac)
     _run(wl, oracle_units=[3], steps=34, rebalance_interval=2)

@@ -43,3 +43,32 @@ def test_two_ranks_own_disjoint_sequences_and_agree_on_the_slowest_time():
 def test_single_process_is_the_identity():
     assert sharding.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert sharding.aggregate_steps_per_second(1, 100, 50.0) == 2000.0
+
+
+def _bench(*argv):
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    return subprocess.run([sys.executable, os.path.join(root, "bench.py")] + list(argv), capture_output=True, text=True,
+                          env=env, timeout=600)
+
+
+def test_bench_gpus_n_starts_n_ranks_and_prints_one_line():
+    """`python bench.py --gpus 2` outside a launcher starts two ranks itself; the CPU arm shows it without a GPU:
+    rank 0 alone prints the line, which names two ranks."""
+    import json
+    r = _bench("--gpus", "2", "--impl", "reference", "--steps", "1", "--warmup", "0")
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["impl"] == "reference" and line["value"] > 0
+
+
+def test_bench_refuses_to_run_fewer_ranks_than_asked():
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 8:
+        return
+    r = _bench("--gpus", "8", "--steps", "1", "--warmup", "0")
+    assert r.returncode != 0 and "--gpus 8" in r.stderr
+    assert not [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
