@@ -393,6 +393,13 @@ QEVICT_API const char* qevict_last_error(qevict_handle h);
 QEVICT_API const char* qevict_status_string(qevict_status s);
 /* Library version, "major.minor". */
 QEVICT_API const char* qevict_version(void);
+/* Which build of the sources this library is: 0 the normal one; 1 the tracing build (-DQEVICT_TRACE: kernel
+ * timeline); 2 the checking build (-DQEVICT_DEBUG_BOUNDS: every page id, window index, work-list entry and
+ * migration record a kernel reads from a table is range-checked before use -- a value out of range is recorded
+ * (qevict_get_stats then returns QEVICT_ERR_DEVICE_CHECK with the code in qevict_last_error) and the access is
+ * skipped, nothing traps -- and both pools start filled with a NaN pattern so that a read of a page nobody wrote
+ * shows in the results).  The checking build stands in for a memory checker; it computes the same results. */
+QEVICT_API int32_t qevict_build_flavour(void);
 
 #ifdef __cplusplus
 }

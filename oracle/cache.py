@@ -15,7 +15,7 @@ Paper basis:
     "Byte-Constrained Tier Allocation"; per-window byte costs: the memory
     accounting appendix.
 
-Readings taken where the paper is silent (each is listed in the design notes):
+Readings taken where the paper is silent:
   * the window size W and the routing interval are separate parameters; routing
     happens when `rebalance()` is called;
   * the protected regions are window-granular: the sink prefix is the first

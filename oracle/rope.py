@@ -11,7 +11,7 @@ the rotation itself; it is the standard one of the models it evaluates (Llama, Q
 
 for a key at absolute position p.
 
-Readings taken where the paper is silent (each is listed in the design notes):
+Readings taken where the paper is silent:
   * every stored key, full precision or low-bit, is pre-RoPE (a window must be quantizable at any routing event, and
     a promoted window holds the dequantized pre-RoPE approximation); the rotation is applied whenever attention
     reads a key; queries arrive already rotated; values are never rotated;

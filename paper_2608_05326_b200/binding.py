@@ -14,6 +14,10 @@ LIB_PATH = os.path.join(_HERE, "libqevict.so")
 # the normal library.
 if os.environ.get("QEVICT_TRACE_LIB", "0") not in ("", "0"):
     LIB_PATH = os.path.join(_HERE, "libqevict_trace.so")
+# QEVICT_CHECK_LIB=1 loads the checking variant (build.build(variant="check")): the same kernels with every table
+# index range-checked before use and the pools poisoned with NaN at creation.
+if os.environ.get("QEVICT_CHECK_LIB", "0") not in ("", "0"):
+    LIB_PATH = os.path.join(_HERE, "libqevict_check.so")
 
 QEVICT_OK = 0
 DTYPE_FP16, DTYPE_BF16 = 0, 1
@@ -69,6 +73,7 @@ _lib = None
 
 _SIGNATURES = {
     "qevict_version": (C.c_char_p, []),
+    "qevict_build_flavour": (C.c_int32, []),
     "qevict_status_string": (C.c_char_p, [C.c_int]),
     "qevict_last_error": (C.c_char_p, [C.c_void_p]),
     "qevict_launch_count": (C.c_uint64, [C.c_void_p]),

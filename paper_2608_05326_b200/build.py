@@ -15,6 +15,12 @@ LIB = os.path.join(HERE, "libqevict.so")
 # none of it
 OBJ_TRACE = os.path.join(HERE, "build_trace")
 LIB_TRACE = os.path.join(HERE, "libqevict_trace.so")
+# the same sources with -DQEVICT_DEBUG_BOUNDS: every index a kernel reads from a table is range-checked before use
+# (recorded and skipped, never trapped) and the pools start as NaN; the parity tests run against it once
+OBJ_CHECK = os.path.join(HERE, "build_check")
+LIB_CHECK = os.path.join(HERE, "libqevict_check.so")
+_VARIANTS = {None: (OBJ, LIB, []), "trace": (OBJ_TRACE, LIB_TRACE, ["-DQEVICT_TRACE"]),
+             "check": (OBJ_CHECK, LIB_CHECK, ["-DQEVICT_DEBUG_BOUNDS"])}
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,26 +49,28 @@ def _stale(lib=LIB):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def _compile(nvcc, src, verbose, trace=False):
-    obj = os.path.join(OBJ_TRACE if trace else OBJ, src[:-3] + ".o")
-    cmd = [nvcc] + NVCC_FLAGS + (["-DQEVICT_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else []) + \
-          ["-c", os.path.join(CSRC, src), "-o", obj]
+def _compile(nvcc, src, verbose, variant=None):
+    obj_dir, _, defs = _VARIANTS[variant]
+    obj = os.path.join(obj_dir, src[:-3] + ".o")
+    cmd = [nvcc] + NVCC_FLAGS + defs + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s" % (src, r.stderr))
     return obj, r.stderr
 
 
-def build(force=False, verbose=False, trace=False):
-    """Compile and link the library (the tracing variant with trace=True) if any source is newer than it.
-    Returns the library path."""
-    lib = LIB_TRACE if trace else LIB
+def build(force=False, verbose=False, trace=False, variant=None):
+    """Compile and link the library (variant "trace" or "check" for the tracing / checking build; trace=True is the
+    former) if any source is newer than it.  Returns the library path."""
+    if trace:
+        variant = "trace"
+    obj_dir, lib, _ = _VARIANTS[variant]
     if not force and not _stale(lib):
         return lib
     nvcc = _nvcc()
-    os.makedirs(OBJ_TRACE if trace else OBJ, exist_ok=True)
+    os.makedirs(obj_dir, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as ex:
-        results = list(ex.map(lambda s: _compile(nvcc, s, verbose, trace), _sources()))
+        results = list(ex.map(lambda s: _compile(nvcc, s, verbose, variant), _sources()))
     if verbose:
         for _, log in results:
             sys.stderr.write(log)
@@ -75,4 +83,5 @@ def build(force=False, verbose=False, trace=False):
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                variant="trace" if "--trace" in sys.argv else ("check" if "--check" in sys.argv else None)))

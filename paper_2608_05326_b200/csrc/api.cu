@@ -324,7 +324,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   p.q = q; p.entries = h->st.entries; p.n_live = h->st.n_live; p.open_fill = h->st.open_fill;
   p.fp_pool = h->st.fp_pool; p.q_pool = h->st.q_pool; p.o_part = h->st.o_part; p.ml = h->st.ml; p.wrec = h->st.wrec;
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
-  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
+  p.PF = g.PF; p.PQ = g.PQ; p.NW = g.NW; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2; p.status = h->st.status;
   p.rope = reinterpret_cast<const char*>(h->st.rope_table);
 #ifdef QEVICT_TRACE
   p.trace = a.trace;
@@ -340,7 +340,17 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
 
 extern "C" {
 
-QEVICT_API const char* qevict_version(void) { return "0.1"; }
+QEVICT_API const char* qevict_version(void) { return "0.2"; }
+
+QEVICT_API int32_t qevict_build_flavour(void) {
+#if defined(QEVICT_DEBUG_BOUNDS)
+  return 2;
+#elif defined(QEVICT_TRACE)
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 QEVICT_API const char* qevict_status_string(qevict_status s) {
   switch (s) {
@@ -435,6 +445,12 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
     const size_t U = g.n_units;
     // tables: everything between the pools and the scratch starts cleared
     e = cudaMemset(h->st.tier, 0, U * g.NW);
+#ifdef QEVICT_DEBUG_BOUNDS
+    // checking build: both pools start as a NaN pattern (all ones is a NaN in fp16 and in bf16), so that a read
+    // of a page nobody wrote shows in the results
+    if (e == cudaSuccess) e = cudaMemset(h->st.fp_pool, 0xFF, U * g.PF * (size_t)g.fp_page_bytes);
+    if (e == cudaSuccess) e = cudaMemset(h->st.q_pool, 0xFF, U * g.PQ * (size_t)g.q_page_bytes);
+#endif
     if (e == cudaSuccess) e = cudaMemset(h->st.ledger, 0, U * g.NW);
     if (e == cudaSuccess) e = cudaMemset(h->st.fp_page, 0xFF, U * g.NW * 4);
     if (e == cudaSuccess) e = cudaMemset(h->st.q_page, 0xFF, U * g.NW * 4);

@@ -105,7 +105,8 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
 #pragma unroll
   for (int k = 0; k < NE; ++k) {
     const int e = e0 + wid + 4 * k;
-    old[k] = (e < e1 && e < n && lane == 0) ? score[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] : 0.f;
+    if (e < e1 && e < n && !QE_IN_RANGE((int)(ewin[k] & ENTRY_WINDOW_MASK) < g.NW, a.st.status, CHECK_BOUNDS_WINDOW)) ewin[k] = 0xFFFFFFFFu;
+    old[k] = (e < e1 && e < n && lane == 0 && ewin[k] != 0xFFFFFFFFu) ? score[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] : 0.f;
   }
   __syncthreads();
 
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(COMBINE_THREADS) combine_kernel(const KernelAr
 #pragma unroll
   for (int k = 0; k < NE; ++k) {
     const int e = e0 + wid + 4 * k;
-    const bool live = e < e1 && e < n;
+    const bool live = e < e1 && e < n && ewin[k] != 0xFFFFFFFFu;  // (all ones: a window index the checking build refused)
     const float mass = live ? head_sum(rec[k], e) : 0.f;
     if (live && lane == 0) {
       score[(size_t)u * g.NW + (ewin[k] & ENTRY_WINDOW_MASK)] = old[k] + mass;

@@ -23,6 +23,11 @@ enum : int {
   CHECK_ENTRY_OVERFLOW = 3,
   CHECK_WINDOW_OVERFLOW = 4,
   CHECK_COPY_TIMEOUT = 5,
+  // checking build only (-DQEVICT_DEBUG_BOUNDS): an index read from a table was out of range; the access was skipped
+  CHECK_BOUNDS_ENTRY = 6,    // work-list entry (kind, window or page)
+  CHECK_BOUNDS_PAGE = 7,     // page id in a window table or a list
+  CHECK_BOUNDS_WINDOW = 8,   // window index
+  CHECK_BOUNDS_RECORD = 9,   // migration record
 };
 
 static constexpr int TILE_TOKENS = 32;    // tokens per attention tile
@@ -177,6 +182,17 @@ __device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
 }
 
 __device__ __forceinline__ void record_check(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// Checking build (-DQEVICT_DEBUG_BOUNDS, a library of its own): every page id, window index, work-list entry and
+// migration record that a kernel reads from a table is range-checked before it is used as an index; a value out
+// of range records a code in the device status word and the access is skipped -- no trap, no assert, the context
+// stays usable.  The pools start filled with a NaN pattern in that build, so a read of a page nobody wrote
+// surfaces in the results.  In the normal build QE_IN_RANGE is the constant true and costs nothing.
+#ifdef QEVICT_DEBUG_BOUNDS
+#define QE_IN_RANGE(cond, status, code) ((cond) ? true : (record_check((status), (code)), false))
+#else
+#define QE_IN_RANGE(cond, status, code) true
+#endif
 
 // Programmatic dependent launch: the kernels of a step are enqueued with launch_pdl and begin with
 // pdl_prologue().  The prologue first lets the next kernel of the stream start scheduling its CTAs, then

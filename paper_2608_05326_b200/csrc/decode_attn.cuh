@@ -51,7 +51,7 @@ struct DecodeParams {
   float* ml;              // [n_units][Hq][MAX_SPLITS][2]
   float2* wrec;           // [n_units][EMAX][Hq]
   int32_t* status;
-  int unit0, S, Hq, Hkv, G, EMAX, PF, PQ;
+  int unit0, S, Hq, Hkv, G, EMAX, PF, PQ, NW;
   int e_bound;            // upper bound of every unit's work-list length (host's mirror of the window counts)
   uint32_t fp_page_bytes, q_page_bytes;
   float scale_log2;
@@ -483,9 +483,20 @@ __global__ void __launch_bounds__(DECODE_WARPS * 32, ROPE ? 2 : 3) decode_attn_k
   if (lane < my_cap && first + lane < p.EMAX) my_ent = p.entries[(size_t)u * p.EMAX + first + lane];
   const int n_live = p.n_live[u];
   const int fill = p.open_fill[u];
-  const int my_n = max(0, min(my_cap, n_live - first));
+  int my_n = max(0, min(my_cap, n_live - first));
   // the runs cover the host's bound of the list length: a longer list would be attended to only in part
   if (n_live > p.e_bound && s == 0 && threadIdx.x == 0) record_check(p.status, CHECK_ENTRY_OVERFLOW);
+#ifdef QEVICT_DEBUG_BOUNDS
+  {  // an entry with an impossible kind, window or page ends the warp's run before it
+    const uint32_t kind = my_ent.x >> ENTRY_KIND_SHIFT, win = my_ent.x & ENTRY_WINDOW_MASK;
+    const bool bad = lane < my_n && (kind > KIND_OPEN || win >= (uint32_t)p.NW || my_ent.y >= (uint32_t)(kind == KIND_Q ? p.PQ : p.PF));
+    const unsigned bad_lanes = __ballot_sync(0xffffffffu, bad);
+    if (bad_lanes) {
+      if (lane == 0) record_check(p.status, CHECK_BOUNDS_ENTRY);
+      my_n = min(my_n, __ffs(bad_lanes) - 1);
+    }
+  }
+#endif
   if (lane >= my_n) my_ent = make_uint2(0u, 0u);
 
   // ---- producer: pieces are issued in consumption order into slots 0,1,..,NSLOT-1,0,.. ------------------

@@ -105,7 +105,7 @@ extern "C" QEVICT_API qevict_status qevict_decode_attn_noalloc(qevict_handle h, 
   p.trace = a.trace;
 #endif
   p.unit0 = a.unit0; p.S = choose_splits(h, a.n_units); p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.EMAX = g.EMAX;
-  p.PF = g.PF; p.PQ = g.PQ; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
+  p.PF = g.PF; p.PQ = g.PQ; p.NW = g.NW; p.fp_page_bytes = g.fp_page_bytes; p.q_page_bytes = g.q_page_bytes; p.scale_log2 = g.scale_log2;
   e = h->decode_fn(p, a.n_units, stream);
   if (e != cudaSuccess) { h->broken = k_new != nullptr; h->last_error = std::string("attention: ") + cudaGetErrorString(e); return QEVICT_ERR_CUDA; }
   h->launches++;

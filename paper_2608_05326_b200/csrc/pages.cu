@@ -324,7 +324,11 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
   QE_TRACE_SCOPE(a.trace, 4);
   int32_t* cnt = a.st.mig_count + 2 * (a.unit0 / g.batch);
   const int4* queue = a.st.mig_queue + (size_t)a.unit0 * (g.PF + g.Kq + g.Kf) * 2;
-  const int n_entries = *reinterpret_cast<volatile int32_t*>(cnt + a.mig_parity);
+  int n_entries = *reinterpret_cast<volatile int32_t*>(cnt + a.mig_parity);
+#ifdef QEVICT_DEBUG_BOUNDS
+  if (!QE_IN_RANGE(n_entries >= 0 && (long long)n_entries <= (long long)a.n_units * (g.PF + g.Kq + g.Kf), a.st.status, CHECK_BOUNDS_RECORD))
+    n_entries = 0;
+#endif
   // the next routing event of these units counts in the other counter: nothing reads it before this kernel ends
   if (blockIdx.x == 0 && threadIdx.x == 0) cnt[a.mig_parity ^ 1] = 0;
   const int lane = threadIdx.x & 31;
@@ -340,6 +344,18 @@ __global__ void __launch_bounds__(MIGRATE_THREADS, 6) migrate_kernel(const Kerne
     const int4 r0 = queue[2 * rec], r1 = queue[2 * rec + 1];
     const int u = r0.x, kind = r0.y, ul = u - a.unit0;
     if (kind == 2) continue;
+#ifdef QEVICT_DEBUG_BOUNDS
+    {  // a record whose unit, kind, window or pages are out of range is recorded and skipped
+      bool ok = ul >= 0 && ul < a.n_units && kind >= 0 && kind <= 1 && r0.z >= 0 && r0.z < g.NW;
+      if (kind == 0) ok = ok && r0.w >= -1 && r0.w < g.PF && r1.x >= 0 && r1.x < g.PQ && r1.y >= -1 && r1.y < g.PQ &&
+                          (r0.w >= 0 || (k_prompt && (long long)(r0.z + 1) * g.W <= ctx)) && (r1.y < 0 || r0.w >= 0);
+      else ok = ok && r0.w >= 0 && r0.w < g.PQ && r1.x >= 0 && r1.x < g.PF;
+      if (!ok) {
+        if (lane == 0) record_check(a.st.status, CHECK_BOUNDS_RECORD);
+        continue;
+      }
+    }
+#endif
     char* fp_u = a.st.fp_pool + (size_t)u * g.PF * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;
     char* q_u = a.st.q_pool + (size_t)u * g.PQ * g.q_page_bytes + (size_t)hk * g.q_head_bytes;
     // task coordinates
@@ -382,6 +398,7 @@ __global__ void __launch_bounds__(PAGE_THREADS) copy_prompt_kernel(const KernelA
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
   const int4 it = a.st.copy_list[(size_t)u * g.Kfp + item];
   const int w = it.x, dst = it.y, D = g.D;
+  if (!QE_IN_RANGE(w >= 0 && (long long)(w + 1) * g.W <= ctx && dst >= 0 && dst < g.PF, a.st.status, CHECK_BOUNDS_RECORD)) continue;
   const T* kr = k_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * g.W) * D;
   const T* vr = v_prompt + (((size_t)ul * g.Hkv + hk) * ctx + (size_t)w * g.W) * D;
   char* fb = a.st.fp_pool + ((size_t)u * g.PF + dst) * g.fp_page_bytes + (size_t)hk * g.fp_head_bytes;

@@ -6,6 +6,7 @@
 // tables, the page-owner tables, the decode work list, the unit's pages of both pools (in the library's own
 // page layout -- opaque to the caller, valid for a cache of the same configuration) and the host's mirror of
 // the layer.  Scratch (split partials) and the device status word are not part of it.
+#include <stdlib.h>
 #include <string.h>
 
 #include <string>
@@ -116,16 +117,23 @@ QEVICT_API qevict_status qevict_import_state(qevict_handle h, int32_t layer, int
   if (v->layer_n_windows != v->n_windows || (v->layer_has_open != 0) != (v->open_window >= 0) ||
       v->layer_open_fill != v->open_fill || v->layer_aged < 0 || v->layer_aged > g.aged_cap + 1)
     return fail(h, QEVICT_ERR_INVALID_ARG, "the layer mirror of the snapshot disagrees with its tables");
-  for (int w = 0; w < g.NW; ++w) {
+#ifdef QEVICT_DEBUG_BOUNDS
+  // checking build only: with QEVICT_IMPORT_UNCHECKED set in the environment the index checks below are left
+  // out, so that a test can hand the kernels a table entry that is out of range and see their own checks refuse it
+  const bool unchecked = getenv("QEVICT_IMPORT_UNCHECKED") != nullptr;
+#else
+  const bool unchecked = false;
+#endif
+  for (int w = 0; w < g.NW && !unchecked; ++w) {
     if (v->tier[w] > QEVICT_TIER_SINK || v->ledger[w] > QEVICT_LEDGER_DORMANT || v->fp_page[w] < -1 || v->fp_page[w] >= g.PF ||
         v->q_page[w] < -1 || v->q_page[w] >= g.PQ)
       return fail(h, QEVICT_ERR_INVALID_ARG, "a window table entry of the snapshot is out of range");
   }
-  for (int p = 0; p < g.PF; ++p)
+  for (int p = 0; p < g.PF && !unchecked; ++p)
     if (v->fp_owner[p] < -1 || v->fp_owner[p] >= g.NW) return fail(h, QEVICT_ERR_INVALID_ARG, "a full-precision page owner of the snapshot is out of range");
-  for (int p = 0; p < g.PQ; ++p)
+  for (int p = 0; p < g.PQ && !unchecked; ++p)
     if (v->q_owner[p] < -1 || v->q_owner[p] >= g.NW) return fail(h, QEVICT_ERR_INVALID_ARG, "a quantized page owner of the snapshot is out of range");
-  for (int e = 0; e < v->n_live; ++e) {
+  for (int e = 0; e < v->n_live && !unchecked; ++e) {
     const uint32_t x = v->entries[2 * e], page = v->entries[2 * e + 1], kind = x >> ENTRY_KIND_SHIFT;
     if (kind > KIND_OPEN || (int)(x & ENTRY_WINDOW_MASK) >= g.NW || (int)page >= (kind == KIND_Q ? g.PQ : g.PF))
       return fail(h, QEVICT_ERR_INVALID_ARG, "a work-list entry of the snapshot is out of range");

@@ -157,7 +157,9 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
   } else {
     window = ow0;
     slot = fill0;
+    if (!QE_IN_RANGE(ow0 < g.NW && fill0 >= 0 && fill0 < g.W, a.st.status, CHECK_BOUNDS_WINDOW)) return;
     page = a.st.fp_page[(size_t)u * g.NW + ow0];
+    if (!QE_IN_RANGE(page >= 0 && page < g.PF, a.st.status, CHECK_BOUNDS_PAGE)) return;
   }
   char* pbase = a.st.fp_pool + ((size_t)u * g.PF + page) * g.fp_page_bytes;
   if (is_new) {
@@ -514,6 +516,16 @@ __global__ void __launch_bounds__(NT) route_kernel(const KernelArgs a, int prefi
     n_real = *s_real;
   }
   const int n_cand = min(n_all, sort_cap);
+#ifdef QEVICT_DEBUG_BOUNDS
+  // page ids of the gathered windows index the owner tables below: one out of range is recorded and dropped
+#pragma unroll 1
+  for (int c = tid; c < n_cand; c += NT) {
+    if (!QE_IN_RANGE(cfp[c] >= -1 && cfp[c] < g.PF, a.st.status, CHECK_BOUNDS_PAGE)) cfp[c] = -1;
+    if (!QE_IN_RANGE(cq[c] >= -1 && cq[c] < g.PQ, a.st.status, CHECK_BOUNDS_PAGE)) cq[c] = -1;
+    if (!QE_IN_RANGE(cw[c] >= 0 && cw[c] < g.NW, a.st.status, CHECK_BOUNDS_WINDOW)) cw[c] = 0;
+  }
+  __syncthreads();
+#endif
 
   // ---- rank: score higher first, window index lower first; TopK_{K_f} -> Full, next TopK_{K_q} ->
   // Quantized, remainder -> Evicted -----------------------------------------------------------------
