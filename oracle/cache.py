@@ -61,10 +61,11 @@ E' = the rest.
 
 Pre-RoPE keys (rope_base > 0): see rope.py.
 
-Parity unpinned: the page-id assignment order above is this build's own rule (the
-paper never speaks of pages), so nothing outside this file fixes it; and the
-prefill window scores are an input here (the paper only says that prompt attention
-initialises them), so their definition is pinned by nothing beyond Eq. 1's form.
+Parity unpinned: the prefill window scores are an input here (the paper only says
+that prompt attention initialises them), so their definition is pinned by nothing
+beyond Eq. 1's form.  The page-id assignment order above is this build's own rule
+(the paper never speaks of pages): the tests pin this file to the rule as stated, on
+a run worked by hand, but nothing in the paper fixes the rule itself.
 """
 
 from dataclasses import dataclass

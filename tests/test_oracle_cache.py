@@ -573,3 +573,50 @@ def test_pre_rope_cache_with_full_budget_equals_attention_over_rotated_keys():
     o2, _ = u2.decode_attn(q)
     o1, _ = u.decode_attn(q)
     assert np.abs(o1 - o2).max() > 1e-2
+
+
+# ------------------------------------------------------------------------------ hand-worked pins
+def test_page_ids_at_routing_events_follow_the_stated_rule_on_a_hand_worked_run():
+    """Page hand-out rule of a routing event, worked by hand: all releases of the event first, then the windows
+    that need a page take the free ids in ascending order, in ascending window index (full-precision pages for
+    the windows entering the Full tier, quantized pages for first demotions); a promoted window keeps its
+    quantized page (dormant ledger), a re-demoted window gets no new one."""
+    rng = np.random.default_rng(41)
+    cfg = _small_cfg(k_f=2, k_q=2, ctx_windows=6, extra=4)
+    u, *_ = _prefilled(cfg, rng, ctx_windows=6, scores=np.array([6, 5, 4, 3, 2, 1], dtype=np.float32))
+    # prefill: Full {0, 1} -> full-precision pages 0, 1; Quantized {2, 3} -> quantized pages 0, 1; 4, 5 evicted
+    assert u.fp_page[:6].tolist() == [0, 1, -1, -1, -1, -1] and u.q_page[:6].tolist() == [-1, -1, 0, 1, -1, -1]
+    # event 1: ranks 2, 3, 1, 0 -> Full {2, 3}, Quantized {0, 1}.  Releases: windows 0 and 1 give up full-precision
+    # pages 0 and 1.  Then window 2 takes page 0 and window 3 page 1 (ascending window, ascending free id); the first
+    # demotions 0 and 1 take the free quantized pages 2 and 3 (pages 0, 1 stay with the promoted windows' codes).
+    u.importance[:4] = [1.0, 2.0, 10.0, 9.0]
+    u.rebalance()
+    assert u.tier[:4].tolist() == [TIER_QUANT, TIER_QUANT, TIER_FULL, TIER_FULL]
+    assert u.fp_page[:4].tolist() == [-1, -1, 0, 1] and u.q_page[:4].tolist() == [2, 3, 0, 1]
+    assert u.ledger_flag[:4].tolist() == [LEDGER_ACTIVE, LEDGER_ACTIVE, LEDGER_DORMANT, LEDGER_DORMANT]
+    assert (u.stats["promotions"], u.stats["quantizations"], u.stats["reactivations"]) == (2, 4, 0)
+    # event 2: ranks 1, 3, 0, 2 -> Full {1, 3}, Quantized {0, 2}.  Window 2 is demoted again: its codes are reused
+    # (no new quantized page), its full-precision page 0 is released and goes to window 1, the only window that
+    # needs one.
+    u.importance[:4] = [8.0, 10.0, 1.0, 9.0]
+    u.rebalance()
+    assert u.tier[:4].tolist() == [TIER_QUANT, TIER_FULL, TIER_QUANT, TIER_FULL]
+    assert u.fp_page[:4].tolist() == [-1, 0, -1, 1] and u.q_page[:4].tolist() == [2, 3, 0, 1]
+    assert u.ledger_flag[:4].tolist() == [LEDGER_ACTIVE, LEDGER_DORMANT, LEDGER_ACTIVE, LEDGER_DORMANT]
+    assert (u.stats["promotions"], u.stats["quantizations"], u.stats["reactivations"]) == (3, 4, 1)
+    assert u.fp_owner[:2].tolist() == [1, 3] and u.q_owner[:4].tolist() == [2, 3, 0, 1]
+
+
+def test_decayed_score_is_folded_with_each_float32_operation_rounded_on_its_own():
+    """S <- lambda S + u in float32, product rounded, then sum rounded (worked by hand): lambda = 0.75,
+    S = 1 + 3 ulp (ulp = 2^-23), u = 2^-26.  The exact product 0.75 + 4.5 * 2^-24 is a tie and rounds to the even
+    0.75 + 4 * 2^-24; adding u gives 0.75 + 4.25 * 2^-24, which rounds to 0.75 + 4 * 2^-24.  A fused
+    multiply-add would see 0.75 + 4.75 * 2^-24 and return 0.75 + 5 * 2^-24."""
+    rng = np.random.default_rng(42)
+    cfg = OracleConfig(4, 2, 64, "fp16", 32, 4, 32, 2, 2, 10 * 32, aged_windows=2, rank_mode=1, rank_param=0.75)
+    u, *_ = _prefilled(cfg, rng, ctx_windows=6, scores=np.array([6, 5, 4, 3, 2, 1], dtype=np.float32))
+    u.importance[0] = 1.0 + 3 * 2.0 ** -23
+    u.event_mass[0] = 2.0 ** -26
+    u.fold_event_mass()
+    assert u.importance[0] == 0.75 + 4 * 2.0 ** -24
+    assert u.importance[0] != 0.75 + 5 * 2.0 ** -24 and u.event_mass[0] == 0.0

@@ -78,3 +78,17 @@ def test_execution_datatype_variant_stays_within_its_rounding_bound(dtype, ulp):
     # and a wrong sign or a swapped table would not pass: the error against the inverse rotation is large
     wrong = rotate_exact(k, -pos, 5e5)
     assert np.abs(r - wrong).max() > 0.5
+
+
+def test_execution_datatype_rotation_bit_for_bit_on_a_hand_worked_pair():
+    """d = 2 (one pair, theta = 1), position 1, bf16, every rounding worked by hand (two of them are ties):
+    cos 1 = 0.5403023 -> 0.5390625, sin 1 = 0.8414710 -> 0.83984375; (x, y) = (1.5, 2.5):
+      x c = 0.80859375 (exact)             y s = 2.099609375 -> 2.09375
+      x' = RN(0.80859375 - 2.09375) = RN(-1.28515625), a tie -> -1.28125 (even)
+      y c = 1.34765625, a tie -> 1.34375   x s = 1.259765625 -> 1.2578125
+      y' = RN(1.34375 + 1.2578125) = RN(2.6015625), a tie -> 2.59375
+    Unrounded products would give x' = RN(-1.291015625) = -1.2890625 instead."""
+    r = apply_rope(np.array([[1.5, 2.5]]), [1], 10000.0, "bf16")
+    assert r.tolist() == [[-1.28125, 2.59375]]
+    r0 = apply_rope(np.array([[1.5, 2.5]]), [0], 10000.0, "bf16")
+    assert r0.tolist() == [[1.5, 2.5]]
