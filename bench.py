@@ -419,7 +419,8 @@ def run_ours(args, rank, world):
     if also:
         line["also"] = {"workload": also["workload"], "value": sharding.aggregate_steps_per_second(world, K, also["ms"]),
                         "unit": UNIT, "ms_per_step": also["ms"] / K, "repeats": also["repeats"], "roofline": also["roofline"],
-                        "kernel_us_per_step": also["kernel_us_per_step"], "gpu_launches": also["launches"]}
+                        "kernel_us_per_step": also["kernel_us_per_step"], "gpu_launches": also["launches"],
+                        "clocks": also["clocks"]}
         if "interval_w" in also:
             line["also"]["rebalance_every_window"] = also["interval_w"]
     return line, wl
@@ -464,9 +465,10 @@ def _cpu_seconds():
     return t.user + t.system
 
 
-def time_oracle(wl, n_steps, warmup, budget_s):
+def time_oracle(wl, n_steps, warmup, budget_s, one_thread_s=0.0):
     """Times the CPU oracle, as it stands, on unit 0 of the workload: `n_steps` decode + rebalance steps
-    (at most `budget_s` seconds).  Returns (whole-workload steps/s, description)."""
+    (at most `budget_s` seconds).  Returns (whole-workload steps/s, description, steps, seconds, cores kept busy,
+    whole-workload steps/s with the BLAS pool limited to one thread over a further `one_thread_s` seconds or None)."""
     import numpy as np
 
     from oracle import OracleConfig, UnitOracle
@@ -500,12 +502,30 @@ def time_oracle(wl, n_steps, warmup, budget_s):
     unit_steps_per_s = done / dt
     value = unit_steps_per_s / wl.n_units
     sample = "unit 0 of %d, %d decode+rebalance steps in %.1f s" % (wl.n_units, done, dt)
-    return value, sample, done, dt, busy
+    one = None
+    if one_thread_s > 0:
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                n1, t1 = 0, time.perf_counter()
+                while t < q.shape[0] and time.perf_counter() - t1 < one_thread_s:
+                    orc.decode_attn(q[t], kn[t], vn[t])
+                    if (t + 1) % wl.rebalance_interval == 0:
+                        orc.rebalance()
+                    t += 1; n1 += 1
+                if n1:
+                    one = n1 / (time.perf_counter() - t1) / wl.n_units
+        except Exception:
+            one = None
+    return value, sample, done, dt, busy, one
 
 
-def cpu_baseline_record(value, sample, busy):
-    return {"value": value, "unit": UNIT, "cores": max(1, round(busy)), "kind": "oracle", "sample": sample,
-            "cores_busy_avg": round(busy, 2), "blas_threads": oracle_threads(), "host_cores": os.cpu_count()}
+def cpu_baseline_record(value, sample, busy, one_thread=None):
+    rec = {"value": value, "unit": UNIT, "cores": max(1, round(busy)), "kind": "oracle", "sample": sample,
+           "cores_busy_avg": round(busy, 2), "blas_threads": oracle_threads(), "host_cores": os.cpu_count()}
+    if one_thread is not None:
+        rec["value_one_thread"] = one_thread  # the same oracle with the BLAS pool limited to one thread
+    return rec
 
 
 def run_reference(args, rank):
@@ -513,7 +533,7 @@ def run_reference(args, rank):
         return None
     K, W = args.steps, args.warmup
     wl = make_workload(args, max(W + K, 8))
-    value, sample, done, dt, busy = time_oracle(wl, K, W, budget_s=180.0)
+    value, sample, done, dt, busy, _ = time_oracle(wl, K, W, budget_s=180.0)
     return {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": done,
         "warmup": W, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -601,8 +621,9 @@ def main():
         line, wl = res
         if not args.timeline and not args.no_cpu_baseline and world >= 1:
             small = replace(wl, steps=256, seed=wl.seed)
-            value, sample, _, _, busy = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds)
-            line["cpu_baseline"] = cpu_baseline_record(value, sample, busy)
+            value, sample, _, _, busy, one = time_oracle(small, 1000, 1, budget_s=args.cpu_seconds * 2 / 3,
+                                                         one_thread_s=args.cpu_seconds / 3)
+            line["cpu_baseline"] = cpu_baseline_record(value, sample, busy, one)
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
