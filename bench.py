@@ -380,7 +380,10 @@ def run_ours(args, rank, world):
         build.build(trace=args.timeline)  # no-op when the in-tree library is newer than its sources
     if world > 1:
         torch.distributed.barrier()
-    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    if os.environ.get("QEVICT_BENCH_SHARE_GPU"):  # test aid: several ranks on one device (the ranks never wait on one another on the GPU)
+        local %= torch.cuda.device_count()
+    dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     K, W = args.steps, args.warmup
     wl = sharding.rank_workload(make_workload(args, K), rank)  # every rank owns its own sequences (weak scaling, no exchange)
@@ -628,7 +631,9 @@ def main():
         return
     if world > 1:
         os.environ.setdefault("NCCL_DEBUG", "WARN")
-        torch.distributed.init_process_group("nccl")
+        # NCCL is used for the barrier and the max over ranks only; QEVICT_BENCH_BACKEND=gloo lets a test run two
+        # ranks on one device (NCCL refuses two ranks per GPU)
+        torch.distributed.init_process_group(os.environ.get("QEVICT_BENCH_BACKEND", "nccl"))
     res = run_ours(args, rank, world)
     if rank == 0:
         line, wl = res

@@ -19,6 +19,8 @@ def max_over_ranks(values, device="cpu"):
     """Element-wise maximum over all ranks of a list of floats (identity without a process group)."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
         return [float(v) for v in values]
+    if dist.get_backend() == "gloo":
+        device = "cpu"
     t = torch.tensor(list(values), dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return [float(x) for x in t.tolist()]

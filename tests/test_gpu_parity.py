@@ -514,3 +514,23 @@ def test_pre_rope_keys_change_the_result():
     ob = b.step(append=True, check_mass=False)
     assert (oa.float() - ob.float()).abs().max() > 1e-2
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("kw,gain", [
+    (dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2), 6.0),
+    (dict(dtype="fp16", head_dim=64, n_q_heads=7, n_kv_heads=1, quant_bits=2), 8.0),
+    (dict(dtype="bf16", head_dim=128, n_q_heads=4, n_kv_heads=1, window=64, group_size=64, quant_bits=2), 0.02),
+], ids=["bf16-sharp", "fp16-gqa7-sharp", "w64-flat"])
+def test_sharp_and_flat_attention_distributions(kw, gain):
+    """Queries scaled up (logits spread over hundreds of log2 units: a few tokens take all the mass, and the running
+    reference exponent of the online softmax is overtaken again and again) and down (every token matters
+    equally): outputs, window mass and routing must stay within the same tolerances."""
+    ls = _lockstep()
+    wl = _small("sharp", steps=24, context=2048, fp_budget_windows=6, q_budget_windows=12, **kw)
+    run = ls.LockstepRun(wl)
+    for u in list(run.queries):
+        run.queries[u] = (run.queries[u].float() * gain).to(run.queries[u].dtype)
+    for _ in range(wl.steps):
+        run.step(append=True)
+    run.rebalance(full_check=True)
+    run.close()

@@ -165,3 +165,30 @@ def test_device_is_left_as_the_caller_had_it():
     finally:
         torch.cuda.set_device(0)
     run.close()
+
+
+def test_bench_under_a_launcher_with_two_ranks():
+    """The N > 1 path of bench.py for real: two ranks under torch.distributed.run, each with its own sequences; both
+    on this one device and over gloo (NCCL refuses two ranks per GPU; the ranks exchange nothing but a barrier and a
+    max of their times, and never wait on one another on the GPU).  Rank 0 prints one line for two ranks."""
+    import json
+    import os
+    import socket
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    env.update(QEVICT_BENCH_BACKEND="gloo", QEVICT_BENCH_SHARE_GPU="1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.join(root, "bench.py"), "--gpus", "2", "--config", "0", "--steps", "8",
+           "--warmup", "3", "--settle-steps", "8", "--no-cpu-baseline"]
+    r = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=900)
+    assert r.returncode == 0, r.stderr[-3000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout[-2000:]
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak" and line["value"] > 0 and line["gpu_launches"] > 0
+    assert line["e2e"]["value"] > 0 and line["roofline"]["kernel_launches_timed"] == 8
