@@ -272,6 +272,13 @@ QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* 
 /* Counters of one layer (layer == -1: all layers), summed over its sequences.  Synchronises. */
 QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict_stats* out);
 
+/* Synchronises the device and reports the device status word: QEVICT_OK, or QEVICT_ERR_DEVICE_CHECK if a kernel
+ * of this cache has recorded a failed internal check since creation (pool exhausted, work list longer than the
+ * host's bound, a page copy that did not arrive in time; in the checking build also an index out of range).
+ * *code (may be NULL) receives the recorded code, 0 if none; the first failure is the one kept.  The same report
+ * comes with qevict_get_stats. */
+QEVICT_API qevict_status qevict_check_device(qevict_handle h, int32_t* code);
+
 /* Tables of one unit, written to DEVICE buffers sized for max_context / W windows (any may be NULL):
  * n_windows int32[1], tier uint8[], ledger uint8[], fp_page int32[], q_page int32[] (-1 = none),
  * importance float32[].  Enqueues only. */

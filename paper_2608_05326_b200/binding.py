@@ -102,6 +102,7 @@ _SIGNATURES = {
     "qevict_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(qevict_state_view)]),
     "qevict_import_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(qevict_state_view)]),
     "qevict_get_stats": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(qevict_stats)]),
+    "qevict_check_device": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
     "qevict_export_tables": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 7),
     "qevict_export_last_mass": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "qevict_export_fp_page": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -303,6 +304,13 @@ def qevict_get_stats(h, layer=-1):
     return {n: getattr(st, n) for n, _ in qevict_stats._fields_}
 
 
+def qevict_check_device(h):
+    """Synchronises; raises QEvictError(DEVICE_CHECK) if a kernel recorded a failed check, else returns 0."""
+    code = C.c_int32(0)
+    _check(lib().qevict_check_device(h, C.byref(code)), h)
+    return code.value
+
+
 def qevict_launch_count(h):
     return lib().qevict_launch_count(h)
 
@@ -391,6 +399,9 @@ class QEvictCache:
 
     def launch_count(self):
         return qevict_launch_count(self.handle)
+
+    def check_device(self):
+        return qevict_check_device(self.handle)
 
     # -- exports (parity checks, snapshots) -------------------------------------------------------
     def export_state(self, layer, seq):

@@ -721,6 +721,21 @@ QEVICT_API qevict_status qevict_get_stats(qevict_handle h, int32_t layer, qevict
   return QEVICT_OK;
 }
 
+QEVICT_API qevict_status qevict_check_device(qevict_handle h, int32_t* code) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  QE_DEVICE(h);
+  QE_CUDA(h, cudaDeviceSynchronize());
+  int32_t status = 0;
+  QE_CUDA(h, cudaMemcpy(&status, h->st.status, 4, cudaMemcpyDeviceToHost));
+  if (code) *code = status;
+  if (status != 0) {
+    char buf[96];
+    snprintf(buf, sizeof(buf), "device check %d failed", status);
+    return fail(h, QEVICT_ERR_DEVICE_CHECK, buf);
+  }
+  return QEVICT_OK;
+}
+
 static bool unit_of(qevict_handle h, int layer, int seq, int* u) {
   if (layer < 0 || layer >= h->geo.n_layers || seq < 0 || seq >= h->geo.batch) return false;
   *u = layer * h->geo.batch + seq;

@@ -64,11 +64,12 @@ _FIRE = """
         vn = torch.stack([workloads.gen_new_kv(wl, u)[1] for u in range(2)], 1).to(dev)
         cache.decode_attn(0, q[0], kn[0], vn[0])
         cache.rebalance(0)
-        assert cache.stats()["n_full"] == 8  # no check has fired on good tables
+        assert cache.stats()["n_full"] == 8 and cache.check_device() == 0  # no check has fired on good tables
         return cache, q, kn, vn
 
     def expect_check(cache, code):
         try:
+            cache.check_device()
             cache.stats()
         except binding.QEvictError as e:
             assert e.status == 6 and ("check %d " % code) in str(e), str(e)
