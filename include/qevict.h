@@ -212,12 +212,12 @@ QEVICT_API qevict_status qevict_decode_attn(qevict_handle h, int32_t layer, cons
                                  const void* v_new, void* out, void* stream);
 
 /* The same step with HOST buffers (pageable or page-locked): brings q, k_new, v_new to the device, runs the
- * step, returns `out` to the host and synchronises the stream.  q always goes through a copy into device
- * memory (every CTA of the attention kernel reads it).  Page-locked buffers the device can address (any
- * cudaHostAlloc / cudaHostRegister memory under unified addressing) are otherwise used in place: the append
- * kernel reads k_new and v_new from them and the merge kernel writes `out` into them over the bus, which
- * saves three copy operations per step; pageable buffers take staged copies.  The bytes that cross the bus
- * are the same either way. */
+ * step, returns `out` to the host and synchronises the stream.  q always ends up in device memory before the
+ * attention kernel runs (every CTA of that kernel reads it).  Page-locked buffers the device can address (any
+ * cudaHostAlloc / cudaHostRegister memory under unified addressing) need no copy operation at all: the append
+ * kernel reads k_new and v_new from them in place and, in the same launch, brings q into the cache's staging
+ * buffer; the merge kernel writes `out` into the host buffer over the bus.  Pageable buffers, and q when there
+ * is no new token, take staged copies.  The bytes that cross the bus are the same either way. */
 QEVICT_API qevict_status qevict_decode_attn_host(qevict_handle h, int32_t layer, const void* q_host,
                                       const void* k_new_host, const void* v_new_host, void* out_host,
                                       void* stream);

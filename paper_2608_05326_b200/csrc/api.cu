@@ -297,8 +297,10 @@ namespace {
     if (e__ != cudaSuccess) return fail(h, QEVICT_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
   } while (0)
 
+// q_host_alias != nullptr (only with k_new): `q` is the handle's staging buffer and the append kernel fills it from
+// that page-locked host buffer, so the caller needs no copy operation of its own for the queries.
 qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void* k_new, const void* v_new, void* out,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, const void* q_host_alias = nullptr) {
   int l0, l1;
   qevict_status pst;
   if (const char* msg = decode_precheck(h, layer, q, k_new, v_new, out, &l0, &l1, &pst)) return fail(h, pst, msg);
@@ -306,7 +308,7 @@ qevict_status decode_impl(qevict_handle h, int layer, const void* q, const void*
   QE_DEVICE(h);
   const KernelArgs a = make_args(h, l0, l1);
   if (k_new) {
-    QE_CUDA(h, timed_launch(h, 0, stream, [&] { return launch_append(a, k_new, v_new, stream); }));
+    QE_CUDA(h, timed_launch(h, 0, stream, [&] { return launch_append(a, k_new, v_new, stream, q_host_alias, q_host_alias ? const_cast<void*>(q) : nullptr); }));
     for (int l = l0; l < l1; ++l) {
       LayerMirror& m = h->layers[l];
       if (!m.has_open) { m.has_open = true; m.open_fill = 0; m.n_windows++; }
@@ -627,7 +629,6 @@ static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void
     if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
     return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
   };
-  QE_CUDA(h, cudaMemcpyAsync(h->stage_q, q_host, qb, cudaMemcpyHostToDevice, s));
   const void* k_dev = nullptr;
   const void* v_dev = nullptr;
   if (k_new_host) {
@@ -640,8 +641,12 @@ static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void
       v_dev = h->stage_v;
     }
   }
+  // the queries: every CTA of the attention kernel reads them, so they go to device memory first -- through the
+  // append kernel when there is one and the buffer is page-locked (no copy operation at all), else by a copy
+  const void* q_alias = k_new_host ? device_alias(q_host) : nullptr;
+  if (!q_alias) QE_CUDA(h, cudaMemcpyAsync(h->stage_q, q_host, qb, cudaMemcpyHostToDevice, s));
   void* out_dev = device_alias(out_host);
-  const qevict_status st = decode_impl(h, layer, h->stage_q, k_dev, v_dev, out_dev ? out_dev : h->stage_out, s);
+  const qevict_status st = decode_impl(h, layer, h->stage_q, k_dev, v_dev, out_dev ? out_dev : h->stage_out, s, q_alias);
   if (st != QEVICT_OK) return st;
   if (!out_dev) QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
   if (sync) QE_CUDA(h, cudaStreamSynchronize(s));

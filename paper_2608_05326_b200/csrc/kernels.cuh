@@ -23,7 +23,9 @@ cudaError_t launch_rope_rotate_prompt(const Geometry& g, const void* k, void* ou
 
 // decode step ---------------------------------------------------------------------------------------
 // A0: append one token per unit to its open window (opens one first if needed, zeroing the page).
-cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s);
+// q_src / q_dst (optional): the kernel also copies the call's queries from page-locked host memory into device memory.
+cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s,
+                          const void* q_src = nullptr, void* q_dst = nullptr);
 // A2: merge the split partials into `out`, add each window's mass to its score in fixed head order.
 cudaError_t launch_combine(const KernelArgs& a, int n_splits, int e_bound, void* out, cudaStream_t s);
 

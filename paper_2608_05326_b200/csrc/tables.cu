@@ -104,9 +104,13 @@ __device__ int block_compact(int n, int* scratch, Pred pred, Emit emit) {
 // ------------------------------------------------------------------------------------------ append
 // One CTA per unit.  Global memory is waited on twice: the unit's scalars together with the new token,
 // then the open window's page id; everything else is stores.
+// q_src != nullptr: the step's queries are also brought from `q_src` (page-locked host memory the device can
+// address) into `q_dst` (device memory), [units of the call][q_vecs] 16-byte pieces: the host entry point then
+// needs no separate copy operation for them, and the attention kernel finds them in device memory.
 template <class T>
 __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T* __restrict__ k_new,
-                                                     const T* __restrict__ v_new) {
+                                                     const T* __restrict__ v_new, const uint4* __restrict__ q_src,
+                                                     uint4* __restrict__ q_dst, int q_vecs) {
   const Geometry& g = a.geo;
   const int ul = blockIdx.x, u = a.unit0 + ul, tid = threadIdx.x;
   __shared__ int s_page;
@@ -127,6 +131,22 @@ __global__ void __launch_bounds__(128) append_kernel(const KernelArgs a, const T
     if (v < nvec) {
       kx[i] = __ldg(reinterpret_cast<const uint4*>(k_new + (size_t)ul * g.Hkv * g.D) + v);
       vx[i] = __ldg(reinterpret_cast<const uint4*>(v_new + (size_t)ul * g.Hkv * g.D) + v);
+    }
+  }
+  if (q_src) {  // all loads of a round are issued before the first store waits for one
+#pragma unroll 1
+    for (int base = 0; base < q_vecs; base += 4 * 128) {
+      uint4 qx[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int v = base + tid + i * 128;
+        if (v < q_vecs) qx[i] = __ldg(q_src + (size_t)ul * q_vecs + v);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int v = base + tid + i * 128;
+        if (v < q_vecs) q_dst[(size_t)ul * q_vecs + v] = qx[i];
+      }
     }
   }
   int page, slot, window;
@@ -865,11 +885,14 @@ cudaError_t route_prepare(size_t max_smem) {
   return e;
 }
 
-cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s) {
+cudaError_t launch_append(const KernelArgs& a, const void* k_new, const void* v_new, cudaStream_t s, const void* q_src,
+                          void* q_dst) {
+  const int q_vecs = a.geo.Hq * a.geo.D / 8;
   if (a.geo.dtype == QEVICT_DTYPE_FP16)
-    return launch_pdl(append_kernel<__half>, dim3(a.n_units), dim3(128), 0, s, a, (const __half*)k_new, (const __half*)v_new);
+    return launch_pdl(append_kernel<__half>, dim3(a.n_units), dim3(128), 0, s, a, (const __half*)k_new, (const __half*)v_new,
+                      (const uint4*)q_src, (uint4*)q_dst, q_vecs);
   return launch_pdl(append_kernel<__nv_bfloat16>, dim3(a.n_units), dim3(128), 0, s, a, (const __nv_bfloat16*)k_new,
-                    (const __nv_bfloat16*)v_new);
+                    (const __nv_bfloat16*)v_new, (const uint4*)q_src, (uint4*)q_dst, q_vecs);
 }
 
 cudaError_t launch_key_norm_scores(const KernelArgs& a, const void* k_prompt, int ctx, int n_prompt, cudaStream_t s) {
