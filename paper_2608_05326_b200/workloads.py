@@ -7,6 +7,12 @@ method's arithmetic (no attention, no quantizer, no routing): both the CUDA
 path and the CPU oracle consume the tensors produced here, so they provably see
 the same bytes.  Everything is drawn from `torch.Generator` streams keyed by
 (seed, unit, stream); a "unit" is one (layer, sequence) pair, unit = layer * batch + seq.
+
+Two helpers here restate a definition of the method because the workload DEFINITIONS need it, not because anything
+is checked with them: `Workload.fp_window_bytes / q_window_bytes` (bytes of a window in either tier: configuration 4
+sizes its quantized tier "to equal memory", and bench.py counts algorithmic bytes) and `initial_quantized_set` (which
+windows a ranking puts in the quantized tier at prefill: configuration 3 steers a tenth of its queries at windows
+"previously quantized").  Neither the CUDA path nor the oracle calls them.
 """
 
 from dataclasses import dataclass, replace
