@@ -364,13 +364,13 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
                                              float (&l_part)[2], float (&wsum)[2], float (&o)[MT][4],
                                              uint32_t (&pa)[2][2], uint32_t (&pb)[2][2]) {
   const int g = lane >> 2;
-  float x[2][2][2];  // [token block][row half][head]
+  float x[2][2][2];  // raw logits, [token block][row half][head]; the softmax scale is folded into the exponent below
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
-      x[mt][r][0] = s[mt][2 * r] * scale_log2;
-      x[mt][r][1] = s[mt][2 * r + 1] * scale_log2;
+      x[mt][r][0] = s[mt][2 * r];
+      x[mt][r][1] = s[mt][2 * r + 1];
     }
   }
   if (ntok < 32) {  // only the open window has unfilled token slots
@@ -382,9 +382,9 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
       }
     }
   }
-  float lm[2];
+  float lm[2];  // the lane's largest scaled logit per head (the scale is positive)
 #pragma unroll
-  for (int h = 0; h < 2; ++h) lm[h] = fmaxf(fmaxf(x[0][0][h], x[0][1][h]), fmaxf(x[1][0][h], x[1][1][h]));
+  for (int h = 0; h < 2; ++h) lm[h] = fmaxf(fmaxf(x[0][0][h], x[0][1][h]), fmaxf(x[1][0][h], x[1][1][h])) * scale_log2;
   if (__any_sync(0xffffffffu, lm[0] > m_run[0] + REF_SLACK || lm[1] > m_run[1] + REF_SLACK)) {
     float alpha[2];
 #pragma unroll
@@ -413,7 +413,7 @@ __device__ __forceinline__ void softmax_tile(float (&s)[2][4], int ntok, float s
     for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
-        p[mt][r][h] = ex2(x[mt][r][h] - m_run[h]);
+        p[mt][r][h] = ex2(fmaf(x[mt][r][h], scale_log2, -m_run[h]));
         rs += p[mt][r][h];
       }
     }
