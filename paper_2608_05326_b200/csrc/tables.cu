@@ -912,7 +912,9 @@ cudaError_t launch_route(const KernelArgs& a, int prefill, int sort_cap, cudaStr
   // more threads only pay when there are enough candidates (every phase is a loop over them): from 129 candidate
   // slots on, 512 threads rank them in one round (two lanes per candidate) instead of two: route 9.1 -> 7.7 us on
   // the 32k configuration (193 candidates), 12.7 -> 10.4 us on the 128k one
-  if (sort_cap > 128)
+  // (only while the launch is a single wave of CTAs: with hundreds of units the kernel is bound by throughput, not
+  // by one CTA's latency, and the narrower CTAs pack better: 512 units of config 2 took 38 instead of 27 us)
+  if (sort_cap > 512 || (sort_cap > 128 && a.n_units <= 160))
     return launch_pdl(route_kernel<ROUTE_MAX_THREADS>, dim3(a.n_units), dim3(ROUTE_MAX_THREADS), route_smem_bytes(a.geo, sort_cap), s, a,
                       prefill, sort_cap);
   return launch_pdl(route_kernel<256>, dim3(a.n_units), dim3(256), route_smem_bytes(a.geo, sort_cap), s, a, prefill, sort_cap);
