@@ -326,15 +326,13 @@ def measure_workload(args, wl, rank, world, dev, K, W, with_e2e, timeline=False)
         barrier()
         t0 = time.perf_counter()
         # every step: inputs leave pinned host memory, the step and its routing event are enqueued, and the host
-        # waits until the result is in host memory before it sends the next step's inputs (the final barrier
-        # waits for the last routing event)
-        got = torch.cuda.Event()
+        # waits until the result is in host memory (qevict_wait_result: an event behind the write of `out`) before it
+        # sends the next step's inputs (the final barrier waits for the last routing event)
         for i in range(K):
             cache.decode_attn_host_async(-1, qh[i], knh[i] if append else None, vnh[i] if append else None, outh)
-            got.record()          # the result is in host memory once this event has passed
             if (state["t"] + i + 1) % R == 0:
                 cache.rebalance(-1)
-            got.synchronize()     # the routing event keeps running while the host turns around
+            cache.wait_result()   # the result is in host memory; the routing event keeps running while the host turns around
         barrier()
         e2e_s = sharding.max_over_ranks([time.perf_counter() - t0], device=dev)[0]
         state["t"] += K

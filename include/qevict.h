@@ -230,6 +230,12 @@ QEVICT_API qevict_status qevict_decode_attn_host_async(qevict_handle h, int32_t 
                                                        const void* k_new_host, const void* v_new_host,
                                                        void* out_host, void* stream);
 
+/* Blocks the calling thread until the `out_host` of this cache's most recent qevict_decode_attn_host_async call is
+ * complete in host memory -- and no longer: work enqueued behind that call (the step's routing event, say) keeps
+ * running.  The call records an event behind the last operation that writes `out_host`; this waits for it.
+ * QEVICT_ERR_BAD_STATE if no such call has been made. */
+QEVICT_API qevict_status qevict_wait_result(qevict_handle h);
+
 /* The same decode step for callers that must not allocate device memory (the paper has no counterpart:
  * this is a deployment variant of qevict_decode_attn, not a step of the method).
  *

@@ -97,6 +97,7 @@ _SIGNATURES = {
     "qevict_decode_attn_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_host_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "qevict_decode_attn_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "qevict_wait_result": (C.c_int, [C.c_void_p]),
     "qevict_rebalance": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "qevict_state_layout_of": (C.c_int, [C.c_void_p, C.POINTER(qevict_state_layout)]),
     "qevict_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(qevict_state_view)]),
@@ -203,6 +204,11 @@ def qevict_decode_attn_noalloc(h, layer, q, k_new, v_new, out, stream=None):
     """qevict_decode_attn with the attention scratch in the library's built-in device array: for callers
     that must not allocate device memory.  Raises QEvictError(NO_MEMORY) if the call's scratch does not fit."""
     _check(lib().qevict_decode_attn_noalloc(h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream)), h)
+
+
+def qevict_wait_result(h):
+    """Blocks until the result of the last qevict_decode_attn_host_async call is in host memory."""
+    _check(lib().qevict_wait_result(h), h)
 
 
 def qevict_rebalance(h, layer, stream=None):
@@ -371,6 +377,9 @@ class QEvictCache:
 
     def decode_attn_host_async(self, layer, q, k_new, v_new, out, stream=None):
         qevict_decode_attn_host_async(self.handle, layer, q, k_new, v_new, out, stream)
+
+    def wait_result(self):
+        qevict_wait_result(self.handle)
 
     def rebalance(self, layer, stream=None):
         qevict_rebalance(self.handle, layer, stream)

@@ -488,6 +488,7 @@ QEVICT_API qevict_status qevict_create(const qevict_config* cfg, void* device_me
 QEVICT_API qevict_status qevict_destroy(qevict_handle h) {
   if (!h) return QEVICT_ERR_INVALID_ARG;
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  if (h->out_ready) cudaEventDestroy(h->out_ready);
   delete h;
   return QEVICT_OK;
 }
@@ -649,7 +650,13 @@ static qevict_status decode_host_impl(qevict_handle h, int32_t layer, const void
   const qevict_status st = decode_impl(h, layer, h->stage_q, k_dev, v_dev, out_dev ? out_dev : h->stage_out, s, q_alias);
   if (st != QEVICT_OK) return st;
   if (!out_dev) QE_CUDA(h, cudaMemcpyAsync(out_host, h->stage_out, qb, cudaMemcpyDeviceToHost, s));
-  if (sync) QE_CUDA(h, cudaStreamSynchronize(s));
+  if (sync) {
+    QE_CUDA(h, cudaStreamSynchronize(s));
+  } else {
+    // qevict_wait_result waits for exactly this point of the stream, whatever the caller enqueues behind it
+    if (!h->out_ready) QE_CUDA(h, cudaEventCreateWithFlags(&h->out_ready, cudaEventDisableTiming));
+    QE_CUDA(h, cudaEventRecord(h->out_ready, s));
+  }
   return QEVICT_OK;
 }
 
@@ -662,6 +669,13 @@ QEVICT_API qevict_status qevict_decode_attn_host_async(qevict_handle h, int32_t 
                                                        const void* k_new_host, const void* v_new_host, void* out_host,
                                                        void* stream) {
   return decode_host_impl(h, layer, q_host, k_new_host, v_new_host, out_host, stream, false);
+}
+
+QEVICT_API qevict_status qevict_wait_result(qevict_handle h) {
+  if (!h) return QEVICT_ERR_INVALID_ARG;
+  if (!h->out_ready) return fail(h, QEVICT_ERR_BAD_STATE, "no qevict_decode_attn_host_async call has been made on this cache");
+  QE_CUDA(h, cudaEventSynchronize(h->out_ready));
+  return QEVICT_OK;
 }
 
 QEVICT_API qevict_status qevict_rebalance(qevict_handle h, int32_t layer, void* stream) {

@@ -58,6 +58,7 @@ struct qevict_ctx {
   std::vector<cudaEvent_t> ev_pool;   // start/stop pairs, reused
   std::vector<int> ev_kind;           // kernel index of each pair
   size_t ev_used = 0;
+  cudaEvent_t out_ready = nullptr;  // recorded behind the last operation that writes a host entry point's `out`
   char* stage_q = nullptr;    // device staging for the host-buffer entry point
   char* stage_k = nullptr;
   char* stage_v = nullptr;
