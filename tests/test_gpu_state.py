@@ -192,3 +192,41 @@ def test_bench_under_a_launcher_with_two_ranks():
     line = json.loads(lines[0])
     assert line["n_gpus"] == 2 and line["scaling"] == "weak" and line["value"] > 0 and line["gpu_launches"] > 0
     assert line["e2e"]["value"] > 0 and line["roofline"]["kernel_launches_timed"] == 8
+
+
+def test_two_caches_on_two_streams_give_the_same_bits_as_one_after_the_other():
+    """Independent caches stepped on different streams (so that one cache's table kernels run under the other's
+    attention kernel) must not disturb each other: same outputs, same tables as the same caches stepped one after
+    the other on one stream."""
+    ls = _lockstep()
+    wl_a = _wl("streams-a", n_layers=2, steps=24)
+    wl_b = _wl("streams-b", n_layers=2, steps=24, quant_bits=2, fp_budget_windows=3, q_budget_windows=11)
+    serial = [ls.LockstepRun(w, oracle_units=[], score_mode="synthetic") for w in (wl_a, wl_b)]
+    overlapped = [ls.LockstepRun(w, oracle_units=[], score_mode="synthetic") for w in (wl_a, wl_b)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    dev = serial[0].dev
+    torch.cuda.synchronize()
+    for t in range(24):
+        outs_serial = [r.step(append=True, check_mass=False) for r in serial]
+        outs = []
+        for r, s in zip(overlapped, streams):
+            wl = r.wl
+            q = torch.stack([r.queries[u][t] for u in range(wl.n_units)]).reshape(wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim).to(dev)
+            kn = torch.stack([r.new_kv[u][0][t] for u in range(wl.n_units)]).reshape(wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim).to(dev)
+            vn = torch.stack([r.new_kv[u][1][t] for u in range(wl.n_units)]).reshape(wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim).to(dev)
+            torch.cuda.current_stream().synchronize()  # the inputs were produced on the current stream
+            with torch.cuda.stream(s):
+                out = torch.empty_like(q)
+            r.cache.decode_attn(-1, q, kn, vn, out, stream=s)
+            r.cache.rebalance(-1, stream=s)
+            outs.append((out, q, kn, vn))
+        torch.cuda.synchronize()
+        for (out, *_), ref, r in zip(outs, outs_serial, overlapped):
+            assert torch.equal(out.cpu().reshape(r.wl.n_units, r.wl.n_q_heads, r.wl.head_dim), ref), t
+    for a, b in zip(serial, overlapped):
+        for u in range(a.wl.n_units):
+            x = a.cache.export_tables(u // a.wl.batch, u % a.wl.batch)
+            y = b.cache.export_tables(u // b.wl.batch, u % b.wl.batch)
+            for key in x:
+                assert torch.equal(x[key], y[key]), (u, key)
+        a.close(); b.close()
