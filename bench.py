@@ -383,7 +383,7 @@ def measure_two_streams(args, wl, dev, K, W, kbytes):
     cache's attention kernel.  A pattern of the caller's, not of the library: reported beside the headline."""
     from paper_2608_05326_b200 import binding
     half = replace(wl, n_layers=wl.n_layers // 2)
-    total_steps = args.settle_steps + W + (MAX_REPEATS + 1) * K + 2 * wl.window
+    total_steps = args.settle_steps + W + (MAX_REPEATS + 1) * K + max(K, 4 * wl.window) + 3 * wl.window
     n_in = min(total_steps, INPUT_POOL)
     half = replace(half, steps=total_steps)
     groups = []
@@ -405,12 +405,26 @@ def measure_two_streams(args, wl, dev, K, W, kbytes):
         groups.append((cache, q, kn, vn, torch.empty_like(q[0]), torch.cuda.Stream(device=dev)))
     state = {"t": 0}
 
-    def step():
+    def step(interval=1):
         i = state["t"] % n_in
         for cache, q, kn, vn, out, stream in groups:
             cache.decode_attn(-1, q[i], kn[i], vn[i], out, stream=stream)
-            cache.rebalance(-1, stream=stream)
+            if (state["t"] + 1) % interval == 0:
+                cache.rebalance(-1, stream=stream)
         state["t"] += 1
+
+    def timed(n, interval=1):
+        torch.cuda.synchronize()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in groups]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in groups]
+        for ev, g in zip(starts, groups):
+            ev.record(g[5])
+        for _ in range(n):
+            step(interval)
+        for ev, g in zip(ends, groups):
+            ev.record(g[5])
+        torch.cuda.synchronize()
+        return max(starts[0].elapsed_time(e) for e in ends)  # from the first start to the last end
 
     for _ in range(args.settle_steps):
         step()
@@ -418,26 +432,21 @@ def measure_two_streams(args, wl, dev, K, W, kbytes):
     time.sleep(IDLE_AFTER_SETTLE_S)
     for _ in range(W):
         step()
-    reps = []
-    for _ in range(MAX_REPEATS):
-        torch.cuda.synchronize()
-        starts = [torch.cuda.Event(enable_timing=True) for _ in groups]
-        ends = [torch.cuda.Event(enable_timing=True) for _ in groups]
-        for ev, g in zip(starts, groups):
-            ev.record(g[5])
-        for _ in range(K):
-            step()
-        for ev, g in zip(ends, groups):
-            ev.record(g[5])
-        torch.cuda.synchronize()
-        reps.append(max(starts[0].elapsed_time(e) for e in ends))  # from the first start to the last end
+    reps = [timed(K) for _ in range(MAX_REPEATS)]
+    while state["t"] % wl.window:
+        step()
+    n_w = max(K, 4 * wl.window) // wl.window * wl.window
+    ms_w = timed(n_w, interval=wl.window)  # one routing event per filled window
     for g in groups:
         g[0].close()
     ms = statistics.median(reps)
     peak, _ = peak_hbm_gbs()
     gbs = kbytes / (ms / K * 1e-3) / 1e9
+    gbs_w = kbytes / (ms_w / n_w * 1e-3) / 1e9
     return {"caches": 2, "layers_per_cache": half.n_layers, "streams": 2, "steps": K, "repeats": len(reps),
             "ms_per_step": ms / K, "value": K / (ms * 1e-3), "unit": UNIT, "step_frac": gbs / peak, "step_frac_of_8TBs": gbs / 8000.0,
+            "rebalance_every_window": {"rebalance_interval": wl.window, "steps": n_w, "ms_per_step": ms_w / n_w,
+                                       "value": n_w / (ms_w * 1e-3), "step_frac": gbs_w / peak, "step_frac_of_8TBs": gbs_w / 8000.0},
             "what": "two caches of half the layers each on two streams, a routing event after every step: one cache's table "
                     "kernels run under the other's attention kernel"}
 
